@@ -1,0 +1,159 @@
+/*
+ * asi.h -- C ABI of the B200 (sm_100a) ASI library.
+ *
+ * ASI (Activation Subspace Iteration) keeps, for every trained layer, a Tucker
+ * form of the layer's input activation instead of the activation itself:
+ *
+ *     A  ~=  S x_1 U_1 x_2 U_2 ... x_n U_n          (Sec. 3.2, Tucker form)
+ *
+ * with core S in R^{r_1 x .. x r_n} and factors U_m in R^{D_m x r_m} with
+ * orthonormal columns.  Each training step the factors are refreshed by ONE
+ * warm-started subspace iteration per mode (Algorithm 1), and the backward
+ * pass computes the weight gradient from (S, U, dY) without rebuilding A
+ * (appendix "Speedup", cost model C_ASI).
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers unless the name ends in _host.
+ *   - The caller owns every buffer, including the workspace; the library
+ *     allocates no device memory and keeps no mutable state in a plan, so one
+ *     plan may be used from several streams (with distinct workspaces).
+ *   - Tensors are contiguous, row-major: activation [B,C,H,W] (conv) or
+ *     [B,N,Din] / [B,Din] (linear); dY [B,Cout,H',W'] or [..,Dout];
+ *     dW [Cout, C/groups, kh, kw] or [Dout, Din]; core [r_1,..,r_n].
+ *   - "U" buffers hold all factors back to back: U_m is row-major
+ *     [D_m x r_m] and starts at element asi_plan_info_t.u_offset[m].
+ *   - act and dY have the plan's in_dtype (fp32 or bf16); everything else is
+ *     fp32.  Accumulation is fp32 or wider.
+ *   - Calls are asynchronous on `stream`.  Errors the host can see are
+ *     returned immediately and nothing is enqueued.  Conditions only the
+ *     device can see (a rank-deficient A_m A_m^T U_m) are written to a status
+ *     word at the start of the workspace and read back by asi_poll_status.
+ *   - Workspaces must be 256-byte aligned.
+ */
+#ifndef ASI_B200_H
+#define ASI_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ASI_OK = 0,
+  ASI_ERR_INVALID_ARG = 1,    /* null pointer, bad enum, non-positive size, aliasing */
+  ASI_ERR_UNSUPPORTED = 2,    /* dilation != 1, rank > 64, ndim out of range */
+  ASI_ERR_RANK_RANGE = 3,     /* r_m outside [1, min(a_m, b_m)] (Algorithm 1, inputs) */
+  ASI_ERR_WORKSPACE = 4,      /* workspace too small or misaligned */
+  ASI_ERR_CUDA = 5,           /* a CUDA runtime call failed */
+  ASI_ERR_RANK_DEFICIENT = 6, /* device: Orthogonalize met a dependent column */
+  ASI_ERR_TIMEOUT = 7         /* device: a bounded wait expired */
+} asi_status_t;
+
+typedef enum { ASI_F32 = 0, ASI_BF16 = 1 } asi_dtype_t;
+typedef enum { ASI_CONV2D = 0, ASI_LINEAR = 1 } asi_kind_t;
+
+#define ASI_MAX_MODES 4
+#define ASI_MAX_RANK 64
+
+/* One trained layer.  conv: ndim = 4, dims = (B,C,H,W).  linear: ndim = 2 or 3,
+ * dims = (B[,N],Din), cout = Dout and the conv fields are ignored. */
+typedef struct {
+  int32_t kind;                  /* asi_kind_t */
+  int32_t in_dtype;              /* asi_dtype_t of act and dY */
+  int32_t ndim;
+  int64_t dims[ASI_MAX_MODES];
+  int32_t ranks[ASI_MAX_MODES];  /* 1 <= r_m <= min(a_m, b_m), r_m <= 64 */
+  int32_t cout;
+  int32_t kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, groups;
+} asi_layer_desc_t;
+
+/* Sizes and the paper's closed forms for one plan. */
+typedef struct {
+  size_t compress_ws_bytes;      /* workspace asi_compress needs */
+  size_t wgrad_ws_bytes;         /* workspace asi_*_wgrad needs */
+  int64_t u_offset[ASI_MAX_MODES];
+  int64_t u_elems;               /* sum_m D_m r_m */
+  int64_t core_elems;            /* prod_m r_m */
+  int64_t act_elems, dy_elems, dw_elems;
+  int64_t out_h, out_w;          /* conv output size H', W' */
+  int64_t compressed_elems;      /* M_i = prod r_m + sum D_m r_m   (Sec. 3.2, storage equation) */
+  double ratio_RC;               /* prod D_m / M_i                  (appendix, space complexity) */
+  double macs_O_ASI;             /* sum_m (2 a_m b_m r_m + r_m^3)   (appendix, overhead) */
+  double macs_C_ASI;             /* five-term backward cost         (appendix, speedup); conv only, else 0 */
+  double macs_C_vanilla;         /* D^2 C C' B H' W' (conv) or B N Din Dout (linear) */
+} asi_plan_info_t;
+
+typedef struct asi_plan asi_plan_t;
+
+/* Host only; validates the descriptor and fixes kernel variants and workspace
+ * layout.  No GPU work, no CUDA context needed.  *out is set only on ASI_OK. */
+asi_status_t asi_plan_create(const asi_layer_desc_t* desc, asi_plan_t** out);
+asi_status_t asi_plan_destroy(asi_plan_t* plan);
+asi_status_t asi_plan_query(const asi_plan_t* plan, asi_plan_info_t* info);
+
+/* Algorithm 1 (ASI), branch t > 0, for one layer and one step:
+ *   for every mode m (each on the ORIGINAL activation):
+ *       V = A_m^T U_m^{prev};  U_m^{new} = Orthogonalize(A_m V)
+ *   core = A x_1 U_1^{new T} ... x_n U_n^{new T}
+ * Orthogonalize returns the Gram-Schmidt basis (thin-QR Q with diag(R) > 0).
+ *   act     [in]  device, in_dtype, dims as planned; not modified
+ *   U_prev  [in]  device fp32, u_elems; previous step's factors
+ *   U_new   [out] device fp32, u_elems; must not alias U_prev
+ *   core    [out] device fp32, core_elems
+ *   ws      device scratch of at least compress_ws_bytes; contents undefined
+ *           afterwards except the status word. */
+asi_status_t asi_compress(const asi_plan_t* plan, const void* act, const float* U_prev,
+                          float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
+
+/* Algorithm 1, branch t = 0 (cold start) with caller-supplied Gaussian test
+ * matrices: U_m = Orthogonalize(A_m Omega_m), then the core as above.
+ *   omega  [in] device fp32: Omega_m row-major [b_m x r_m], modes back to back
+ *          (offset of mode m = sum_{j<m} b_j r_j), rows ordered like the
+ *          columns of the mode-m unfolding with the remaining modes in
+ *          increasing order, last mode fastest. */
+asi_status_t asi_init_factors(const asi_plan_t* plan, const void* act, const float* omega,
+                              float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
+
+/* Weight gradient of a conv2d layer from the compressed activation, in the
+ * order the five terms of C_ASI fix (appendix "Speedup"):
+ *   Z1 = dY x_1 U_1^T;  Z3 = core x_3 U_3 x_4 U_4;
+ *   Z4 = conv_wgrad(Z3, Z1) with the layer's kernel/stride/padding;
+ *   dW = Z4 x_2 U_2  (per group when groups > 1).
+ * Equals the vanilla gradient (Sec. 3.1) of the reconstructed activation.
+ *   core, U [in] device fp32 (outputs of asi_compress);  dY [in] device in_dtype
+ *   dW [out] device fp32 [Cout, C/groups, kh, kw], overwritten. */
+asi_status_t asi_conv_wgrad(const asi_plan_t* plan, const float* core, const float* U,
+                            const void* dY, float* dW, void* ws, size_t ws_bytes, void* stream);
+
+/* Same for a linear layer y = x W^T on [B(,N),Din] tokens:
+ *   Z = dY x_1 U_1^T (x_2 U_2^T);  Z4[o,k] = sum Z[..,o] core[..,k];  dW = Z4 U_last^T.
+ *   dW [out] device fp32 [Dout, Din]. */
+asi_status_t asi_linear_wgrad(const asi_plan_t* plan, const float* core, const float* U,
+                              const void* dY, float* dW, void* ws, size_t ws_bytes, void* stream);
+
+/* One whole layer-step from HOST buffers (pinned memory recommended): copies
+ * act, dY and U_prev to the caller's device arena, runs asi_compress and the
+ * matching wgrad, and copies U_new, core and dW back.  Everything is enqueued
+ * on `stream`; the host buffers may be read after the stream is synchronised.
+ *   arena  device scratch of at least asi_step_host_arena_bytes(plan). */
+size_t asi_step_host_arena_bytes(const asi_plan_t* plan);
+asi_status_t asi_step_host(const asi_plan_t* plan, const void* act_host, const void* dY_host,
+                           const float* U_prev_host, float* U_new_host, float* core_host,
+                           float* dW_host, void* arena, size_t arena_bytes, void* stream);
+
+/* Reads the device status word of a workspace after synchronising `stream`.
+ * *device_status is ASI_OK, ASI_ERR_RANK_DEFICIENT or ASI_ERR_TIMEOUT. */
+asi_status_t asi_poll_status(const asi_plan_t* plan, const void* ws, void* stream,
+                             asi_status_t* device_status);
+
+/* Number of kernel launches the last call of each kind enqueues for this plan. */
+int32_t asi_launch_count(const asi_plan_t* plan, int32_t which /* 0 compress, 1 wgrad */);
+
+const char* asi_status_string(asi_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASI_B200_H */

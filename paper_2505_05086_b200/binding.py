@@ -1,0 +1,183 @@
+"""ctypes binding of the ASI C ABI (include/asi.h).
+
+Argument marshalling only: every step of the path runs inside the CUDA library.  Tensors are
+passed as raw device pointers (``tensor.data_ptr()``); PyTorch is used by callers for device
+memory and streams.  There is no CPU fallback: if the shared library is missing the import of
+``lib()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libasi_b200.so")
+_lib = None
+
+ASI_OK = 0
+ASI_ERR_INVALID_ARG = 1
+ASI_ERR_UNSUPPORTED = 2
+ASI_ERR_RANK_RANGE = 3
+ASI_ERR_WORKSPACE = 4
+ASI_ERR_CUDA = 5
+ASI_ERR_RANK_DEFICIENT = 6
+ASI_ERR_TIMEOUT = 7
+ASI_F32, ASI_BF16 = 0, 1
+ASI_CONV2D, ASI_LINEAR = 0, 1
+ASI_MAX_MODES = 4
+
+EXPORTS = (
+    "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_init_factors",
+    "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host",
+    "asi_poll_status", "asi_launch_count", "asi_status_string",
+)
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("in_dtype", C.c_int32), ("ndim", C.c_int32),
+                ("dims", C.c_int64 * ASI_MAX_MODES), ("ranks", C.c_int32 * ASI_MAX_MODES),
+                ("cout", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride_h", C.c_int32), ("stride_w", C.c_int32), ("pad_h", C.c_int32),
+                ("pad_w", C.c_int32), ("dil_h", C.c_int32), ("dil_w", C.c_int32),
+                ("groups", C.c_int32)]
+
+
+class PlanInfo(C.Structure):
+    _fields_ = [("compress_ws_bytes", C.c_size_t), ("wgrad_ws_bytes", C.c_size_t),
+                ("u_offset", C.c_int64 * ASI_MAX_MODES), ("u_elems", C.c_int64),
+                ("core_elems", C.c_int64), ("act_elems", C.c_int64), ("dy_elems", C.c_int64),
+                ("dw_elems", C.c_int64), ("out_h", C.c_int64), ("out_w", C.c_int64),
+                ("compressed_elems", C.c_int64), ("ratio_RC", C.c_double),
+                ("macs_O_ASI", C.c_double), ("macs_C_ASI", C.c_double),
+                ("macs_C_vanilla", C.c_double)]
+
+
+class AsiError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} (status {int(code)})")
+
+
+def lib():
+    """Loads libasi_b200.so (built in-tree by paper_2505_05086_b200.build).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} not built: run `python -m paper_2505_05086_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    vp, sz, i32 = C.c_void_p, C.c_size_t, C.c_int32
+    L.asi_plan_create.argtypes = [C.POINTER(LayerDesc), C.POINTER(vp)]
+    L.asi_plan_destroy.argtypes = [vp]
+    L.asi_plan_query.argtypes = [vp, C.POINTER(PlanInfo)]
+    L.asi_compress.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_init_factors.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_linear_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_step_host_arena_bytes.argtypes = [vp]
+    L.asi_step_host_arena_bytes.restype = sz
+    L.asi_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_poll_status.argtypes = [vp, vp, vp, C.POINTER(i32)]
+    L.asi_launch_count.argtypes = [vp, i32]
+    L.asi_launch_count.restype = i32
+    L.asi_status_string.argtypes = [i32]
+    L.asi_status_string.restype = C.c_char_p
+    for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress",
+                 "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
+                 "asi_poll_status"):
+        getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+def status_string(code) -> str:
+    return lib().asi_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != ASI_OK:
+        raise AsiError(code, where)
+
+
+def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False, dilation=1):
+    d = LayerDesc()
+    d.kind = ASI_CONV2D if kind == "conv" else ASI_LINEAR
+    d.in_dtype = ASI_BF16 if bf16 else ASI_F32
+    d.ndim = len(dims)
+    for i, v in enumerate(dims):
+        d.dims[i] = int(v)
+    for i, v in enumerate(ranks):
+        d.ranks[i] = int(v)
+    d.cout = int(cout)
+    kh, kw = (k, k) if isinstance(k, int) else k
+    sh, sw = (stride, stride) if isinstance(stride, int) else stride
+    ph, pw = (pad, pad) if isinstance(pad, int) else pad
+    d.kh, d.kw, d.stride_h, d.stride_w, d.pad_h, d.pad_w = kh, kw, sh, sw, ph, pw
+    d.dil_h = d.dil_w = int(dilation)
+    d.groups = int(groups)
+    return d
+
+
+class Plan:
+    """Owns one asi_plan_t.  Methods mirror the C entry points one to one; pointer arguments are
+    integers (device or host addresses), ``stream`` is a CUDA stream handle (0 = default)."""
+
+    def __init__(self, kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False,
+                 dilation=1):
+        self._h = C.c_void_p()
+        self.desc = make_desc(kind, dims, ranks, cout, k, stride, pad, groups, bf16, dilation)
+        _check(lib().asi_plan_create(C.byref(self.desc), C.byref(self._h)), "asi_plan_create")
+        self.kind = kind
+        self.info = PlanInfo()
+        _check(lib().asi_plan_query(self._h, C.byref(self.info)), "asi_plan_query")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().asi_plan_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+    def launch_count(self, which):
+        return lib().asi_launch_count(self._h, which)
+
+    def compress(self, act, U_prev, U_new, core, ws, ws_bytes, stream=0):
+        _check(lib().asi_compress(self._h, act, U_prev, U_new, core, ws, ws_bytes, stream),
+               "asi_compress")
+
+    def init_factors(self, act, omega, U_new, core, ws, ws_bytes, stream=0):
+        _check(lib().asi_init_factors(self._h, act, omega, U_new, core, ws, ws_bytes, stream),
+               "asi_init_factors")
+
+    def conv_wgrad(self, core, U, dY, dW, ws, ws_bytes, stream=0):
+        _check(lib().asi_conv_wgrad(self._h, core, U, dY, dW, ws, ws_bytes, stream), "asi_conv_wgrad")
+
+    def linear_wgrad(self, core, U, dY, dW, ws, ws_bytes, stream=0):
+        _check(lib().asi_linear_wgrad(self._h, core, U, dY, dW, ws, ws_bytes, stream),
+               "asi_linear_wgrad")
+
+    def wgrad(self, core, U, dY, dW, ws, ws_bytes, stream=0):
+        if self.kind == "conv":
+            self.conv_wgrad(core, U, dY, dW, ws, ws_bytes, stream)
+        else:
+            self.linear_wgrad(core, U, dY, dW, ws, ws_bytes, stream)
+
+    def step_host_arena_bytes(self):
+        return lib().asi_step_host_arena_bytes(self._h)
+
+    def step_host(self, act_h, dY_h, U_prev_h, U_new_h, core_h, dW_h, arena, arena_bytes, stream=0):
+        _check(lib().asi_step_host(self._h, act_h, dY_h, U_prev_h, U_new_h, core_h, dW_h, arena,
+                                   arena_bytes, stream), "asi_step_host")
+
+    def poll_status(self, ws, stream=0):
+        out = C.c_int32(0)
+        _check(lib().asi_poll_status(self._h, ws, stream, C.byref(out)), "asi_poll_status")
+        return out.value

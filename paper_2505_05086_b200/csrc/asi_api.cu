@@ -1,0 +1,524 @@
+// C ABI of the ASI library: plan construction (host only) and the enqueue sequences.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "asi_internal.h"
+
+using namespace asi;
+
+namespace {
+
+bool valid_ptr(const void* p) { return p != nullptr; }
+
+size_t elem_bytes(const asi_plan* pl) { return pl->bf16 ? 2 : 4; }
+
+void set_mode_views(asi_plan* pl) {
+  for (int m = 0; m < pl->nd; ++m) {
+    int64_t O = 1, I = 1;
+    for (int j = 0; j < m; ++j) O *= pl->dims[j];
+    for (int j = m + 1; j < pl->nd; ++j) I *= pl->dims[j];
+    pl->mv[m] = ModeView{O, pl->dims[m], I, O * I, pl->r[m]};
+  }
+}
+
+// Workspace layouts.  Every region is 256-byte aligned; region 0 is the status word.
+void layout_compress(asi_plan* pl) {
+  size_t off = kStatusBytes;
+  int64_t vmax = 0;
+  for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
+  pl->off_V = off;
+  off = align_up(off + (size_t)vmax * 4, 256);
+  for (int m = 0; m < pl->nd; ++m) {
+    const ModeView& v = pl->mv[m];
+    const int64_t kchunks = (v.a + kExpandKC - 1) / kExpandKC;
+    // about two waves of CTAs, at least four 64-column tiles per split
+    int64_t ns = std::max<int64_t>(1, 296 / kchunks);
+    ns = std::min<int64_t>(ns, std::max<int64_t>(1, v.Q / 256));
+    int64_t qps = (v.Q + ns - 1) / ns;
+    qps = (qps + 63) / 64 * 64;
+    ns = (v.Q + qps - 1) / qps;
+    pl->nsplit[m] = (int)ns;
+    pl->q_per_split[m] = qps;
+    pl->nchunk[m] = (int)((v.a + kQRRows - 1) / kQRRows);
+    pl->off_Pp[m] = off;
+    off = align_up(off + (size_t)ns * v.a * v.r * 4, 256);
+    pl->off_Pred[m] = off;
+    off = align_up(off + (size_t)v.a * v.r * 8, 256);
+    pl->off_Gp[m] = off;
+    off = align_up(off + (size_t)pl->nchunk[m] * v.r * v.r * 8, 256);
+  }
+  // core chain: contract the mode with the largest a_m / r_m first, then the rest in order
+  int order[ASI_MAX_MODES];
+  for (int m = 0; m < pl->nd; ++m) order[m] = m;
+  int best = 0;
+  for (int m = 1; m < pl->nd; ++m)
+    if ((double)pl->dims[m] / pl->r[m] > (double)pl->dims[best] / pl->r[best]) best = m;
+  std::swap(order[0], order[best]);
+  std::sort(order + 1, order + pl->nd);
+  std::memcpy(pl->core_order, order, sizeof(order));
+  int64_t cd[ASI_MAX_MODES];
+  for (int m = 0; m < pl->nd; ++m) cd[m] = pl->dims[m];
+  int64_t tmax[2] = {0, 0};
+  for (int s = 0; s + 1 < pl->nd; ++s) {
+    cd[order[s]] = pl->r[order[s]];
+    int64_t n = 1;
+    for (int m = 0; m < pl->nd; ++m) n *= cd[m];
+    tmax[s & 1] = std::max(tmax[s & 1], n);
+  }
+  for (int t = 0; t < 2; ++t) {
+    pl->off_T[t] = off;
+    off = align_up(off + (size_t)tmax[t] * 4, 256);
+  }
+  pl->compress_ws = off;
+  pl->launches_compress = 2 * pl->nd + 2 + pl->nd;
+}
+
+void layout_wgrad(asi_plan* pl) {
+  size_t off = kStatusBytes;
+  int64_t z[3] = {0, 0, 0};
+  if (pl->d.kind == ASI_CONV2D) {
+    z[0] = (int64_t)pl->r[0] * pl->d.cout * pl->Ho * pl->Wo;          // Z1
+    z[1] = (int64_t)pl->r[0] * pl->r[1] * pl->dims[2] * pl->r[3];     // core x_3 U_3
+    z[2] = (int64_t)pl->r[0] * pl->r[1] * pl->dims[2] * pl->dims[3];  // Z3
+    pl->launches_wgrad = 4;
+  } else {
+    const int nlead = pl->nd - 1;
+    int64_t rest = pl->d.cout;
+    for (int m = 1; m < nlead; ++m) rest *= pl->dims[m];
+    z[0] = (int64_t)pl->r[0] * rest;                                   // dY x_1 U_1^T
+    z[1] = (nlead > 1) ? (int64_t)pl->r[0] * pl->r[1] * pl->d.cout : 0;  // .. x_2 U_2^T
+    z[2] = (int64_t)pl->r[pl->nd - 1] * pl->d.cout;                    // Z4^T
+    pl->launches_wgrad = nlead + 2;
+  }
+  for (int t = 0; t < 3; ++t) {
+    pl->off_Z[t] = off;
+    off = align_up(off + (size_t)z[t] * 4, 256);
+  }
+  pl->wgrad_ws = off;
+}
+
+asi_status_t check_ws(const void* ws, size_t have, size_t need) {
+  if (!valid_ptr(ws)) return ASI_ERR_INVALID_ARG;
+  if (have < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return ASI_ERR_WORKSPACE;
+  return ASI_OK;
+}
+
+#define ASI_CUDA(call)                         \
+  do {                                         \
+    cudaError_t e__ = (call);                  \
+    if (e__ != cudaSuccess) return ASI_ERR_CUDA; \
+  } while (0)
+
+// U_m^{new} = Orthogonalize(P_m) for all modes given the split partials, then the core.
+asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, float* core,
+                             char* w, cudaStream_t st) {
+  QRArgs qa;
+  std::memset(&qa, 0, sizeof(qa));
+  int max_chunks = 1;
+  for (int m = 0; m < pl->nd; ++m) {
+    qa.m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
+    qa.m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
+    qa.m[m].Gp = reinterpret_cast<double*>(w + pl->off_Gp[m]);
+    qa.m[m].Uout = U_new + pl->u_off[m];
+    qa.m[m].a = (int)pl->dims[m];
+    qa.m[m].r = pl->r[m];
+    qa.m[m].nsplit = pl->nsplit[m];
+    qa.m[m].nchunk = pl->nchunk[m];
+    max_chunks = std::max(max_chunks, pl->nchunk[m]);
+  }
+  qa.status = reinterpret_cast<int*>(w);
+  ASI_CUDA(launch_qr(qa, pl->nd, max_chunks, st));
+
+  // core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T)
+  int64_t cd[ASI_MAX_MODES];
+  for (int m = 0; m < pl->nd; ++m) cd[m] = pl->dims[m];
+  const void* src = act;
+  bool src_bf16 = pl->bf16;
+  for (int s = 0; s < pl->nd; ++s) {
+    const int m = pl->core_order[s];
+    ModeProdArgs a;
+    a.X = src;
+    a.B = U_new + pl->u_off[m];
+    a.O = 1;
+    a.I = 1;
+    for (int j = 0; j < m; ++j) a.O *= cd[j];
+    for (int j = m + 1; j < pl->nd; ++j) a.I *= cd[j];
+    a.a = cd[m];
+    a.Q = a.O * a.I;
+    a.n_out = pl->r[m];
+    a.ldb_k = pl->r[m];
+    a.ldb_j = 1;
+    a.so = (int64_t)pl->r[m] * a.I;
+    a.sj = a.I;
+    a.si = 1;
+    float* dst = (s == pl->nd - 1) ? core : reinterpret_cast<float*>(w + pl->off_T[s & 1]);
+    a.Y = dst;
+    ASI_CUDA(launch_modeprod(a, src_bf16, st));
+    cd[m] = pl->r[m];
+    src = dst;
+    src_bf16 = false;
+  }
+  return ASI_OK;
+}
+
+asi_status_t expand_mode(const asi_plan* pl, int m, const void* act, const float* V, char* w,
+                         cudaStream_t st) {
+  const ModeView& v = pl->mv[m];
+  ExpandArgs e;
+  e.X = act;
+  e.V = V;
+  e.Pp = reinterpret_cast<float*>(w + pl->off_Pp[m]);
+  e.O = v.O;
+  e.a = v.a;
+  e.I = v.I;
+  e.Q = v.Q;
+  e.r = v.r;
+  e.nsplit = pl->nsplit[m];
+  e.q_per_split = pl->q_per_split[m];
+  ASI_CUDA(launch_expand(e, pl->bf16, st));
+  return ASI_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* asi_status_string(asi_status_t s) {
+  switch (s) {
+    case ASI_OK: return "ok";
+    case ASI_ERR_INVALID_ARG: return "invalid argument";
+    case ASI_ERR_UNSUPPORTED: return "unsupported configuration";
+    case ASI_ERR_RANK_RANGE: return "rank outside [1, min(a_m, b_m)]";
+    case ASI_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case ASI_ERR_CUDA: return "CUDA runtime error";
+    case ASI_ERR_RANK_DEFICIENT: return "rank-deficient subspace iterate";
+    case ASI_ERR_TIMEOUT: return "bounded device wait expired";
+  }
+  return "unknown status";
+}
+
+asi_status_t asi_plan_create(const asi_layer_desc_t* desc, asi_plan_t** out) {
+  if (!desc || !out) return ASI_ERR_INVALID_ARG;
+  const asi_layer_desc_t& d = *desc;
+  if (d.kind != ASI_CONV2D && d.kind != ASI_LINEAR) return ASI_ERR_INVALID_ARG;
+  if (d.in_dtype != ASI_F32 && d.in_dtype != ASI_BF16) return ASI_ERR_INVALID_ARG;
+  if (d.kind == ASI_CONV2D && d.ndim != 4) return ASI_ERR_UNSUPPORTED;
+  if (d.kind == ASI_LINEAR && d.ndim != 2 && d.ndim != 3) return ASI_ERR_UNSUPPORTED;
+  if (d.cout < 1) return ASI_ERR_INVALID_ARG;
+  int64_t N = 1;
+  for (int m = 0; m < d.ndim; ++m) {
+    if (d.dims[m] < 1 || d.dims[m] > (int64_t)1 << 31) return ASI_ERR_INVALID_ARG;
+    N *= d.dims[m];
+    if (N > (int64_t)1 << 40) return ASI_ERR_UNSUPPORTED;
+  }
+  for (int m = 0; m < d.ndim; ++m) {
+    const int64_t a = d.dims[m], b = N / a;
+    if (d.ranks[m] < 1 || d.ranks[m] > std::min(a, b)) return ASI_ERR_RANK_RANGE;
+    if (d.ranks[m] > ASI_MAX_RANK) return ASI_ERR_UNSUPPORTED;
+  }
+  int64_t Ho = 0, Wo = 0;
+  if (d.kind == ASI_CONV2D) {
+    if (d.kh < 1 || d.kw < 1 || d.stride_h < 1 || d.stride_w < 1 || d.pad_h < 0 || d.pad_w < 0 ||
+        d.groups < 1)
+      return ASI_ERR_INVALID_ARG;
+    if (d.dil_h != 1 || d.dil_w != 1) return ASI_ERR_UNSUPPORTED;
+    if (d.dims[1] % d.groups || d.cout % d.groups) return ASI_ERR_INVALID_ARG;
+    if (d.kh > 16 || d.kw > 16) return ASI_ERR_UNSUPPORTED;
+    const int64_t hn = d.dims[2] + 2 * d.pad_h - d.kh, wn = d.dims[3] + 2 * d.pad_w - d.kw;
+    if (hn < 0 || wn < 0) return ASI_ERR_INVALID_ARG;
+    Ho = hn / d.stride_h + 1;
+    Wo = wn / d.stride_w + 1;
+  }
+  asi_plan* pl = new (std::nothrow) asi_plan;
+  if (!pl) return ASI_ERR_INVALID_ARG;
+  std::memset(pl, 0, sizeof(*pl));
+  pl->d = d;
+  pl->nd = d.ndim;
+  pl->N = N;
+  pl->bf16 = d.in_dtype == ASI_BF16;
+  pl->Ho = Ho;
+  pl->Wo = Wo;
+  int64_t uo = 0, ce = 1;
+  for (int m = 0; m < d.ndim; ++m) {
+    pl->dims[m] = d.dims[m];
+    pl->r[m] = d.ranks[m];
+    pl->u_off[m] = uo;
+    uo += d.dims[m] * d.ranks[m];
+    ce *= d.ranks[m];
+  }
+  pl->u_elems = uo;
+  pl->core_elems = ce;
+  if (d.kind == ASI_CONV2D) {
+    pl->dy_elems = d.dims[0] * d.cout * Ho * Wo;
+    pl->dw_elems = (int64_t)d.cout * (d.dims[1] / d.groups) * d.kh * d.kw;
+  } else {
+    pl->dy_elems = N / d.dims[d.ndim - 1] * d.cout;
+    pl->dw_elems = (int64_t)d.cout * d.dims[d.ndim - 1];
+  }
+  set_mode_views(pl);
+  layout_compress(pl);
+  layout_wgrad(pl);
+  *out = pl;
+  return ASI_OK;
+}
+
+asi_status_t asi_plan_destroy(asi_plan_t* plan) {
+  if (!plan) return ASI_ERR_INVALID_ARG;
+  delete plan;
+  return ASI_OK;
+}
+
+asi_status_t asi_plan_query(const asi_plan_t* pl, asi_plan_info_t* info) {
+  if (!pl || !info) return ASI_ERR_INVALID_ARG;
+  std::memset(info, 0, sizeof(*info));
+  info->compress_ws_bytes = pl->compress_ws;
+  info->wgrad_ws_bytes = pl->wgrad_ws;
+  double sum_r = 0, sum_r3 = 0;
+  for (int m = 0; m < pl->nd; ++m) {
+    info->u_offset[m] = pl->u_off[m];
+    sum_r += pl->r[m];
+    sum_r3 += (double)pl->r[m] * pl->r[m] * pl->r[m];
+  }
+  info->u_elems = pl->u_elems;
+  info->core_elems = pl->core_elems;
+  info->act_elems = pl->N;
+  info->dy_elems = pl->dy_elems;
+  info->dw_elems = pl->dw_elems;
+  info->out_h = pl->Ho;
+  info->out_w = pl->Wo;
+  info->compressed_elems = pl->core_elems + pl->u_elems;
+  info->ratio_RC = (double)pl->N / (double)info->compressed_elems;
+  info->macs_O_ASI = 2.0 * (double)pl->N * sum_r + sum_r3;
+  if (pl->d.kind == ASI_CONV2D) {
+    const double B = pl->dims[0], C = pl->dims[1], H = pl->dims[2], W = pl->dims[3];
+    const double r1 = pl->r[0], r2 = pl->r[1], r3 = pl->r[2], r4 = pl->r[3];
+    const double Co = pl->d.cout, HoWo = (double)pl->Ho * pl->Wo, D2 = (double)pl->d.kh * pl->d.kw;
+    info->macs_C_ASI = r1 * B * Co * HoWo + r1 * r2 * r3 * r4 * H + r1 * r2 * r4 * H * W +
+                       r1 * r2 * Co * HoWo * D2 + r2 * Co * C * D2;
+    info->macs_C_vanilla = D2 * C * Co * B * HoWo;
+  } else {
+    info->macs_C_ASI = 0.0;
+    info->macs_C_vanilla = (double)pl->N * pl->d.cout;
+  }
+  return ASI_OK;
+}
+
+int32_t asi_launch_count(const asi_plan_t* pl, int32_t which) {
+  if (!pl) return -1;
+  return which == 0 ? pl->launches_compress : pl->launches_wgrad;
+}
+
+asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_prev, float* U_new,
+                          float* core, void* ws, size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(act) || !valid_ptr(U_prev) || !valid_ptr(U_new) || !valid_ptr(core))
+    return ASI_ERR_INVALID_ARG;
+  if (U_prev == U_new) return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(ws, ws_bytes, pl->compress_ws);
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
+  float* V = reinterpret_cast<float*>(w + pl->off_V);
+  for (int m = 0; m < pl->nd; ++m) {
+    const ModeView& v = pl->mv[m];
+    // V = A_m^T U_m^{prev}, stored [b_m x r_m]
+    ModeProdArgs a;
+    a.X = act;
+    a.B = U_prev + pl->u_off[m];
+    a.Y = V;
+    a.O = v.O;
+    a.a = v.a;
+    a.I = v.I;
+    a.Q = v.Q;
+    a.n_out = v.r;
+    a.ldb_k = v.r;
+    a.ldb_j = 1;
+    a.so = v.I * v.r;
+    a.sj = 1;
+    a.si = v.r;
+    ASI_CUDA(launch_modeprod(a, pl->bf16, st));
+    // P = A_m V
+    s = expand_mode(pl, m, act, V, w, st);
+    if (s != ASI_OK) return s;
+  }
+  return finish_compress(pl, act, U_new, core, w, st);
+}
+
+asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float* omega, float* U_new,
+                              float* core, void* ws, size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(act) || !valid_ptr(omega) || !valid_ptr(U_new) || !valid_ptr(core))
+    return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(ws, ws_bytes, pl->compress_ws);
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
+  int64_t off = 0;
+  for (int m = 0; m < pl->nd; ++m) {
+    s = expand_mode(pl, m, act, omega + off, w, st);
+    if (s != ASI_OK) return s;
+    off += pl->mv[m].Q * pl->r[m];
+  }
+  return finish_compress(pl, act, U_new, core, w, st);
+}
+
+asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float* U, const void* dY,
+                            float* dW, void* ws, size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(core) || !valid_ptr(U) || !valid_ptr(dY) || !valid_ptr(dW))
+    return ASI_ERR_INVALID_ARG;
+  if (pl->d.kind != ASI_CONV2D) return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(ws, ws_bytes, pl->wgrad_ws);
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  float* Z1 = reinterpret_cast<float*>(w + pl->off_Z[0]);
+  float* Z3a = reinterpret_cast<float*>(w + pl->off_Z[1]);
+  float* Z3 = reinterpret_cast<float*>(w + pl->off_Z[2]);
+  const int64_t B = pl->dims[0], H = pl->dims[2], W = pl->dims[3];
+  const int r1 = pl->r[0], r2 = pl->r[1], r3 = pl->r[2], r4 = pl->r[3];
+  const int64_t per_sample = (int64_t)pl->d.cout * pl->Ho * pl->Wo;
+
+  ModeProdArgs a;
+  // term 1: Z1 = dY x_1 U_1^T
+  a.X = dY; a.B = U + pl->u_off[0]; a.Y = Z1;
+  a.O = 1; a.a = B; a.I = per_sample; a.Q = per_sample;
+  a.n_out = r1; a.ldb_k = r1; a.ldb_j = 1;
+  a.so = 0; a.sj = per_sample; a.si = 1;
+  ASI_CUDA(launch_modeprod(a, pl->bf16, st));
+  // term 2: core x_3 U_3  -> [r1 r2, H, r4]
+  a.X = core; a.B = U + pl->u_off[2]; a.Y = Z3a;
+  a.O = (int64_t)r1 * r2; a.a = r3; a.I = r4; a.Q = a.O * a.I;
+  a.n_out = (int)H; a.ldb_k = 1; a.ldb_j = r3;
+  a.so = H * r4; a.sj = r4; a.si = 1;
+  ASI_CUDA(launch_modeprod(a, false, st));
+  // term 3: .. x_4 U_4 -> Z3 [r1 r2 H, W]
+  a.X = Z3a; a.B = U + pl->u_off[3]; a.Y = Z3;
+  a.O = (int64_t)r1 * r2 * H; a.a = r4; a.I = 1; a.Q = a.O;
+  a.n_out = (int)W; a.ldb_k = 1; a.ldb_j = r4;
+  a.so = W; a.sj = 1; a.si = 1;
+  ASI_CUDA(launch_modeprod(a, false, st));
+  // terms 4 and 5
+  ConvTailArgs t;
+  t.Z1 = Z1; t.Z3 = Z3; t.U2 = U + pl->u_off[1]; t.dW = dW;
+  t.r1 = r1; t.r2 = r2; t.C = (int)pl->dims[1]; t.Cout = pl->d.cout;
+  t.H = (int)H; t.W = (int)W; t.Ho = (int)pl->Ho; t.Wo = (int)pl->Wo;
+  t.kh = pl->d.kh; t.kw = pl->d.kw; t.sh = pl->d.stride_h; t.sw = pl->d.stride_w;
+  t.ph = pl->d.pad_h; t.pw = pl->d.pad_w; t.groups = pl->d.groups;
+  ASI_CUDA(launch_conv_tail(t, st));
+  return ASI_OK;
+}
+
+asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const float* U, const void* dY,
+                              float* dW, void* ws, size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(core) || !valid_ptr(U) || !valid_ptr(dY) || !valid_ptr(dW))
+    return ASI_ERR_INVALID_ARG;
+  if (pl->d.kind != ASI_LINEAR) return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(ws, ws_bytes, pl->wgrad_ws);
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  const int nd = pl->nd, nlead = nd - 1;
+  const int64_t Dout = pl->d.cout, Din = pl->dims[nd - 1];
+  const int rl = pl->r[nd - 1];
+
+  // Z = dY x_1 U_1^T (x_2 U_2^T): leading modes one by one
+  int64_t cd[ASI_MAX_MODES];
+  for (int m = 0; m < nlead; ++m) cd[m] = pl->dims[m];
+  cd[nlead] = Dout;
+  const void* src = dY;
+  bool src_bf16 = pl->bf16;
+  int64_t lead_r = 1;
+  ModeProdArgs a;
+  for (int m = 0; m < nlead; ++m) {
+    a.X = src; a.B = U + pl->u_off[m];
+    a.Y = reinterpret_cast<float*>(w + pl->off_Z[m]);
+    a.O = 1; a.I = 1;
+    for (int j = 0; j < m; ++j) a.O *= cd[j];
+    for (int j = m + 1; j <= nlead; ++j) a.I *= cd[j];
+    a.a = cd[m]; a.Q = a.O * a.I;
+    a.n_out = pl->r[m]; a.ldb_k = pl->r[m]; a.ldb_j = 1;
+    a.so = (int64_t)pl->r[m] * a.I; a.sj = a.I; a.si = 1;
+    ASI_CUDA(launch_modeprod(a, src_bf16, st));
+    cd[m] = pl->r[m];
+    lead_r *= pl->r[m];
+    src = a.Y;
+    src_bf16 = false;
+  }
+  // Z4^T[k, o] = sum_{lead} Z[lead, o] core[lead, k]
+  float* Z4t = reinterpret_cast<float*>(w + pl->off_Z[2]);
+  a.X = src; a.B = core; a.Y = Z4t;
+  a.O = 1; a.a = lead_r; a.I = Dout; a.Q = Dout;
+  a.n_out = rl; a.ldb_k = rl; a.ldb_j = 1;
+  a.so = 0; a.sj = Dout; a.si = 1;
+  ASI_CUDA(launch_modeprod(a, false, st));
+  // dW[o, d] = sum_k Z4^T[k, o] U_last[d, k]
+  a.X = Z4t; a.B = U + pl->u_off[nd - 1]; a.Y = dW;
+  a.O = 1; a.a = rl; a.I = Dout; a.Q = Dout;
+  a.n_out = (int)Din; a.ldb_k = 1; a.ldb_j = rl;
+  a.so = 0; a.sj = 1; a.si = Din;
+  ASI_CUDA(launch_modeprod(a, false, st));
+  return ASI_OK;
+}
+
+size_t asi_step_host_arena_bytes(const asi_plan_t* pl) {
+  if (!pl) return 0;
+  const size_t eb = elem_bytes(pl);
+  size_t off = 0;
+  off = align_up(off + (size_t)pl->N * eb, 256);
+  off = align_up(off + (size_t)pl->dy_elems * eb, 256);
+  off = align_up(off + (size_t)pl->u_elems * 4, 256) * 1;
+  off = align_up(off + (size_t)pl->u_elems * 4, 256);
+  off = align_up(off + (size_t)pl->core_elems * 4, 256);
+  off = align_up(off + (size_t)pl->dw_elems * 4, 256);
+  off += align_up(std::max(pl->compress_ws, pl->wgrad_ws), 256);
+  return off;
+}
+
+asi_status_t asi_step_host(const asi_plan_t* pl, const void* act_host, const void* dY_host,
+                           const float* U_prev_host, float* U_new_host, float* core_host,
+                           float* dW_host, void* arena, size_t arena_bytes, void* stream) {
+  if (!pl || !act_host || !dY_host || !U_prev_host || !U_new_host || !core_host || !dW_host)
+    return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(arena, arena_bytes, asi_step_host_arena_bytes(pl));
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t eb = elem_bytes(pl);
+  char* base = static_cast<char*>(arena);
+  size_t off = 0;
+  char* d_act = base + off; off = align_up(off + (size_t)pl->N * eb, 256);
+  char* d_dy = base + off; off = align_up(off + (size_t)pl->dy_elems * eb, 256);
+  float* d_up = reinterpret_cast<float*>(base + off); off = align_up(off + (size_t)pl->u_elems * 4, 256);
+  float* d_un = reinterpret_cast<float*>(base + off); off = align_up(off + (size_t)pl->u_elems * 4, 256);
+  float* d_core = reinterpret_cast<float*>(base + off); off = align_up(off + (size_t)pl->core_elems * 4, 256);
+  float* d_dw = reinterpret_cast<float*>(base + off); off = align_up(off + (size_t)pl->dw_elems * 4, 256);
+  void* d_ws = base + off;
+  const size_t ws_bytes = align_up(std::max(pl->compress_ws, pl->wgrad_ws), 256);
+  ASI_CUDA(cudaMemcpyAsync(d_act, act_host, (size_t)pl->N * eb, cudaMemcpyHostToDevice, st));
+  ASI_CUDA(cudaMemcpyAsync(d_up, U_prev_host, (size_t)pl->u_elems * 4, cudaMemcpyHostToDevice, st));
+  s = asi_compress(pl, d_act, d_up, d_un, d_core, d_ws, ws_bytes, stream);
+  if (s != ASI_OK) return s;
+  ASI_CUDA(cudaMemcpyAsync(d_dy, dY_host, (size_t)pl->dy_elems * eb, cudaMemcpyHostToDevice, st));
+  if (pl->d.kind == ASI_CONV2D)
+    s = asi_conv_wgrad(pl, d_core, d_un, d_dy, d_dw, d_ws, ws_bytes, stream);
+  else
+    s = asi_linear_wgrad(pl, d_core, d_un, d_dy, d_dw, d_ws, ws_bytes, stream);
+  if (s != ASI_OK) return s;
+  ASI_CUDA(cudaMemcpyAsync(U_new_host, d_un, (size_t)pl->u_elems * 4, cudaMemcpyDeviceToHost, st));
+  ASI_CUDA(cudaMemcpyAsync(core_host, d_core, (size_t)pl->core_elems * 4, cudaMemcpyDeviceToHost, st));
+  ASI_CUDA(cudaMemcpyAsync(dW_host, d_dw, (size_t)pl->dw_elems * 4, cudaMemcpyDeviceToHost, st));
+  return ASI_OK;
+}
+
+asi_status_t asi_poll_status(const asi_plan_t* pl, const void* ws, void* stream,
+                             asi_status_t* device_status) {
+  if (!pl || !ws || !device_status) return ASI_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int v = 0;
+  ASI_CUDA(cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, st));
+  ASI_CUDA(cudaStreamSynchronize(st));
+  *device_status = static_cast<asi_status_t>(v);
+  return ASI_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of the ASI library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "asi.h"
+
+namespace asi {
+
+// Mode-m view of a contiguous tensor: element (o, k, i) at o*a*I + k*I + i.
+// Fibers of the mode are indexed by the flat column q = o*I + i.
+struct ModeView {
+  int64_t O, a, I, Q;   // Q = O*I = b_m
+  int r;
+};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+constexpr int kStatusBytes = 256;
+constexpr int kQRRows = 64;          // rows per CTA in the orthonormalisation kernels
+constexpr int kExpandKC = 32;        // rows of P per CTA in the expand kernel
+
+// Y(o, j, i) = sum_k X(o, k, i) * B(k, j): the small-mode contraction that serves the
+// projection V = A_m^T U, the core products, Z1, Z3, and the final expansions.
+struct ModeProdArgs {
+  const void* X;
+  const float* B;
+  float* Y;
+  int64_t O, a, I, Q;
+  int n_out;
+  int64_t ldb_k, ldb_j;    // B(k, j) = B[k*ldb_k + j*ldb_j]
+  int64_t so, sj, si;      // Y(o, j, i) = Y[o*so + j*sj + i*si]
+};
+
+// Pp[s](k, j) = sum_{q in split s} X(k, q) * V[q*r + j]
+struct ExpandArgs {
+  const void* X;
+  const float* V;
+  float* Pp;
+  int64_t O, a, I, Q;
+  int r, nsplit;
+  int64_t q_per_split;
+};
+
+struct QRMode {
+  const float* Pp;     // [nsplit][a][r]
+  double* Pred;        // [a][r]
+  double* Gp;          // [nchunk][r][r]
+  float* Uout;         // [a][r]
+  int a, r, nsplit, nchunk;
+};
+struct QRArgs {
+  QRMode m[ASI_MAX_MODES];
+  int* status;
+};
+
+// Z4[c', j, kh, kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p], then
+// dW[c', cl, kh, kw] = sum_j Z4[c', j, kh, kw] U2[(g*cg + cl), j].
+struct ConvTailArgs {
+  const float* Z1;     // [r1][Cout][Ho][Wo]
+  const float* Z3;     // [r1][r2][H][W]
+  const float* U2;     // [C][r2]
+  float* dW;           // [Cout][C/groups][kh][kw]
+  int r1, r2, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups;
+};
+
+cudaError_t launch_modeprod(const ModeProdArgs& p, bool x_bf16, cudaStream_t st);
+cudaError_t launch_expand(const ExpandArgs& p, bool x_bf16, cudaStream_t st);
+cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
+cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
+
+}  // namespace asi
+
+struct asi_plan {
+  asi_layer_desc_t d;
+  int nd;
+  int64_t dims[ASI_MAX_MODES];
+  int r[ASI_MAX_MODES];
+  int64_t N;
+  int64_t u_off[ASI_MAX_MODES], u_elems, core_elems;
+  int64_t dy_elems, dw_elems, Ho, Wo;
+  asi::ModeView mv[ASI_MAX_MODES];
+  bool bf16;
+
+  // compress workspace (byte offsets)
+  size_t off_V, off_Pp[ASI_MAX_MODES], off_Pred[ASI_MAX_MODES], off_Gp[ASI_MAX_MODES], off_T[2];
+  int nsplit[ASI_MAX_MODES], nchunk[ASI_MAX_MODES];
+  int64_t q_per_split[ASI_MAX_MODES];
+  int core_order[ASI_MAX_MODES];
+  size_t compress_ws;
+
+  // wgrad workspace (byte offsets)
+  size_t off_Z[3];
+  size_t wgrad_ws;
+
+  int launches_compress, launches_wgrad;
+};

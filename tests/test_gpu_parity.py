@@ -1,0 +1,205 @@
+"""CUDA path vs fp64 oracle, element by element, through the C ABI, on seeded inputs.
+
+Tolerances (relative Frobenius error): fp32 inputs -- projectors U U^T <= 1e-4, sign-aligned
+core <= 1e-4, dW <= 5e-4; bf16-input mode -- <= 2e-2 on all three."""
+import numpy as np
+import pytest
+import torch
+
+from asi_inputs.configs import LayerSpec, get_config, make_stream
+from asi_inputs.generator import LayerStream
+from oracle import asi_oracle as O
+from tests.gpu_util import TOL_BF16, TOL_F32, check, compare_step, make_runner, oracle_wgrad
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_config(cfg, layer_index, steps, tol, bf16=None):
+    L = cfg.layers[layer_index]
+    st = make_stream(cfg, layer_index)
+    run = make_runner(L, bf16=cfg.bf16)
+    U_prev = st.u_prev0()
+    worst = {}
+    for t in range(steps):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, tol, f"{cfg.name}/{L.name}/step{t}")
+        for k, v in err.items():
+            worst[k] = max(worst.get(k, 0.0), v) if k != "sign" else min(worst.get(k, 1.0), v)
+    return worst
+
+
+def test_config1_single_conv_three_warm_steps():
+    _run_config(get_config(0), 0, 3, TOL_F32)
+
+
+SMALL = [  # ragged sizes spanning several tiles with tails; (dims, ranks, cout, k, s, p, groups)
+    ((5, 12, 9, 11), (3, 5, 4, 6), 7, 3, 1, 1, 1),
+    ((6, 10, 13, 13), (2, 3, 3, 3), 9, 3, 2, 1, 1),
+    ((4, 16, 7, 7), (3, 4, 3, 3), 16, 3, 1, 1, 16),      # depthwise
+    ((9, 24, 6, 5), (4, 6, 2, 2), 20, 1, 1, 0, 1),       # pointwise
+    ((7, 8, 10, 10), (3, 3, 3, 3), 12, 1, 2, 0, 4),      # strided 1x1, four groups
+    ((3, 70, 5, 5), (2, 33, 2, 2), 5, 3, 1, 1, 1),       # rank above 32 in one mode
+    ((2, 3, 4, 5), (2, 3, 4, 5), 3, 3, 1, 1, 1),         # full rank everywhere
+    ((1, 40, 8, 8), (1, 4, 3, 3), 6, 5, 1, 2, 1),        # batch of one, 5x5 kernel
+]
+
+
+@pytest.mark.parametrize("case", SMALL)
+def test_small_ragged_conv_layers(case):
+    dims, ranks, cout, k, s, p, g = case
+    L = LayerSpec("t", "conv", dims, cout, k, s, p, g, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=sum(dims) + k,
+                     gen_ranks=tuple(min(d, max(r + 2, 4)) for d, r in zip(dims, ranks)))
+    run = make_runner(L)
+    U_prev = st.u_prev0()
+    for t in range(2):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, TOL_F32, str(case))
+
+
+def test_full_rank_reproduces_vanilla_gradient():
+    dims, cout = (3, 6, 5, 4), 5
+    L = LayerSpec("t", "conv", dims, cout, 3, 1, 1, 1, ranks=dims)
+    rng = np.random.default_rng(0)
+    A = rng.standard_normal(dims).astype(np.float32)
+    dY = rng.standard_normal(L.dy_shape).astype(np.float32)
+    U_prev = [np.linalg.qr(rng.standard_normal((d, d)))[0].astype(np.float32) for d in dims]
+    run = make_runner(L)
+    run.set_factors(U_prev)
+    run.compress(run.to_device(A))
+    run.wgrad(run.to_device(dY))
+    vanilla = O.conv_wgrad_direct(A, dY, 3, 3, 1, 1)
+    assert O.rel_fro(run.dW_np(L.dw_shape), vanilla) < 5e-5
+    assert O.rel_fro(O.reconstruct(run.core_np(), run.factors()), A) < 5e-5
+
+
+@pytest.mark.parametrize("dims,ranks,cout", [((6, 37, 50), (3, 5, 7), 21), ((45, 33), (6, 9), 17),
+                                             ((4, 19, 130), (4, 16, 64), 40)])
+def test_linear_layers(dims, ranks, cout):
+    L = LayerSpec("t", "linear", dims, cout, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=11 + len(dims),
+                     rho=tuple(0.7 ** (8.0 / max(r, 8)) for r in ranks),
+                     gen_ranks=tuple(min(d, 2 * r) for d, r in zip(dims, ranks)))
+    run = make_runner(L)
+    U_prev = st.u_prev0()
+    for t in range(2):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, TOL_F32, f"linear {dims}")
+
+
+def test_bf16_input_mode_small():
+    dims, ranks = (6, 20, 9, 9), (3, 4, 3, 3)
+    L = LayerSpec("t", "conv", dims, 10, 3, 1, 1, 1, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=5, bf16=True)
+    run = make_runner(L, bf16=True)
+    U_prev = st.u_prev0()
+    A, dY = st.next()
+    err, _ = compare_step(run, L, A, dY, U_prev)
+    check(err, TOL_BF16, "bf16")
+    # inputs are exactly representable, arithmetic is fp32: the fp32 bar holds as well
+    check(err, TOL_F32, "bf16 at fp32 bar")
+
+
+def test_cold_start_with_explicit_gaussian_matrices():
+    dims, ranks = (5, 14, 6, 7), (2, 4, 3, 3)
+    L = LayerSpec("t", "conv", dims, 4, 3, 1, 1, 1, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=3)
+    A, _ = st.next()
+    rng = np.random.default_rng(1)
+    n = int(np.prod(dims))
+    Omega = [rng.standard_normal((n // d, r)).astype(np.float32) for d, r in zip(dims, ranks)]
+    run = make_runner(L)
+    om = torch.from_numpy(np.concatenate([o.ravel() for o in Omega])).cuda()
+    run.init_factors(run.to_device(A), om)
+    assert run.ok()
+    S_ref, U_ref = O.asi_cold_start(A.astype(np.float64), [o.astype(np.float64) for o in Omega])
+    U_gpu = run.factors()
+    for ug, ur in zip(U_gpu, U_ref):
+        assert O.rel_fro(O.projector(ug), O.projector(ur)) < 1e-4
+    S_al, _ = O.sign_align(run.core_np(), U_gpu, U_ref)
+    assert O.rel_fro(S_al, S_ref) < 1e-4
+
+
+def test_rank_deficient_iterate_is_reported_not_hidden():
+    dims, ranks = (4, 6, 5, 5), (2, 3, 2, 2)
+    L = LayerSpec("t", "conv", dims, 4, 3, 1, 1, 1, ranks=ranks)
+    rng = np.random.default_rng(2)
+    A = rng.standard_normal(dims).astype(np.float32)
+    U_prev = [np.linalg.qr(rng.standard_normal((d, r)))[0].astype(np.float32) for d, r in zip(dims, ranks)]
+    U_prev[1][:, 2] = U_prev[1][:, 0]          # two identical columns: P_2 has rank 2 < 3
+    run = make_runner(L)
+    run.set_factors(U_prev)
+    run.compress(run.to_device(A))
+    assert run.device_status() == 6
+    with pytest.raises(O.RankDeficientError):
+        O.asi_compress(A.astype(np.float64), [u.astype(np.float64) for u in U_prev])
+    # a healthy call on the same workspace clears the word
+    U_prev[1] = np.linalg.qr(rng.standard_normal((6, 3)))[0].astype(np.float32)
+    run.set_factors(U_prev)
+    run.compress(run.to_device(A))
+    assert run.device_status() == 0
+
+
+def test_results_are_bitwise_reproducible():
+    cfg = get_config(0)
+    L = cfg.layers[0]
+    st = make_stream(cfg, 0)
+    A, dY = st.next()
+    outs = []
+    for _ in range(2):
+        run = make_runner(L)
+        run.set_factors(st.u_prev0())
+        run.compress(run.to_device(A))
+        run.wgrad(run.to_device(dY))
+        outs.append((np.concatenate([u.ravel() for u in run.factors()]), run.core_np(), run.dW_np(L.dw_shape)))
+    for a, b in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a, b)
+
+
+def test_free_running_warm_start_does_not_drift_from_oracle():
+    """Without teacher forcing (each side feeds on its own previous factors) the errors stay at
+    the one-step level: the iteration contracts perturbations."""
+    cfg = get_config(0)
+    L = cfg.layers[0]
+    st = make_stream(cfg, 0)
+    run = make_runner(L)
+    run.set_factors(st.u_prev0())
+    U_ref = [u.astype(np.float64) for u in st.u_prev0()]
+    for t in range(3):
+        A, dY = st.next()
+        run.compress(run.to_device(A))
+        run.wgrad(run.to_device(dY))
+        S_ref, U_ref = O.asi_compress(A.astype(np.float64), U_ref)
+        dW_ref = oracle_wgrad(L, S_ref, U_ref, dY.astype(np.float64))
+        for ug, ur in zip(run.factors(), U_ref):
+            assert O.rel_fro(O.projector(ug), O.projector(ur)) < 3e-4
+        assert O.rel_fro(run.dW_np(L.dw_shape), dW_ref) < 1e-3
+
+
+def test_step_from_host_buffers_matches_device_path():
+    cfg = get_config(0)
+    L = cfg.layers[0]
+    st = make_stream(cfg, 0)
+    A, dY = st.next()
+    run = make_runner(L)
+    run.set_factors(st.u_prev0())
+    run.compress(run.to_device(A))
+    run.wgrad(run.to_device(dY))
+    p = run.plan
+    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).pin_memory()
+    hA, hdY = pin(A), pin(dY)
+    hUp = pin(np.concatenate([u.ravel() for u in st.u_prev0()]))
+    hUn = torch.empty(p.info.u_elems).pin_memory()
+    hS = torch.empty(p.info.core_elems).pin_memory()
+    hdW = torch.empty(p.info.dw_elems).pin_memory()
+    arena = torch.empty(p.step_host_arena_bytes(), dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream()
+    p.step_host(hA.data_ptr(), hdY.data_ptr(), hUp.data_ptr(), hUn.data_ptr(), hS.data_ptr(),
+                hdW.data_ptr(), arena.data_ptr(), arena.numel(), int(s.cuda_stream))
+    s.synchronize()
+    np.testing.assert_array_equal(hUn.numpy(), run.U[run.cur].cpu().numpy())
+    np.testing.assert_array_equal(hS.numpy(), run.core.cpu().numpy())
+    np.testing.assert_array_equal(hdW.numpy(), run.dW.cpu().numpy())
