@@ -55,7 +55,10 @@ def _rotate(Ustar, rng, theta):
     d = Ustar.shape[0]
     X = rng.standard_normal((d, d))
     K = X - X.T
-    K /= _spectral_norm(K, rng)
+    nrm = _spectral_norm(K, rng) if d > 1 else 0.0
+    if nrm == 0.0:                      # a mode of size one has nothing to rotate
+        return Ustar.copy()
+    K /= nrm
     term = Ustar.copy()
     out = Ustar.copy()
     for k in range(1, 9):
