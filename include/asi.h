@@ -151,6 +151,23 @@ asi_status_t asi_poll_status(const asi_plan_t* plan, const void* ws, void* strea
 /* Number of kernel launches the last call of each kind enqueues for this plan. */
 int32_t asi_launch_count(const asi_plan_t* plan, int32_t which /* 0 compress, 1 wgrad */);
 
+/* Timing aid for benchmarks: while active, every launch of kernel family `kernel_id` is
+ * bracketed by cudaEventRecord on its own stream, using the caller's events pairwise:
+ * events[2i] before and events[2i+1] after the i-th such launch (launches beyond n_pairs are
+ * counted but not recorded).  Process-global and not thread-safe: enable it from one thread,
+ * for one measurement pass, never during stream capture.  asi_profile_end returns the number
+ * of launches seen since asi_profile_begin, stores in *alg_bytes (if not null) the sum over
+ * those launches of the bytes each launch must move at least -- its distinct inputs read once
+ * plus its outputs written once -- and switches recording off. */
+typedef enum {
+  ASI_K_MODEPROD = 1,     /* small-mode contraction (projection, core products, Z1, Z3, expansions) */
+  ASI_K_EXPAND = 2,       /* P_m = A_m V_m */
+  ASI_K_QR = 3,           /* Orthogonalize */
+  ASI_K_CONV_TAIL = 4     /* terms 4-5 of the backward cost: Z4 and dW */
+} asi_kernel_id_t;
+asi_status_t asi_profile_begin(int32_t kernel_id, void** events, int32_t n_pairs);
+int32_t asi_profile_end(double* alg_bytes);
+
 const char* asi_status_string(asi_status_t s);
 
 #ifdef __cplusplus

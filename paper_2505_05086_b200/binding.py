@@ -29,7 +29,8 @@ ASI_MAX_MODES = 4
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_init_factors",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host",
-    "asi_poll_status", "asi_launch_count", "asi_status_string",
+    "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
+    "asi_profile_end",
 )
 
 
@@ -80,6 +81,10 @@ def lib():
     L.asi_poll_status.argtypes = [vp, vp, vp, C.POINTER(i32)]
     L.asi_launch_count.argtypes = [vp, i32]
     L.asi_launch_count.restype = i32
+    L.asi_profile_begin.argtypes = [i32, C.POINTER(vp), i32]
+    L.asi_profile_begin.restype = i32
+    L.asi_profile_end.argtypes = [C.POINTER(C.c_double)]
+    L.asi_profile_end.restype = i32
     L.asi_status_string.argtypes = [i32]
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress",
@@ -181,3 +186,20 @@ class Plan:
         out = C.c_int32(0)
         _check(lib().asi_poll_status(self._h, ws, stream, C.byref(out)), "asi_poll_status")
         return out.value
+
+
+KERNEL_IDS = {"modeprod": 1, "expand": 2, "qr": 3, "conv_tail": 4}
+
+
+def profile_begin(kernel_id: int, event_handles):
+    """event_handles: flat list of CUDA event handles, [begin0, end0, begin1, end1, ...]."""
+    n = len(event_handles) // 2
+    arr = (C.c_void_p * (2 * n))(*event_handles)
+    _check(lib().asi_profile_begin(int(kernel_id), arr, n), "asi_profile_begin")
+    return arr            # keep alive until profile_end
+
+
+def profile_end():
+    b = C.c_double(0.0)
+    n = lib().asi_profile_end(C.byref(b))
+    return n, b.value

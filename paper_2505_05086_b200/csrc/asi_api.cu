@@ -510,6 +510,23 @@ asi_status_t asi_step_host(const asi_plan_t* pl, const void* act_host, const voi
   return ASI_OK;
 }
 
+asi_status_t asi_profile_begin(int32_t kernel_id, void** events, int32_t n_pairs) {
+  if (kernel_id < 1 || !events || n_pairs < 1) return ASI_ERR_INVALID_ARG;
+  g_prof.ev = reinterpret_cast<cudaEvent_t*>(events);
+  g_prof.n_pairs = n_pairs;
+  g_prof.used = 0;
+  g_prof.bytes = 0.0;
+  g_prof.id = kernel_id;
+  return ASI_OK;
+}
+
+int32_t asi_profile_end(double* alg_bytes) {
+  const int used = g_prof.used;
+  if (alg_bytes) *alg_bytes = g_prof.bytes;
+  g_prof = ProfState{0, nullptr, 0, 0, 0.0};
+  return used;
+}
+
 asi_status_t asi_poll_status(const asi_plan_t* pl, const void* ws, void* stream,
                              asi_status_t* device_status) {
   if (!pl || !ws || !device_status) return ASI_ERR_INVALID_ARG;

@@ -13,6 +13,8 @@
 
 namespace asi {
 
+ProfState g_prof = {0, nullptr, 0, 0, 0.0};
+
 __device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
@@ -105,6 +107,8 @@ __global__ void __launch_bounds__(128) k_modeprod(ModeProdArgs p) {
 template <typename TX>
 static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
   if (p.Q <= 0 || p.n_out <= 0) return cudaSuccess;
+  ProfScope prof(ASI_K_MODEPROD, st,
+                 (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
   int R = 4;
   while (R < p.n_out && R < 64) R *= 2;
   dim3 grid((unsigned)((p.Q + 127) / 128), (unsigned)((p.n_out + R - 1) / R));
@@ -173,6 +177,8 @@ __global__ void __launch_bounds__(256) k_expand(ExpandArgs p) {
 
 template <typename TX>
 static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
+  ProfScope prof(ASI_K_EXPAND, st,
+                 (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.Q * p.r + (double)p.nsplit * p.a * p.r));
   int R = 8;
   while (R < p.r) R *= 2;
   dim3 grid((unsigned)((p.a + kExpandKC - 1) / kExpandKC), (unsigned)p.nsplit);
@@ -283,6 +289,10 @@ __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
 }
 
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) {
+  double qr_bytes = 0.0;
+  for (int m = 0; m < nd; ++m)
+    qr_bytes += 4.0 * p.m[m].a * p.m[m].r * (p.m[m].nsplit + 1);
+  ProfScope prof(ASI_K_QR, st, qr_bytes);
   dim3 grid((unsigned)max_chunks, (unsigned)nd);
   k_qr_gram<<<grid, 256, 0, st>>>(p);
   cudaError_t e = cudaGetLastError();
@@ -366,6 +376,9 @@ __global__ void __launch_bounds__(256) k_conv_tail(ConvTailArgs p) {
 }
 
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st) {
+  ProfScope prof(ASI_K_CONV_TAIL, st,
+                 4.0 * ((double)p.r1 * p.Cout * p.Ho * p.Wo + (double)p.r1 * p.r2 * p.H * p.W +
+                        (double)p.C * p.r2 + (double)p.Cout * (p.C / p.groups) * p.kh * p.kw));
   const int n_out = p.r2 * p.kh * p.kw;
   const int nsplit_max = (n_out <= 128) ? 256 / n_out : 1;
   const size_t smem = (size_t)(((n_out + 31) / 32) * 32 + (size_t)nsplit_max * n_out) * sizeof(float);

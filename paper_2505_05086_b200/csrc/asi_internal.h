@@ -66,6 +66,32 @@ struct ConvTailArgs {
   int r1, r2, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups;
 };
 
+// Benchmark timing aid (asi_profile_begin / asi_profile_end).
+struct ProfState {
+  int id;
+  cudaEvent_t* ev;
+  int n_pairs, used;
+  double bytes;
+};
+extern ProfState g_prof;
+struct ProfScope {
+  cudaStream_t st;
+  int slot;
+  ProfScope(int id, cudaStream_t s, double alg_bytes) : st(s), slot(-1) {
+    if (g_prof.id == id) {
+      g_prof.bytes += alg_bytes;
+      if (g_prof.used < g_prof.n_pairs) {
+        slot = g_prof.used;
+        cudaEventRecord(g_prof.ev[2 * slot], st);
+      }
+      ++g_prof.used;
+    }
+  }
+  ~ProfScope() {
+    if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], st);
+  }
+};
+
 cudaError_t launch_modeprod(const ModeProdArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_expand(const ExpandArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
