@@ -67,7 +67,12 @@ typedef struct {
   int32_t ranks[ASI_MAX_MODES];  /* 1 <= r_m <= min(a_m, b_m), r_m <= 64 */
   int32_t cout;
   int32_t kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, groups;
+  int32_t flags;                 /* ASI_FLAG_* bits, 0 for defaults */
 } asi_layer_desc_t;
+
+/* Use only the shape-generic kernels even where a fused kernel covers the layer
+ * (same results up to fp32 rounding; for testing and comparison). */
+#define ASI_FLAG_GENERIC_ONLY 1
 
 /* Sizes and the paper's closed forms for one plan. */
 typedef struct {
@@ -163,12 +168,19 @@ typedef enum {
   ASI_K_MODEPROD = 1,     /* small-mode contraction (projection, core products, Z1, Z3, expansions) */
   ASI_K_EXPAND = 2,       /* P_m = A_m V_m */
   ASI_K_QR = 3,           /* Orthogonalize */
-  ASI_K_CONV_TAIL = 4     /* terms 4-5 of the backward cost: Z4 and dW */
+  ASI_K_CONV_TAIL = 4,    /* terms 4-5 of the backward cost: Z4 and dW */
+  ASI_K_SM_PASS1 = 5,     /* small-map conv: all four P_m in one pass over the activation */
+  ASI_K_SM_CORE = 6,      /* small-map conv: core tensor */
+  ASI_K_SM_WGRAD = 7      /* small-map conv: whole compressed weight gradient */
 } asi_kernel_id_t;
 asi_status_t asi_profile_begin(int32_t kernel_id, void** events, int32_t n_pairs);
 int32_t asi_profile_end(double* alg_bytes);
 
 const char* asi_status_string(asi_status_t s);
+
+/* Text of the CUDA runtime error behind the most recent ASI_ERR_CUDA on this thread
+ * ("" if none).  The pointer stays valid until the next failing call. */
+const char* asi_last_cuda_error(void);
 
 #ifdef __cplusplus
 }

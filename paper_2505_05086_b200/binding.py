@@ -30,7 +30,7 @@ EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_init_factors",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
-    "asi_profile_end",
+    "asi_profile_end", "asi_last_cuda_error",
 )
 
 
@@ -40,7 +40,7 @@ class LayerDesc(C.Structure):
                 ("cout", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
                 ("stride_h", C.c_int32), ("stride_w", C.c_int32), ("pad_h", C.c_int32),
                 ("pad_w", C.c_int32), ("dil_h", C.c_int32), ("dil_w", C.c_int32),
-                ("groups", C.c_int32)]
+                ("groups", C.c_int32), ("flags", C.c_int32)]
 
 
 class PlanInfo(C.Structure):
@@ -56,7 +56,10 @@ class PlanInfo(C.Structure):
 class AsiError(RuntimeError):
     def __init__(self, code, where):
         self.code = int(code)
-        super().__init__(f"{where}: {status_string(code)} (status {int(code)})")
+        detail = ""
+        if self.code == ASI_ERR_CUDA:
+            detail = " [" + lib().asi_last_cuda_error().decode() + "]"
+        super().__init__(f"{where}: {status_string(code)} (status {int(code)}){detail}")
 
 
 def lib():
@@ -85,6 +88,8 @@ def lib():
     L.asi_profile_begin.restype = i32
     L.asi_profile_end.argtypes = [C.POINTER(C.c_double)]
     L.asi_profile_end.restype = i32
+    L.asi_last_cuda_error.argtypes = []
+    L.asi_last_cuda_error.restype = C.c_char_p
     L.asi_status_string.argtypes = [i32]
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress",
@@ -104,7 +109,8 @@ def _check(code, where):
         raise AsiError(code, where)
 
 
-def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False, dilation=1):
+def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False, dilation=1,
+              generic_only=False):
     d = LayerDesc()
     d.kind = ASI_CONV2D if kind == "conv" else ASI_LINEAR
     d.in_dtype = ASI_BF16 if bf16 else ASI_F32
@@ -120,6 +126,7 @@ def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=Fals
     d.kh, d.kw, d.stride_h, d.stride_w, d.pad_h, d.pad_w = kh, kw, sh, sw, ph, pw
     d.dil_h = d.dil_w = int(dilation)
     d.groups = int(groups)
+    d.flags = 1 if generic_only else 0
     return d
 
 
@@ -128,9 +135,10 @@ class Plan:
     integers (device or host addresses), ``stream`` is a CUDA stream handle (0 = default)."""
 
     def __init__(self, kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False,
-                 dilation=1):
+                 dilation=1, generic_only=False):
         self._h = C.c_void_p()
-        self.desc = make_desc(kind, dims, ranks, cout, k, stride, pad, groups, bf16, dilation)
+        self.desc = make_desc(kind, dims, ranks, cout, k, stride, pad, groups, bf16, dilation,
+                              generic_only)
         _check(lib().asi_plan_create(C.byref(self.desc), C.byref(self._h)), "asi_plan_create")
         self.kind = kind
         self.info = PlanInfo()
@@ -188,7 +196,8 @@ class Plan:
         return out.value
 
 
-KERNEL_IDS = {"modeprod": 1, "expand": 2, "qr": 3, "conv_tail": 4}
+KERNEL_IDS = {"modeprod": 1, "expand": 2, "qr": 3, "conv_tail": 4, "sm_pass1": 5, "sm_core": 6,
+              "sm_wgrad": 7}
 
 
 def profile_begin(kernel_id: int, event_handles):

@@ -1,5 +1,6 @@
 // C ABI of the ASI library: plan construction (host only) and the enqueue sequences.
 #include <algorithm>
+#include <cstdio>
 #include <cstring>
 #include <new>
 
@@ -22,11 +23,52 @@ void set_mode_views(asi_plan* pl) {
   }
 }
 
-// Workspace layouts.  Every region is 256-byte aligned; region 0 is the status word.
+constexpr size_t kSmemLimit = 200 * 1024;
+
+// Which fused kernels cover this layer (decided once, at plan creation).
+void choose_kernels(asi_plan* pl) {
+  pl->fast_compress = pl->fast_wgrad = false;
+  pl->fast_S = pl->fast_R = pl->n_tiles_b = pl->cpb = 0;
+  if (pl->d.kind != ASI_CONV2D || (pl->d.flags & ASI_FLAG_GENERIC_ONLY)) return;
+  int rmax = 0;
+  for (int m = 0; m < 4; ++m) rmax = std::max(rmax, pl->r[m]);
+  if (rmax > 8) return;
+  const int R = rmax <= 4 ? 4 : 8;
+  pl->fast_R = R;
+  const int64_t B = pl->dims[0], C = pl->dims[1], H = pl->dims[2], W = pl->dims[3];
+  if (H == W && (H == 7 || H == 14 || H == 16) && B % 8 == 0 && B <= 1024 && C <= 4096 &&
+      (H != 7 || C % 4 == 0)) {
+    const int S = (int)H;
+    if (sm_pass1_smem(S, R, (int)B, (int)C) <= kSmemLimit && sm_core_smem(S, R, (int)C) <= kSmemLimit) {
+      pl->fast_compress = true;
+      pl->fast_S = S;
+      pl->n_tiles_b = (int)((S == 7) ? C / 4 : C);
+    }
+  }
+  if (B <= 4096 && H <= 64 && W <= 64) {
+    const int Cout = pl->d.cout;
+    int cpb = 1;
+    if (Cout % 4 == 0 && Cout / 4 >= 256) cpb = 4;
+    else if (Cout % 2 == 0 && Cout / 2 >= 200) cpb = 2;
+    SmWgradArgs a;
+    std::memset(&a, 0, sizeof(a));
+    for (int m = 0; m < 4; ++m) a.r[m] = pl->r[m];
+    a.B = (int)B; a.C = (int)C; a.Cout = Cout; a.H = (int)H; a.W = (int)W;
+    a.Ho = (int)pl->Ho; a.Wo = (int)pl->Wo; a.kh = pl->d.kh; a.kw = pl->d.kw; a.cpb = cpb;
+    if (sm_wgrad_smem(a, R) <= kSmemLimit) {
+      pl->fast_wgrad = true;
+      pl->cpb = cpb;
+    }
+  }
+}
+
+// Workspace layouts.  Every region is 256-byte aligned; region 0 holds the status word (byte 0)
+// and the completion counter of the core kernel (byte 64).
 void layout_compress(asi_plan* pl) {
   size_t off = kStatusBytes;
   int64_t vmax = 0;
-  for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
+  if (!pl->fast_compress)
+    for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
   pl->off_V = off;
   off = align_up(off + (size_t)vmax * 4, 256);
   for (int m = 0; m < pl->nd; ++m) {
@@ -38,6 +80,7 @@ void layout_compress(asi_plan* pl) {
     int64_t qps = (v.Q + ns - 1) / ns;
     qps = (qps + 63) / 64 * 64;
     ns = (v.Q + qps - 1) / qps;
+    if (pl->fast_compress) ns = (m == 1) ? pl->dims[0] : pl->n_tiles_b;   // one partial per tile
     pl->nsplit[m] = (int)ns;
     pl->q_per_split[m] = qps;
     pl->nchunk[m] = (int)((v.a + kQRRows - 1) / kQRRows);
@@ -66,12 +109,16 @@ void layout_compress(asi_plan* pl) {
     for (int m = 0; m < pl->nd; ++m) n *= cd[m];
     tmax[s & 1] = std::max(tmax[s & 1], n);
   }
+  if (pl->fast_compress) {
+    tmax[0] = pl->dims[0] * pl->r[1] * pl->r[2] * pl->r[3];   // per-sample partial cores
+    tmax[1] = 0;
+  }
   for (int t = 0; t < 2; ++t) {
     pl->off_T[t] = off;
     off = align_up(off + (size_t)tmax[t] * 4, 256);
   }
   pl->compress_ws = off;
-  pl->launches_compress = 2 * pl->nd + 2 + pl->nd;
+  pl->launches_compress = pl->fast_compress ? 4 : 2 * pl->nd + 2 + pl->nd;
 }
 
 void layout_wgrad(asi_plan* pl) {
@@ -81,7 +128,7 @@ void layout_wgrad(asi_plan* pl) {
     z[0] = (int64_t)pl->r[0] * pl->d.cout * pl->Ho * pl->Wo;          // Z1
     z[1] = (int64_t)pl->r[0] * pl->r[1] * pl->dims[2] * pl->r[3];     // core x_3 U_3
     z[2] = (int64_t)pl->r[0] * pl->r[1] * pl->dims[2] * pl->dims[3];  // Z3
-    pl->launches_wgrad = 4;
+    pl->launches_wgrad = pl->fast_wgrad ? 1 : 4;
   } else {
     const int nlead = pl->nd - 1;
     int64_t rest = pl->d.cout;
@@ -104,15 +151,19 @@ asi_status_t check_ws(const void* ws, size_t have, size_t need) {
   return ASI_OK;
 }
 
-#define ASI_CUDA(call)                         \
-  do {                                         \
-    cudaError_t e__ = (call);                  \
-    if (e__ != cudaSuccess) return ASI_ERR_CUDA; \
+thread_local char g_cuda_err[256] = "";
+
+#define ASI_CUDA(call)                                                        \
+  do {                                                                        \
+    cudaError_t e__ = (call);                                                 \
+    if (e__ != cudaSuccess) {                                                 \
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", #call, cudaGetErrorString(e__)); \
+      return ASI_ERR_CUDA;                                                    \
+    }                                                                         \
   } while (0)
 
-// U_m^{new} = Orthogonalize(P_m) for all modes given the split partials, then the core.
-asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, float* core,
-                             char* w, cudaStream_t st) {
+// U_m^{new} = Orthogonalize(P_m) for all modes given the split partials.
+asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, cudaStream_t st) {
   QRArgs qa;
   std::memset(&qa, 0, sizeof(qa));
   int max_chunks = 1;
@@ -129,8 +180,30 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
   }
   qa.status = reinterpret_cast<int*>(w);
   ASI_CUDA(launch_qr(qa, pl->nd, max_chunks, st));
+  return ASI_OK;
+}
 
-  // core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T)
+// Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).
+asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, float* core,
+                             char* w, cudaStream_t st) {
+  asi_status_t qs = orthogonalize_all(pl, U_new, w, st);
+  if (qs != ASI_OK) return qs;
+  if (pl->fast_compress) {
+    SmCoreArgs c;
+    c.act = act;
+    c.U = U_new;
+    c.Tb = reinterpret_cast<float*>(w + pl->off_T[0]);
+    c.core = core;
+    c.counter = reinterpret_cast<int*>(w + 64);
+    for (int m = 0; m < 4; ++m) {
+      c.u_off[m] = pl->u_off[m];
+      c.r[m] = pl->r[m];
+    }
+    c.B = (int)pl->dims[0];
+    c.C = (int)pl->dims[1];
+    ASI_CUDA(launch_sm_core(c, pl->fast_S, pl->fast_R, pl->bf16, st));
+    return ASI_OK;
+  }
   int64_t cd[ASI_MAX_MODES];
   for (int m = 0; m < pl->nd; ++m) cd[m] = pl->dims[m];
   const void* src = act;
@@ -198,6 +271,8 @@ const char* asi_status_string(asi_status_t s) {
   return "unknown status";
 }
 
+const char* asi_last_cuda_error(void) { return g_cuda_err; }
+
 asi_status_t asi_plan_create(const asi_layer_desc_t* desc, asi_plan_t** out) {
   if (!desc || !out) return ASI_ERR_INVALID_ARG;
   const asi_layer_desc_t& d = *desc;
@@ -257,6 +332,7 @@ asi_status_t asi_plan_create(const asi_layer_desc_t* desc, asi_plan_t** out) {
     pl->dw_elems = (int64_t)d.cout * d.dims[d.ndim - 1];
   }
   set_mode_views(pl);
+  choose_kernels(pl);
   layout_compress(pl);
   layout_wgrad(pl);
   *out = pl;
@@ -319,6 +395,21 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
   ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
+  if (pl->fast_compress) {
+    SmPass1Args a;
+    a.act = act;
+    a.U_prev = U_prev;
+    for (int m = 0; m < 4; ++m) {
+      a.Pp[m] = reinterpret_cast<float*>(w + pl->off_Pp[m]);
+      a.u_off[m] = pl->u_off[m];
+      a.r[m] = pl->r[m];
+    }
+    a.B = (int)pl->dims[0];
+    a.C = (int)pl->dims[1];
+    a.n_tiles_b = pl->n_tiles_b;
+    ASI_CUDA(launch_sm_pass1(a, pl->fast_S, pl->fast_R, pl->bf16, st));
+    return finish_compress(pl, act, U_new, core, w, st);
+  }
   float* V = reinterpret_cast<float*>(w + pl->off_V);
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
@@ -372,6 +463,20 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
   if (s != ASI_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
+  if (pl->fast_wgrad) {
+    SmWgradArgs g;
+    g.core = core; g.U = U; g.dY = dY; g.dW = dW;
+    for (int m = 0; m < 4; ++m) {
+      g.u_off[m] = pl->u_off[m];
+      g.r[m] = pl->r[m];
+    }
+    g.B = (int)pl->dims[0]; g.C = (int)pl->dims[1]; g.Cout = pl->d.cout;
+    g.H = (int)pl->dims[2]; g.W = (int)pl->dims[3]; g.Ho = (int)pl->Ho; g.Wo = (int)pl->Wo;
+    g.kh = pl->d.kh; g.kw = pl->d.kw; g.sh = pl->d.stride_h; g.sw = pl->d.stride_w;
+    g.ph = pl->d.pad_h; g.pw = pl->d.pad_w; g.groups = pl->d.groups; g.cpb = pl->cpb;
+    ASI_CUDA(launch_sm_wgrad(g, pl->fast_R, pl->bf16, st));
+    return ASI_OK;
+  }
   float* Z1 = reinterpret_cast<float*>(w + pl->off_Z[0]);
   float* Z3a = reinterpret_cast<float*>(w + pl->off_Z[1]);
   float* Z3 = reinterpret_cast<float*>(w + pl->off_Z[2]);

@@ -66,6 +66,41 @@ struct ConvTailArgs {
   int r1, r2, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups;
 };
 
+// Fused small-map conv kernels (asi_smallmap_kernels.cu)
+struct SmPass1Args {
+  const void* act;
+  const float* U_prev;
+  float* Pp[ASI_MAX_MODES];     // per-mode partials [nsplit][a_m][r_m]
+  int64_t u_off[ASI_MAX_MODES];
+  int r[ASI_MAX_MODES];
+  int B, C, n_tiles_b;
+};
+struct SmCoreArgs {
+  const void* act;
+  const float* U;
+  float* Tb;                    // [B][r2 r3 r4]
+  float* core;
+  int* counter;                 // zero on entry, zero again on exit
+  int64_t u_off[ASI_MAX_MODES];
+  int r[ASI_MAX_MODES];
+  int B, C;
+};
+struct SmWgradArgs {
+  const float* core;
+  const float* U;
+  const void* dY;
+  float* dW;
+  int64_t u_off[ASI_MAX_MODES];
+  int r[ASI_MAX_MODES];
+  int B, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups, cpb;
+};
+size_t sm_pass1_smem(int S, int R, int B, int C);
+size_t sm_core_smem(int S, int R, int C);
+size_t sm_wgrad_smem(const SmWgradArgs& p, int R);
+cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st);
+cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
+cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t st);
+
 // Benchmark timing aid (asi_profile_begin / asi_profile_end).
 struct ProfState {
   int id;
@@ -122,4 +157,8 @@ struct asi_plan {
   size_t wgrad_ws;
 
   int launches_compress, launches_wgrad;
+
+  // fused small-map path
+  bool fast_compress, fast_wgrad;
+  int fast_S, fast_R, n_tiles_b, cpb;
 };

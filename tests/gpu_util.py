@@ -8,13 +8,13 @@ TOL_F32 = dict(proj=1e-4, core=1e-4, dw=5e-4)     # relative Frobenius error, fp
 TOL_BF16 = dict(proj=2e-2, core=2e-2, dw=2e-2)    # bf16-input mode
 
 
-def make_runner(L, ranks=None, bf16=False):
+def make_runner(L, ranks=None, bf16=False, generic_only=False):
     from paper_2505_05086_b200.runner import LayerRunner
     r = tuple(ranks if ranks is not None else L.ranks)
     if L.kind == "linear":
-        return LayerRunner("linear", L.dims, r, L.cout, bf16=bf16)
+        return LayerRunner("linear", L.dims, r, L.cout, bf16=bf16, generic_only=generic_only)
     return LayerRunner("conv", L.dims, r, L.cout, k=L.k, stride=L.stride, pad=L.pad,
-                       groups=L.groups, bf16=bf16)
+                       groups=L.groups, bf16=bf16, generic_only=generic_only)
 
 
 def oracle_wgrad(L, S, U, dY):

@@ -9,10 +9,10 @@ from tests.gpu_util import TOL_BF16, TOL_F32, check, compare_step, make_runner
 pytestmark = pytest.mark.gpu
 
 
-def _layer_steps(cfg, li, steps, tol):
+def _layer_steps(cfg, li, steps, tol, generic_only=False):
     L = cfg.layers[li]
     st = make_stream(cfg, li)
-    run = make_runner(L, bf16=cfg.bf16)
+    run = make_runner(L, bf16=cfg.bf16, generic_only=generic_only)
     U_prev = st.u_prev0()
     for t in range(steps):
         A, dY = st.next()
@@ -20,14 +20,21 @@ def _layer_steps(cfg, li, steps, tol):
         check(err, tol, f"{cfg.name}/{L.name}/step{t}: {err}")
 
 
+@pytest.mark.parametrize("generic_only", [False, True])
 @pytest.mark.parametrize("li", [0, 1, 2, 3])
-def test_config2_resnet18_last4(li):
-    _layer_steps(get_config(1), li, 3, TOL_F32)
+def test_config2_resnet18_last4(li, generic_only):
+    _layer_steps(get_config(1), li, 3, TOL_F32, generic_only)
 
 
+@pytest.mark.parametrize("generic_only", [False, True])
 @pytest.mark.parametrize("li", [0, 1, 2, 3, 4])
-def test_config3_mobilenetv2_last5(li):
-    _layer_steps(get_config(2), li, 2, TOL_F32)
+def test_config3_mobilenetv2_last5(li, generic_only):
+    _layer_steps(get_config(2), li, 2, TOL_F32, generic_only)
+
+
+@pytest.mark.parametrize("li", [6, 9])
+def test_config4_small_maps_generic_kernels(li):
+    _layer_steps(get_config(3, energy=0.9), li, 1, TOL_F32, generic_only=True)
 
 
 @pytest.mark.parametrize("li", range(10))

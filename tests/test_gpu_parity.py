@@ -67,6 +67,37 @@ def test_small_ragged_conv_layers(case):
         check(err, TOL_F32, str(case))
 
 
+FUSED = [  # shapes the fused small-map kernels cover; (dims, ranks, cout, k, s, p, groups, bf16)
+    ((8, 12, 7, 7), (3, 4, 3, 2), 10, 3, 1, 1, 1, False),
+    ((16, 20, 7, 7), (5, 8, 4, 4), 12, 1, 1, 0, 1, False),        # ranks in the 5..8 bucket, 1x1
+    ((8, 16, 7, 7), (2, 3, 3, 3), 16, 3, 1, 1, 16, False),        # depthwise
+    ((16, 6, 14, 14), (4, 3, 4, 4), 8, 3, 2, 1, 1, False),        # stride 2: 14x14 -> 7x7
+    ((8, 5, 14, 14), (3, 5, 6, 5), 6, 3, 1, 1, 1, False),         # 14x14 with ranks above 4
+    ((8, 4, 16, 16), (2, 4, 4, 4), 4, 5, 1, 2, 1, False),         # 16x16, 5x5 kernel
+    ((24, 8, 7, 7), (4, 4, 4, 4), 6, 3, 1, 1, 2, True),           # bf16 inputs, two groups
+]
+
+
+@pytest.mark.parametrize("case", FUSED)
+def test_fused_small_map_kernels(case):
+    dims, ranks, cout, k, s, p, g, bf16 = case
+    L = LayerSpec("t", "conv", dims, cout, k, s, p, g, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=sum(dims) + 7 * k,
+                     rho=tuple(_rho(r) for r in ranks), bf16=bf16,
+                     gen_ranks=tuple(min(d, max(r + 2, 4)) for d, r in zip(dims, ranks)))
+    run = make_runner(L, bf16=bf16)
+    assert run.plan.launch_count(0) == 4 and run.plan.launch_count(1) == 1   # fused path chosen
+    gen = make_runner(L, bf16=bf16, generic_only=True)
+    assert gen.plan.launch_count(0) > 4
+    U_prev = st.u_prev0()
+    for t in range(2):
+        A, dY = st.next()
+        err_g, _ = compare_step(gen, L, A, dY, U_prev)
+        check(err_g, TOL_F32, f"generic {case}")
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, TOL_F32, f"fused {case}")
+
+
 def test_full_rank_reproduces_vanilla_gradient():
     dims, cout = (3, 6, 5, 4), 5
     L = LayerSpec("t", "conv", dims, cout, 3, 1, 1, 1, ranks=dims)
