@@ -37,14 +37,16 @@ WORKLOADS = {0: "single-conv(8x32x16x16,r=4,8,8,8)", 1: "resnet18-last4-convs(B=
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="0-based workload index (default: ResNet-18 last 4 convs)")
     ap.add_argument("--sets", type=int, default=8, help="distinct input sets rotated through the timed loop")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying CUDA graphs")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="only the device-resident timed loop (no end-to-end, per-kernel or CPU legs)")
     return ap.parse_args()
 
 
@@ -149,6 +151,8 @@ def run_reference(args):
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
+    """nvidia-smi polled in a child process; rows are stamped with the host clock on arrival so the
+    ones that fall inside the timed region can be picked out afterwards."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -156,33 +160,41 @@ class ClockSampler:
         self.rows, self.proc, self.thr = [], None, None
         self.gpu = gpu_index
 
-    def start(self):
+    def start(self, wait_s=4.0):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.gpu),
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
         self.thr = threading.Thread(target=self._read, daemon=True)
         self.thr.start()
+        t0 = time.monotonic()
+        while not self.rows and time.monotonic() - t0 < wait_s:     # first row: the poller is up
+            time.sleep(0.02)
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.monotonic(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
+        inside = [r for t, r in self.rows if t_begin is not None and t_begin <= t <= t_end]
+        window = "timed region"
+        if len(inside) < 3:                   # region shorter than a few polls: use every row under load
+            inside = [r for t, r in self.rows if t_begin is None or t >= t_begin - 1.0]
+            window = "warm-up and timed region"
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in inside:
             f = [x.strip() for x in r.split(",")]
             if len(f) < 6:
                 continue
@@ -195,7 +207,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -249,6 +261,7 @@ def run_ours(args):
     elem = 2 if cfg.bf16 else 4
     set_bytes = sum(r.plan.info.act_elems * elem + r.plan.info.dy_elems * elem for r in runners)
     stream = torch.cuda.Stream(device=dev)
+    side = [torch.cuda.Stream(device=dev) for _ in range(nl)]
 
     def step(i):
         s = i % args.sets
@@ -263,32 +276,84 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     launches_per_step = sum(r.plan.launch_count(0) + r.plan.launch_count(1) for r in runners)
+    if args.sets % 2:
+        raise SystemExit("--sets must be even (the two factor buffers of a layer alternate every step)")
+
+    # One CUDA graph per input set: the layers of a step are independent of one another (each compress
+    # reads only its own layer's activation, each wgrad its own dY), so every layer is its own branch.
+    graphs = None
+    with torch.cuda.stream(stream):
+        for i in range(max(2, min(args.warmup, args.sets))):
+            step(i)
+    torch.cuda.synchronize()
+    if not args.no_graph:
+        graphs = []
+        for s in range(args.sets):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                cur = torch.cuda.current_stream()
+                for li in range(nl):
+                    side[li].wait_stream(cur)
+                    runners[li].compress(acts[li][s], side[li])
+                for li in reversed(range(nl)):
+                    runners[li].wgrad(dys[li][s], side[li])
+                for li in range(nl):
+                    cur.wait_stream(side[li])
+            graphs.append(g)
+
+    def run_step(i):
+        if graphs is None:
+            step(i)
+        else:
+            graphs[i % args.sets].replay()
 
     # ---- device-resident timing --------------------------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     with torch.cuda.stream(stream):
         for i in range(args.warmup):
-            step(i)
+            run_step(i)
         barrier()
-        sampler = ClockSampler(local)
-        if rank == 0:
-            sampler.start()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
+        t_begin = time.monotonic()
         e0.record(stream)
         for i in range(args.steps):
-            step(args.warmup + i)
+            run_step(args.warmup + i)
         e1.record(stream)
         barrier()
+        t_end = time.monotonic()
         ms = e0.elapsed_time(e1)
-        clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     for r in runners:
         if not r.ok():
-            raise SystemExit("device status: rank-deficient iterate during the timed loop")
+            raise SystemExit("device status: the timed loop reported an error (rank-deficient iterate or timeout)")
     t = torch.tensor([ms], device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms = float(t.item())
     value = world * nl * args.steps / (ms * 1e-3)
+
+    if args.timed_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                              "warmup": args.warmup, "ms_per_step": ms / args.steps, "timed_only": True,
+                              "launch": "direct" if graphs is None else "cuda-graph", "clocks": clocks}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # the same steps launched kernel by kernel on one stream (no graph), for comparison
+    k_serial = max(10, min(args.steps, 300))
+    with torch.cuda.stream(stream):
+        barrier()
+        e0.record(stream)
+        for i in range(k_serial):
+            step(i)
+        e1.record(stream)
+        barrier()
+        serial_value = nl * k_serial / (e0.elapsed_time(e1) * 1e-3)
 
     # ---- end to end from pinned host buffers --------------------------------------------------
     arenas = [torch.empty(r.plan.step_host_arena_bytes(), dtype=torch.uint8, device=dev) for r in runners]
@@ -374,6 +439,9 @@ def run_ours(args):
                    "ranks": [list(L.ranks) for L in cfg.layers], "in_dtype": "bf16" if cfg.bf16 else "f32",
                    "l2_policy": f"inputs larger than L2: {args.sets} rotating input sets, "
                                 f"{args.sets * set_bytes / 1e6:.0f} MB of act+dY",
+                   "launch": ("direct launches on one stream" if graphs is None else
+                              "CUDA-graph replay, one graph per input set, one branch per layer"),
+                   "single_stream_direct_launch_value": serial_value,
                    "multi_gpu": "replicas only (one independent copy of the workload per GPU)"},
         "activation_GBps": sum(r.plan.info.act_elems * elem for r in runners) * args.steps / (ms * 1e-3) / 1e9,
         "e2e": e2e, "gpu_launches": int(launches_per_step * args.steps), "clocks": clocks, "roofline": roofline,

@@ -23,7 +23,7 @@ void set_mode_views(asi_plan* pl) {
   }
 }
 
-constexpr size_t kSmemLimit = 200 * 1024;
+constexpr size_t kSmemLimit = 208 * 1024;
 
 // Which fused kernels cover this layer (decided once, at plan creation).
 void choose_kernels(asi_plan* pl) {
@@ -39,7 +39,8 @@ void choose_kernels(asi_plan* pl) {
   if (H == W && (H == 7 || H == 14 || H == 16) && B % 8 == 0 && B <= 1024 && C <= 4096 &&
       (H != 7 || C % 4 == 0)) {
     const int S = (int)H;
-    if (sm_pass1_smem(S, R, (int)B, (int)C) <= kSmemLimit && sm_core_smem(S, R, (int)C) <= kSmemLimit) {
+    if (sm_pass1_smem(S, R, (int)B, (int)C) <= kSmemLimit && sm_core_smem(S, R, (int)B) <= kSmemLimit &&
+        B + 4 + 2 * S <= sm_core_max_rows()) {
       pl->fast_compress = true;
       pl->fast_S = S;
       pl->n_tiles_b = (int)((S == 7) ? C / 4 : C);
@@ -47,9 +48,12 @@ void choose_kernels(asi_plan* pl) {
   }
   if (B <= 4096 && H <= 64 && W <= 64) {
     const int Cout = pl->d.cout;
+    const int64_t HoWo = pl->Ho * pl->Wo;
+    // channels per CTA: the smallest count that makes a staged row a multiple of 16 bytes
     int cpb = 1;
-    if (Cout % 4 == 0 && Cout / 4 >= 256) cpb = 4;
-    else if (Cout % 2 == 0 && Cout / 2 >= 200) cpb = 2;
+    while (cpb < 4 && ((cpb * HoWo * 4) % 16 != 0 || Cout % cpb != 0)) cpb *= 2;
+    const bool rows_ok = (cpb * HoWo * 4) % 16 == 0 && Cout % cpb == 0;
+    if (!rows_ok) cpb = 1;
     SmWgradArgs a;
     std::memset(&a, 0, sizeof(a));
     for (int m = 0; m < 4; ++m) a.r[m] = pl->r[m];
@@ -58,6 +62,7 @@ void choose_kernels(asi_plan* pl) {
     if (sm_wgrad_smem(a, R) <= kSmemLimit) {
       pl->fast_wgrad = true;
       pl->cpb = cpb;
+      pl->wgrad_bulk = rows_ok && !pl->bf16;
     }
   }
 }
@@ -80,12 +85,16 @@ void layout_compress(asi_plan* pl) {
     int64_t qps = (v.Q + ns - 1) / ns;
     qps = (qps + 63) / 64 * 64;
     ns = (v.Q + qps - 1) / qps;
-    if (pl->fast_compress) ns = (m == 1) ? pl->dims[0] : pl->n_tiles_b;   // one partial per tile
+    if (pl->fast_compress)                                               // one partial per tile
+      ns = (m == 1) ? sm_pass1_role_c_ctas(pl->fast_S, (int)pl->dims[0]) : pl->n_tiles_b;
     pl->nsplit[m] = (int)ns;
     pl->q_per_split[m] = qps;
-    pl->nchunk[m] = (int)((v.a + kQRRows - 1) / kQRRows);
+    const int qr_rows = pl->fast_compress ? kRedRows : kQRRows;
+    pl->nchunk[m] = (int)((v.a + qr_rows - 1) / qr_rows);
     pl->off_Pp[m] = off;
-    off = align_up(off + (size_t)ns * v.a * v.r * 4, 256);
+    size_t pp_elems = (size_t)ns * v.a * v.r;
+    if (pl->fast_compress && pl->fast_S == 7 && m >= 2) pp_elems = std::max(pp_elems, (size_t)ns * v.a * v.a);
+    off = align_up(off + pp_elems * 4, 256);
     pl->off_Pred[m] = off;
     off = align_up(off + (size_t)v.a * v.r * 8, 256);
     pl->off_Gp[m] = off;
@@ -110,7 +119,7 @@ void layout_compress(asi_plan* pl) {
     tmax[s & 1] = std::max(tmax[s & 1], n);
   }
   if (pl->fast_compress) {
-    tmax[0] = pl->dims[0] * pl->r[1] * pl->r[2] * pl->r[3];   // per-sample partial cores
+    tmax[0] = (int64_t)pl->n_tiles_b * pl->core_elems;          // per-tile partial cores
     tmax[1] = 0;
   }
   for (int t = 0; t < 2; ++t) {
@@ -118,7 +127,7 @@ void layout_compress(asi_plan* pl) {
     off = align_up(off + (size_t)tmax[t] * 4, 256);
   }
   pl->compress_ws = off;
-  pl->launches_compress = pl->fast_compress ? 4 : 2 * pl->nd + 2 + pl->nd;
+  pl->launches_compress = pl->fast_compress ? 3 : 2 * pl->nd + 2 + pl->nd;
 }
 
 void layout_wgrad(asi_plan* pl) {
@@ -163,10 +172,33 @@ thread_local char g_cuda_err[256] = "";
   } while (0)
 
 // U_m^{new} = Orthogonalize(P_m) for all modes given the split partials.
-asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, cudaStream_t st) {
+// gram_U_prev != nullptr: the partials of modes 3 and 4 of a 7x7 map are Gram matrices A_m A_m^T
+// (written by the fused first pass) and P_m = G_m U_m^prev is formed during the reduction.
+asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const float* gram_U_prev,
+                               cudaStream_t st) {
+  int max_chunks = 1;
+  for (int m = 0; m < pl->nd; ++m) max_chunks = std::max(max_chunks, pl->nchunk[m]);
+  if (pl->fast_compress) {
+    SmReduceArgs ra;
+    std::memset(&ra, 0, sizeof(ra));
+    for (int m = 0; m < pl->nd; ++m) {
+      ra.m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
+      ra.m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
+      ra.m[m].Gp = reinterpret_cast<double*>(w + pl->off_Gp[m]);
+      ra.m[m].a = (int)pl->dims[m];
+      ra.m[m].r = pl->r[m];
+      ra.m[m].nsplit = pl->nsplit[m];
+      ra.m[m].nchunk = pl->nchunk[m];
+      if (gram_U_prev && pl->fast_S == 7 && m >= 2) {
+        ra.m[m].gram = 1;
+        ra.m[m].Uprev = gram_U_prev + pl->u_off[m];
+      }
+    }
+    ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
+    return ASI_OK;      // the core kernel finishes the factorisation
+  }
   QRArgs qa;
   std::memset(&qa, 0, sizeof(qa));
-  int max_chunks = 1;
   for (int m = 0; m < pl->nd; ++m) {
     qa.m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
     qa.m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
@@ -176,7 +208,6 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, cudaSt
     qa.m[m].r = pl->r[m];
     qa.m[m].nsplit = pl->nsplit[m];
     qa.m[m].nchunk = pl->nchunk[m];
-    max_chunks = std::max(max_chunks, pl->nchunk[m]);
   }
   qa.status = reinterpret_cast<int*>(w);
   ASI_CUDA(launch_qr(qa, pl->nd, max_chunks, st));
@@ -185,22 +216,27 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, cudaSt
 
 // Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).
 asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, float* core,
-                             char* w, cudaStream_t st) {
-  asi_status_t qs = orthogonalize_all(pl, U_new, w, st);
+                             char* w, const float* gram_U_prev, cudaStream_t st) {
+  asi_status_t qs = orthogonalize_all(pl, U_new, w, gram_U_prev, st);
   if (qs != ASI_OK) return qs;
   if (pl->fast_compress) {
     SmCoreArgs c;
     c.act = act;
-    c.U = U_new;
-    c.Tb = reinterpret_cast<float*>(w + pl->off_T[0]);
+    c.U_new = U_new;
+    c.Tp = reinterpret_cast<float*>(w + pl->off_T[0]);
     c.core = core;
-    c.counter = reinterpret_cast<int*>(w + 64);
+    c.status = reinterpret_cast<int*>(w);
+    c.counter = reinterpret_cast<int*>(w) + 16;
     for (int m = 0; m < 4; ++m) {
+      c.Pred[m] = reinterpret_cast<const double*>(w + pl->off_Pred[m]);
+      c.Gp[m] = reinterpret_cast<const double*>(w + pl->off_Gp[m]);
+      c.nchunk[m] = pl->nchunk[m];
       c.u_off[m] = pl->u_off[m];
       c.r[m] = pl->r[m];
     }
     c.B = (int)pl->dims[0];
     c.C = (int)pl->dims[1];
+    c.n_tiles = pl->n_tiles_b;
     ASI_CUDA(launch_sm_core(c, pl->fast_S, pl->fast_R, pl->bf16, st));
     return ASI_OK;
   }
@@ -394,8 +430,9 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   if (s != ASI_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
-  ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
   if (pl->fast_compress) {
+    // fp32 tiles are staged by the bulk-copy engine, which needs 16-byte aligned sources
+    if (!pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
     SmPass1Args a;
     a.act = act;
     a.U_prev = U_prev;
@@ -404,12 +441,14 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
       a.u_off[m] = pl->u_off[m];
       a.r[m] = pl->r[m];
     }
+    a.status = reinterpret_cast<int*>(w);     // cleared by the kernel itself
     a.B = (int)pl->dims[0];
     a.C = (int)pl->dims[1];
     a.n_tiles_b = pl->n_tiles_b;
     ASI_CUDA(launch_sm_pass1(a, pl->fast_S, pl->fast_R, pl->bf16, st));
-    return finish_compress(pl, act, U_new, core, w, st);
+    return finish_compress(pl, act, U_new, core, w, U_prev, st);
   }
+  ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
   float* V = reinterpret_cast<float*>(w + pl->off_V);
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
@@ -433,7 +472,7 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     s = expand_mode(pl, m, act, V, w, st);
     if (s != ASI_OK) return s;
   }
-  return finish_compress(pl, act, U_new, core, w, st);
+  return finish_compress(pl, act, U_new, core, w, nullptr, st);
 }
 
 asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float* omega, float* U_new,
@@ -444,6 +483,7 @@ asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float
   if (s != ASI_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
+  if (pl->fast_compress && !pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
   ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
   int64_t off = 0;
   for (int m = 0; m < pl->nd; ++m) {
@@ -451,7 +491,7 @@ asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float
     if (s != ASI_OK) return s;
     off += pl->mv[m].Q * pl->r[m];
   }
-  return finish_compress(pl, act, U_new, core, w, st);
+  return finish_compress(pl, act, U_new, core, w, nullptr, st);
 }
 
 asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float* U, const void* dY,
@@ -474,6 +514,10 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
     g.H = (int)pl->dims[2]; g.W = (int)pl->dims[3]; g.Ho = (int)pl->Ho; g.Wo = (int)pl->Wo;
     g.kh = pl->d.kh; g.kw = pl->d.kw; g.sh = pl->d.stride_h; g.sw = pl->d.stride_w;
     g.ph = pl->d.pad_h; g.pw = pl->d.pad_w; g.groups = pl->d.groups; g.cpb = pl->cpb;
+    g.pj = sm_wgrad_pitch(pl->cpb * (int)(pl->Ho * pl->Wo));
+    g.bulk = pl->wgrad_bulk ? 1 : 0;
+    if (g.bulk && (reinterpret_cast<uintptr_t>(dY) & 15u)) return ASI_ERR_INVALID_ARG;
+    g.status = reinterpret_cast<int*>(w);
     ASI_CUDA(launch_sm_wgrad(g, pl->fast_R, pl->bf16, st));
     return ASI_OK;
   }

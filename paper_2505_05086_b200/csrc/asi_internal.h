@@ -67,37 +67,63 @@ struct ConvTailArgs {
 };
 
 // Fused small-map conv kernels (asi_smallmap_kernels.cu)
+constexpr int kRedRows = 16;         // rows of P per CTA in the partial-reduction kernel
 struct SmPass1Args {
   const void* act;
   const float* U_prev;
   float* Pp[ASI_MAX_MODES];     // per-mode partials [nsplit][a_m][r_m]
+  int* status;                  // status word (int 0) and completion counters (ints 16..23) of the workspace
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
   int B, C, n_tiles_b;
 };
+// Fixed-order fp64 reduction of the per-tile partials of every P_m, plus per-chunk shares of
+// G_m = P_m^T P_m.
+struct SmReduceMode {
+  const float* Pp;     // [nsplit][a][r], or [nsplit][a][a] Gram matrices A_m A_m^T when gram != 0
+  double* Pred;        // [a][r]
+  double* Gp;          // [nchunk][r][r]
+  const float* Uprev;  // [a][r] previous factor (gram modes only)
+  int a, r, nsplit, nchunk, gram;
+};
+struct SmReduceArgs {
+  SmReduceMode m[ASI_MAX_MODES];
+};
+// Finishes Orthogonalize (Cholesky of G_m, U_m = P_m R_m^{-1}) in its prologue, then the core.
 struct SmCoreArgs {
   const void* act;
-  const float* U;
-  float* Tb;                    // [B][r2 r3 r4]
+  const double* Pred[ASI_MAX_MODES];
+  const double* Gp[ASI_MAX_MODES];
+  int nchunk[ASI_MAX_MODES];
+  float* U_new;
+  float* Tp;                    // [n_tiles][core_elems] per-tile partial cores
   float* core;
+  int* status;
   int* counter;                 // zero on entry, zero again on exit
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
-  int B, C;
+  int B, C, n_tiles;
 };
 struct SmWgradArgs {
   const float* core;
   const float* U;
   const void* dY;
   float* dW;
+  int* status;
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
   int B, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups, cpb;
+  int pj;                       // row pitch (floats) of the staged dY tile
+  int bulk;                     // 1: rows staged by the bulk-copy engine (fp32, 16-byte aligned rows)
 };
 size_t sm_pass1_smem(int S, int R, int B, int C);
-size_t sm_core_smem(int S, int R, int C);
+int sm_pass1_role_c_ctas(int S, int B);
+size_t sm_core_smem(int S, int R, int B);
+int sm_core_max_rows();
 size_t sm_wgrad_smem(const SmWgradArgs& p, int R);
+int sm_wgrad_pitch(int J);
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st);
+cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
 cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t st);
 
@@ -159,6 +185,6 @@ struct asi_plan {
   int launches_compress, launches_wgrad;
 
   // fused small-map path
-  bool fast_compress, fast_wgrad;
+  bool fast_compress, fast_wgrad, wgrad_bulk;
   int fast_S, fast_R, n_tiles_b, cpb;
 };

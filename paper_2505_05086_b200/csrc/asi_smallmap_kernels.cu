@@ -1,16 +1,25 @@
 // Fused kernels for conv layers with small square feature maps (S x S, S in {7, 14, 16}) and
-// ranks <= 8 -- the shapes of the ResNet / MobileNet tails.  One compress call is
+// ranks <= 8 -- the shapes of the ResNet / MobileNet tails.  One compress call is three launches:
 //
-//   k_sm_pass1  : streams the activation once and forms every P_m = A_m (A_m^T U_m^prev)
-//                 (Algorithm 1) tile-locally: CTAs of role B hold tiles [all B x 196..256
-//                 contiguous (c,h,w)] that contain whole mode-1/3/4 fibers, CTAs of role C hold
-//                 one sample [all C x HW] that contains whole mode-2 fibers;
-//   (generic)   : fixed-order fp64 reduction of the per-tile partials + Cholesky-QR;
-//   k_sm_core   : second traversal (L2-resident): per-sample A[b] x_2 U_2^T x_3 U_3^T x_4 U_4^T,
-//                 last CTA folds in U_1^T and writes the core.
+//   k_sm_pass1  : forms every P_m = A_m (A_m^T U_m^prev) (Algorithm 1) tile-locally, so no V_m ever
+//                 reaches global memory.  CTAs of role B hold a tile [all B x J contiguous (c,h,w)]
+//                 that contains whole mode-1/3/4 fibers (one half of the CTA iterates mode 1 while the
+//                 other half does modes 3 and 4); CTAs of role C hold one sample [all C x HW] that
+//                 contains whole mode-2 fibers.  fp32 tiles are staged in shared memory by the
+//                 bulk-copy engine (cp.async.bulk + mbarrier), one row or chunk per copy; the
+//                 activation comes from HBM once, the other role's traversal is served by L2.
+//   k_sm_reduce : fixed-order fp64 reduction of the per-tile partials of every P_m and per-chunk
+//                 shares of the Gram matrices G_m = P_m^T P_m;
+//   k_sm_core   : every CTA finishes Orthogonalize for the factor rows it needs while its tile is in
+//                 flight (Cholesky G_m = R^T R, U_m = P_m R^{-1}: the Gram-Schmidt basis), then
+//                 contracts its tile [all B x J] with U_1..U_4; the last CTA sums the per-tile cores.
 //
 // and the whole compressed weight gradient is one kernel, k_sm_wgrad (terms 1-5 of C_ASI).
+// Every wait on an mbarrier is bounded (about one second); on expiry the CTA records
+// ASI_ERR_TIMEOUT in the status word and returns.
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "asi_internal.h"
 
@@ -18,9 +27,18 @@ namespace asi {
 
 namespace {
 
+constexpr int kNT = 512;             // threads per CTA of the tile kernels
+constexpr int kNG = 256;             // threads of one half (warp-specialised phases)
+constexpr int kRedNT = 256;          // threads per CTA of the partial-reduction kernel
 // Opt-in dynamic shared memory ceiling of the fused kernels (plans only pick them when the
 // layer needs less); leaves room for static shared memory under the 227 KB per-CTA limit.
-constexpr int kMaxDynSmem = 200 * 1024;
+constexpr int kMaxDynSmem = 214 * 1024;
+
+__host__ __device__ constexpr int pitch4(int J) {      // >= J, multiple of 4, == 4 (mod 32)
+  int p = (J + 3) / 4 * 4;
+  while (p % 32 != 4) p += 4;
+  return p;
+}
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -39,41 +57,309 @@ __device__ __forceinline__ float4 ld4<__nv_bfloat16>(const __nv_bfloat16* p) {
   return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
 }
 
-// Loads a [rows x R] factor (row-major, r <= R real columns) into shared memory, zero-padded.
-template <int R>
-__device__ __forceinline__ void load_factor(float* dst, const float* __restrict__ U, int rows, int r) {
-  for (int idx = threadIdx.x; idx < rows * R; idx += blockDim.x) {
-    const int k = idx / R, j = idx % R;
-    dst[idx] = (j < r) ? U[k * r + j] : 0.f;
+// ---- bulk-copy engine (TMA, untiled form) and mbarrier ------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+// dst and src 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
+  const uint64_t t0 = globaltimer_ns();
+  for (uint32_t it = 0; it < (1u << 28); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && globaltimer_ns() - t0 > limit_ns) return false;
+  }
+  return false;
+}
+// Thread 0 waits for the staged tile with a time limit; every thread learns the outcome.  On expiry
+// the status word gets ASI_ERR_TIMEOUT and thread 0 gives the copies in flight one more bounded
+// wait before the CTA returns.
+__device__ __forceinline__ bool cta_wait_tile(uint64_t* bar, int* s_flag, int* status) {
+  if (threadIdx.x == 0) {
+    bool ok = mbar_wait_bounded(bar, 0, 1000000000ull);
+    if (!ok) {
+      atomicMax(status, (int)ASI_ERR_TIMEOUT);
+      mbar_wait_bounded(bar, 0, 1000000000ull);
+    }
+    *s_flag = ok ? 1 : 0;
+  }
+  __syncthreads();
+  const bool ok = *s_flag != 0;
+  if (ok)
+    for (int it = 0; it < 64 && !mbar_try_wait(bar, 0); ++it) {
+    }
+  return ok;
+}
+
+// Warp 0 stages `rows` rows of `row_bytes` each: row i from src + i*src_stride_bytes to
+// dst + i*dst_stride_bytes.
+__device__ __forceinline__ void stage_rows(uint64_t* bar, char* dst, const char* src, int rows,
+                                           uint32_t row_bytes, int64_t src_stride_bytes,
+                                           uint32_t dst_stride_bytes) {
+  const int lane = threadIdx.x & 31;
+  if ((threadIdx.x >> 5) != 0) return;
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    mbar_expect_tx(bar, (uint32_t)rows * row_bytes);
+  }
+  __syncwarp();
+  for (int i = lane; i < rows; i += 32)
+    bulk_g2s(dst + (size_t)i * dst_stride_bytes, src + (int64_t)i * src_stride_bytes, row_bytes, bar);
+}
+// Warp 0 stages one contiguous block in chunks of 16 KB.
+__device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char* src, uint32_t bytes) {
+  constexpr uint32_t kChunk = 16384;
+  const int lane = threadIdx.x & 31;
+  if ((threadIdx.x >> 5) != 0) return;
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    mbar_expect_tx(bar, bytes);
+  }
+  __syncwarp();
+  const int nchunk = (int)((bytes + kChunk - 1) / kChunk);
+  for (int i = lane; i < nchunk; i += 32) {
+    const uint32_t off = (uint32_t)i * kChunk;
+    const uint32_t n = (bytes - off < kChunk) ? bytes - off : kChunk;
+    bulk_g2s(dst + off, src + off, n, bar);
   }
 }
 
-// Sum of `n` per-thread values over the CTA in a fixed order: warp shuffles, then warps in
-// index order.  red: [8][n] floats of shared memory.  Threads tid < n return the total.
-template <int N>
-__device__ __forceinline__ void block_reduce_store(float (&v)[N], float* red, float* out_global, int n_keep_cols,
-                                                   int R, int r) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+// Small read-only arrays a CTA keeps in shared memory (factors, the core).  All of them are fetched
+// in ONE batch: every thread first issues the loads of all its elements, then stores them, so the
+// prologue costs a single global-memory round trip.  Element (k, j) of array i, j < r_dst:
+// dst[k*r_dst + j] = j < r_src ? src[k*r_src + j] : 0.
+struct FacDesc {
+  const float* src;
+  float* dst;
+  int rows, r_src, r_dst;
+};
+template <int NF>
+__device__ __forceinline__ void load_factors(const FacDesc (&f)[NF]) {
+  constexpr int MAXI = 8;
+  int n[NF], total = 0;
 #pragma unroll
-  for (int i = 0; i < N; ++i) {
-    float x = v[i];
-    x += __shfl_xor_sync(0xffffffffu, x, 16);
-    x += __shfl_xor_sync(0xffffffffu, x, 8);
-    x += __shfl_xor_sync(0xffffffffu, x, 4);
-    x += __shfl_xor_sync(0xffffffffu, x, 2);
-    x += __shfl_xor_sync(0xffffffffu, x, 1);
-    if (lane == 0) red[warp * N + i] = x;
+  for (int i = 0; i < NF; ++i) {
+    n[i] = f[i].rows * f[i].r_dst;
+    total += n[i];
+  }
+  for (int base = 0; base < total; base += kNT * MAXI) {
+    float v[MAXI];
+    float* d[MAXI];
+#pragma unroll
+    for (int k = 0; k < MAXI; ++k) {
+      int idx = base + k * kNT + (int)threadIdx.x;
+      v[k] = 0.f;
+      d[k] = nullptr;
+      if (idx < total) {
+#pragma unroll
+        for (int i = 0; i < NF; ++i) {
+          if (d[k] == nullptr) {
+            if (idx < n[i]) {
+              const int row = idx / f[i].r_dst, j = idx - row * f[i].r_dst;
+              d[k] = f[i].dst + idx;
+              if (j < f[i].r_src) v[k] = __ldg(f[i].src + row * f[i].r_src + j);
+            } else {
+              idx -= n[i];
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < MAXI; ++k)
+      if (d[k] != nullptr) *d[k] = v[k];
+  }
+}
+
+template <int R>
+__device__ __forceinline__ void fma_row(float (&acc)[R], float x, const float* __restrict__ u) {
+#pragma unroll
+  for (int j = 0; j < R; j += 4) {
+    const float4 v = *reinterpret_cast<const float4*>(u + j);
+    acc[j] = fmaf(x, v.x, acc[j]);
+    acc[j + 1] = fmaf(x, v.y, acc[j + 1]);
+    acc[j + 2] = fmaf(x, v.z, acc[j + 2]);
+    acc[j + 3] = fmaf(x, v.w, acc[j + 3]);
+  }
+}
+
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Sum of N per-lane values over the 32 lanes of a warp by recursive halving: every step each lane
+// hands half of its values to its partner, so the whole reduction costs N-N/32 shuffles.  On return
+// v[i], i < N/32, is the total of element scatter_base<N>(lane) + i.  The order of additions is fixed.
+template <int N, int OFF>
+__device__ __forceinline__ void halving_step(float* v, int lane) {
+  constexpr int n = N / 2;
+  const bool up = (lane & OFF) != 0;
+#pragma unroll
+  for (int i = 0; i < n; ++i) {
+    const float send = up ? v[i] : v[i + n];
+    const float keep = up ? v[i + n] : v[i];
+    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);
+  }
+}
+template <int N>
+__device__ __forceinline__ void warp_reduce_scatter(float (&v)[N], int lane) {
+  static_assert(N % 32 == 0, "pad the accumulator count to a multiple of 32");
+  halving_step<N, 16>(v, lane);
+  halving_step<N / 2, 8>(v, lane);
+  halving_step<N / 4, 4>(v, lane);
+  halving_step<N / 8, 2>(v, lane);
+  halving_step<N / 16, 1>(v, lane);
+}
+template <int N>
+__device__ __forceinline__ int scatter_base(int lane) {
+  return ((lane >> 4) & 1) * (N / 2) + ((lane >> 3) & 1) * (N / 4) + ((lane >> 2) & 1) * (N / 8) +
+         ((lane >> 1) & 1) * (N / 16) + (lane & 1) * (N / 32);
+}
+
+// Number of interleaved sample groups project_batch uses for a tile of J columns on nthr threads.
+__host__ __device__ constexpr int batch_groups(int nthr, int J) {
+  const int items = (J % 2 == 0) ? J / 2 : J;
+  int nh = nthr / items;
+  return nh < 1 ? 1 : (nh > 4 ? 4 : nh);
+}
+
+// out[j][0..R) = sum_b Xs[b*PJ + j] * Us[b*R + ..] for j < J: the mode-1 contraction of a staged tile
+// [B x J].  Runs on `nthr` threads (t = 0..nthr-1) that synchronise on named barrier `bar`.  A thread
+// owns two neighbouring columns (one 8-byte shared load per sample) and the samples b == h (mod NH);
+// the NH partial sums meet in `part` ([NH][J][R]) in a fixed order.
+template <int R>
+__device__ __forceinline__ void project_batch(const float* __restrict__ Xs, int PJ,
+                                              const float* __restrict__ Us, int B, int J,
+                                              float* __restrict__ part, float* __restrict__ out, int t,
+                                              int nthr, int bar) {
+  const int NH = batch_groups(nthr, J);
+  if ((J & 1) == 0) {
+    const int J2 = J >> 1;
+    for (int it = t; it < NH * J2; it += nthr) {
+      const int h = it / J2, jp = it - h * J2;
+      float a0[R], a1[R];
+#pragma unroll
+      for (int q = 0; q < R; ++q) a0[q] = a1[q] = 0.f;
+#pragma unroll 8
+      for (int b = h; b < B; b += NH) {
+        const float2 x = *reinterpret_cast<const float2*>(Xs + b * PJ + 2 * jp);
+        fma_row<R>(a0, x.x, Us + b * R);
+        fma_row<R>(a1, x.y, Us + b * R);
+      }
+      float* dst = (NH > 1 ? part + h * J * R : out) + 2 * jp * R;
+#pragma unroll
+      for (int q = 0; q < R; q += 4) {
+        *reinterpret_cast<float4*>(dst + q) = make_float4(a0[q], a0[q + 1], a0[q + 2], a0[q + 3]);
+        *reinterpret_cast<float4*>(dst + R + q) = make_float4(a1[q], a1[q + 1], a1[q + 2], a1[q + 3]);
+      }
+    }
+  } else {
+    for (int it = t; it < NH * J; it += nthr) {
+      const int h = it / J, j = it - h * J;
+      float acc[R];
+#pragma unroll
+      for (int q = 0; q < R; ++q) acc[q] = 0.f;
+#pragma unroll 8
+      for (int b = h; b < B; b += NH) fma_row<R>(acc, Xs[b * PJ + j], Us + b * R);
+      float* dst = (NH > 1 ? part + h * J * R : out) + j * R;
+#pragma unroll
+      for (int q = 0; q < R; ++q) dst[q] = acc[q];
+    }
+  }
+  if (NH > 1) {
+    bar_sync(bar, nthr);
+    for (int idx = t; idx < J * R; idx += nthr) {
+      float s = 0.f;
+      for (int h = 0; h < NH; ++h) s += part[h * J * R + idx];
+      out[idx] = s;
+    }
+  }
+  bar_sync(bar, nthr);
+}
+
+// V[hw][:] = sum_c Xs[c*PC + hw] * Us[c][:] for a staged block Xs [C][HWC] of one sample (the mode-2
+// projection of HWC positions).  Thread (g, hw) sums the channels c = g (mod G); group 0 writes V
+// itself, groups 1..G-1 write Vp ([G-1][HWC][R]; may alias Us: it is written only after every thread
+// has finished reading Us) and the sums meet in a fixed order.  All kNT threads call it.
+template <int HWC, int PC, int R>
+__device__ __forceinline__ void project_channels(const float* __restrict__ Xs, const float* Us, float* Vp,
+                                                 float* V, int C) {
+  constexpr int G = kNT / HWC;
+  const int tid = threadIdx.x;
+  float acc[R];
+#pragma unroll
+  for (int j = 0; j < R; ++j) acc[j] = 0.f;
+  const int g = tid / HWC, hw = tid - g * HWC;
+  if (g < G) {
+#pragma unroll 4
+    for (int c = g; c < C; c += G) fma_row<R>(acc, Xs[c * PC + hw], Us + c * R);
+  }
+  if (G > 1) __syncthreads();
+  if (g < G) {
+    float* dst = (g == 0 ? V : Vp + (g - 1) * HWC * R) + hw * R;
+#pragma unroll
+    for (int j = 0; j < R; j += 4)
+      *reinterpret_cast<float4*>(dst + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
   }
   __syncthreads();
-  const int nwarps = blockDim.x >> 5;
-  for (int i = threadIdx.x; i < N; i += blockDim.x) {
-    float s = 0.f;
-    for (int w = 0; w < nwarps; ++w) s += red[w * N + i];
-    const int k = i / R, j = i % R;      // value i is entry (k, j) of an [n_keep_cols.. x R] block
-    if (j < r) out_global[k * r + j] = s;
+  if (G > 1) {
+    for (int idx = tid; idx < HWC * R; idx += kNT) {
+      float s = V[idx];
+#pragma unroll
+      for (int gg = 0; gg < G - 1; ++gg) s += Vp[gg * HWC * R + idx];
+      V[idx] = s;
+    }
+    __syncthreads();
   }
-  __syncthreads();
-  (void)n_keep_cols;
+}
+
+// Stages one tile [B x J] (row b at src + b*sample_stride) as fp32 rows of pitch PJ.
+template <typename TX>
+__device__ __forceinline__ void stage_tile_begin(const TX* __restrict__ src, int64_t sample_stride, float* Xs,
+                                                 int B, int J, int PJ, uint64_t* bar) {
+  if constexpr (std::is_same<TX, float>::value) {
+    stage_rows(bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(src), B, (uint32_t)J * 4u,
+               sample_stride * 4, (uint32_t)PJ * 4u);
+  } else {
+    const int J4 = J / 4;
+    for (int idx = threadIdx.x; idx < B * J4; idx += kNT) {
+      const int b = idx / J4, v = idx - b * J4;
+      *reinterpret_cast<float4*>(Xs + b * PJ + 4 * v) = ld4<TX>(src + b * sample_stride + 4 * v);
+    }
+  }
+}
+
+__host__ __device__ constexpr int tri_index(int S, int k, int k2) {   // k <= k2 < S, row-major upper triangle
+  return k * S - k * (k - 1) / 2 + (k2 - k);
 }
 
 }  // namespace
@@ -82,177 +368,213 @@ __device__ __forceinline__ void block_reduce_store(float (&v)[N], float* red, fl
 // k_sm_pass1
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
-__global__ void __launch_bounds__(256) k_sm_pass1(SmPass1Args p) {
+__global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
+  constexpr bool kBulk = std::is_same<TX, float>::value;
+  constexpr bool kGram = (S == 7);                   // modes 3, 4 as Gram matrices A_m A_m^T (7 x 7)
   constexpr int HW = S * S;
   constexpr int CC = (S == 7) ? 4 : 1;               // channels per role-B tile
   constexpr int J = CC * HW;                         // contiguous elements per sample in a tile
-  constexpr int PJ = (J % 32 == 4) ? J : J + 4;      // row pitch == 4 (mod 32): conflict-free b x j reads
-  extern __shared__ __align__(16) float smem[];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int PJ = pitch4(J);                      // row pitch == 4 (mod 32): conflict-free (b, j) reads
+  constexpr int NH1 = batch_groups(kNG, J);
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_flag;
+  const int tid = threadIdx.x, lane = tid & 31;
   const TX* __restrict__ A = reinterpret_cast<const TX*>(p.act);
   const int B = p.B, C = p.C;
 
-  if ((int)blockIdx.x < p.n_tiles_b) {
+  if (blockIdx.x == 0 && tid < 9) p.status[tid == 0 ? 0 : 15 + tid] = 0;   // status word, counters 16..23
+
+  constexpr int kNQ = (S == 7) ? 1 : 4;             // role-C CTAs per sample
+  if ((int)blockIdx.x >= B * kNQ) {
     // ---------------- role B: modes 1, 3, 4 on tile [B x J] ----------------
-    const int tile = blockIdx.x;
+    const int tile = blockIdx.x - B * kNQ;
     float* Xs = smem;                                // [B][PJ]
     float* U1s = Xs + B * PJ;                        // [B][R]
     float* U3s = U1s + B * R;                        // [S][R]
     float* U4s = U3s + S * R;                        // [S][R]
-    float* Vs = U4s + S * R;                         // [J][R]
-    float* red = Vs + J * R;                         // [8][S*R]
-    const int64_t sample_stride = (int64_t)C * HW;
-    const TX* src = A + (int64_t)tile * J;
-    for (int idx = tid; idx < B * (J / 4); idx += 256) {
-      const int b = idx / (J / 4), v = idx % (J / 4);
-      const float4 x = ld4<TX>(src + b * sample_stride + 4 * v);
-      *reinterpret_cast<float4*>(Xs + b * PJ + 4 * v) = x;
-    }
-    load_factor<R>(U1s, p.U_prev + p.u_off[0], B, p.r[0]);
-    load_factor<R>(U3s, p.U_prev + p.u_off[2], S, p.r[2]);
-    load_factor<R>(U4s, p.U_prev + p.u_off[3], S, p.r[3]);
-    __syncthreads();
-
-    // mode 1, projection: V[j,:] = sum_b X[b,j] U1[b,:]
-    if (tid < J) {
-      float acc[R];
-#pragma unroll
-      for (int j = 0; j < R; ++j) acc[j] = 0.f;
-      for (int b = 0; b < B; ++b) {
-        const float x = Xs[b * PJ + tid];
-#pragma unroll
-        for (int j = 0; j < R; j += 4) {
-          const float4 u = *reinterpret_cast<const float4*>(U1s + b * R + j);
-          acc[j] = fmaf(x, u.x, acc[j]);
-          acc[j + 1] = fmaf(x, u.y, acc[j + 1]);
-          acc[j + 2] = fmaf(x, u.z, acc[j + 2]);
-          acc[j + 3] = fmaf(x, u.w, acc[j + 3]);
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < R; ++j) Vs[tid * R + j] = acc[j];
-    }
-    __syncthreads();
-    // mode 1, expansion: P1[b,:] = sum_j X[b,j] V[j,:]; a warp covers 8 samples x 4 column phases
+    float* V1s = U4s + S * R;                        // [J][R]
+    float* part = V1s + J * R;                       // [NH1][J][R] (NH1 > 1 only)
+    float* red = part + (NH1 > 1 ? NH1 : 0) * J * R; // [8][32]
+    stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
     {
+      const FacDesc fd[3] = {{p.U_prev + p.u_off[0], U1s, B, p.r[0], R},
+                             {p.U_prev + p.u_off[2], U3s, S, p.r[2], R},
+                             {p.U_prev + p.u_off[3], U4s, S, p.r[3], R}};
+      load_factors<3>(fd);
+    }
+    if constexpr (kBulk) {
+      if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
+    } else {
+      __syncthreads();
+    }
+    const int t = tid & (kNG - 1), wg = t >> 5;
+    if (tid < kNG) {
+      // ---- half 0: mode 1.  V[j,:] = sum_b X[b,j] U1[b,:], then P1[b,:] = sum_j X[b,j] V[j,:]
+      project_batch<R>(Xs, PJ, U1s, B, J, part, V1s, t, kNG, 1);
       float* P1 = p.Pp[0] + (int64_t)tile * B * p.r[0];
-      const int bl = lane >> 2, jl = lane & 3;
-      for (int b0 = warp * 8; b0 < B; b0 += 64) {
+      const int bl = lane >> 2, jl = lane & 3;       // a warp covers 8 samples x 4 column phases
+      for (int b0 = wg * 8; b0 < B; b0 += 64) {
         const int b = b0 + bl;
         float acc[R];
 #pragma unroll
-        for (int j = 0; j < R; ++j) acc[j] = 0.f;
-        for (int jj = jl; jj < J; jj += 4) {
-          const float x = Xs[b * PJ + jj];
+        for (int q = 0; q < R; ++q) acc[q] = 0.f;
+#pragma unroll 7
+        for (int jj = jl; jj < J; jj += 4) fma_row<R>(acc, Xs[b * PJ + jj], V1s + jj * R);
 #pragma unroll
-          for (int j = 0; j < R; j += 4) {
-            const float4 v = *reinterpret_cast<const float4*>(Vs + jj * R + j);
-            acc[j] = fmaf(x, v.x, acc[j]);
-            acc[j + 1] = fmaf(x, v.y, acc[j + 1]);
-            acc[j + 2] = fmaf(x, v.z, acc[j + 2]);
-            acc[j + 3] = fmaf(x, v.w, acc[j + 3]);
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < R; ++j) {
-          acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 1);
-          acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 2);
+        for (int q = 0; q < R; ++q) {
+          acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], 1);
+          acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], 2);
         }
         if (jl == 0) {
 #pragma unroll
-          for (int j = 0; j < R; ++j)
-            if (j < p.r[0]) P1[b * p.r[0] + j] = acc[j];
+          for (int q = 0; q < R; ++q)
+            if (q < p.r[0]) P1[b * p.r[0] + q] = acc[q];
         }
       }
-    }
-    // modes 3 and 4: one column (fiber of S elements) per thread at a time
+    } else if constexpr (kGram) {
+      // ---- half 1, S = 7: G_m = A_m A_m^T for m = 3, 4, one plane (b, c) per thread at a time; the
+      // 32 lanes of a warp touch 32 different banks.  P_m = G_m U_m^prev follows in k_sm_reduce.
+      constexpr int NACC = 32;
+      static_assert(S * (S + 1) / 2 <= NACC, "upper triangle of the Gram matrix");
+      const int nplanes = B * CC;
 #pragma unroll 1
-    for (int mode = 2; mode <= 3; ++mode) {
-      const float* Us = (mode == 2) ? U3s : U4s;
-      const int estride = (mode == 2) ? S : 1;       // step between fiber elements
-      float acc[S * R];
+      for (int mode = 2; mode <= 3; ++mode) {
+        const int es = (mode == 2) ? S : 1;          // step between the elements of a fiber
+        const int cs = (mode == 2) ? 1 : S;          // step between neighbouring fibers
+        float* Gm = p.Pp[mode] + (int64_t)tile * HW;
+        float acc[NACC];
 #pragma unroll
-      for (int i = 0; i < S * R; ++i) acc[i] = 0.f;
-      const int ncols = B * CC * S;
-      for (int q = tid; q < ncols; q += 256) {
-        const int b = q / (CC * S), rem = q % (CC * S);
-        const int cl = rem / S, o = rem % S;         // o = w for mode 3, h for mode 4
-        const float* col = Xs + b * PJ + cl * HW + ((mode == 2) ? o : o * S);
-        float x[S], v[R];
+        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
+        for (int pl = t; pl < nplanes; pl += kNG) {
+          const int b = pl / CC, cl = pl % CC;
+          const float* base = Xs + b * PJ + cl * HW;
+#pragma unroll 1
+          for (int col = 0; col < S; ++col) {
+            const float* colp = base + col * cs;
+            float x[S];
 #pragma unroll
-        for (int j = 0; j < R; ++j) v[j] = 0.f;
+            for (int k = 0; k < S; ++k) x[k] = colp[k * es];
 #pragma unroll
-        for (int k = 0; k < S; ++k) {
-          x[k] = col[k * estride];
+            for (int k = 0; k < S; ++k)
 #pragma unroll
-          for (int j = 0; j < R; ++j) v[j] = fmaf(x[k], Us[k * R + j], v[j]);
+              for (int k2 = k; k2 < S; ++k2) acc[tri_index(S, k, k2)] = fmaf(x[k], x[k2], acc[tri_index(S, k, k2)]);
+          }
         }
+        warp_reduce_scatter<NACC>(acc, lane);
+        red[wg * 32 + scatter_base<NACC>(lane)] = acc[0];
+        bar_sync(2, kNG);
+        for (int o = t; o < HW; o += kNG) {
+          const int k = o / S, k2 = o % S;
+          const int e = (k <= k2) ? tri_index(S, k, k2) : tri_index(S, k2, k);
+          float s = 0.f;
 #pragma unroll
-        for (int k = 0; k < S; ++k)
-#pragma unroll
-          for (int j = 0; j < R; ++j) acc[k * R + j] = fmaf(x[k], v[j], acc[k * R + j]);
+          for (int w = 0; w < 8; ++w) s += red[w * 32 + e];
+          Gm[o] = s;
+        }
+        bar_sync(2, kNG);
       }
-      block_reduce_store<S * R>(acc, red, p.Pp[mode] + (int64_t)tile * S * p.r[mode], S, R, p.r[mode]);
+    } else {
+      // ---- half 1, S > 7: P_m = A_m (A_m^T U_m^prev) for m = 3, 4.  A unit is a quarter of a plane
+      // (columns == part mod 4); unit -> thread so that the 32 lanes of a warp touch 32 different
+      // banks.  Each thread owns 2 columns of the factor; warp w serves column pair w mod JH.
+      constexpr int TPP = 4, JT = 2, JH = R / JT, NACC = 32;
+      static_assert(S * JT <= NACC, "accumulators of one thread");
+      const int jh = wg % JH;
+      const int u0 = (wg / JH) * 32 + lane;
+      const int nunits = B * CC * TPP;
+#pragma unroll 1
+      for (int mode = 2; mode <= 3; ++mode) {
+        const float* Us = ((mode == 2) ? U3s : U4s) + jh * JT;
+        const int es = (mode == 2) ? S : 1;
+        const int cs = (mode == 2) ? 1 : S;
+        const int rm = p.r[mode];
+        float* Pm = p.Pp[mode] + (int64_t)tile * S * rm;
+        float acc[NACC];
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
+        for (int un = u0; un < nunits; un += kNG / JH) {
+          const int pl = un / TPP, part_ = un % TPP;
+          const int b = pl / CC, cl = pl % CC;
+          const float* base = Xs + b * PJ + cl * HW;
+#pragma unroll 1
+          for (int col = part_; col < S; col += TPP) {
+            const float* colp = base + col * cs;
+            float x[S], v0 = 0.f, v1 = 0.f;
+#pragma unroll
+            for (int k = 0; k < S; ++k) {
+              x[k] = colp[k * es];
+              const float2 u = *reinterpret_cast<const float2*>(Us + k * R);
+              v0 = fmaf(x[k], u.x, v0);
+              v1 = fmaf(x[k], u.y, v1);
+            }
+#pragma unroll
+            for (int k = 0; k < S; ++k) {
+              acc[2 * k] = fmaf(x[k], v0, acc[2 * k]);
+              acc[2 * k + 1] = fmaf(x[k], v1, acc[2 * k + 1]);
+            }
+          }
+        }
+        warp_reduce_scatter<NACC>(acc, lane);
+        red[wg * 32 + scatter_base<NACC>(lane)] = acc[0];
+        bar_sync(2, kNG);
+        for (int o = t; o < S * R; o += kNG) {
+          const int k = o / R, j = o % R;
+          const int e = k * JT + (j % JT);
+          float s = 0.f;
+          for (int w = j / JT; w < 8; w += JH) s += red[w * 32 + e];
+          if (j < rm) Pm[k * rm + j] = s;
+        }
+        bar_sync(2, kNG);
+      }
     }
   } else {
-    // ---------------- role C: mode 2 on one sample [C x HW] ----------------
-    constexpr int G = 256 / HW;                      // channel rows covered per sweep of the CTA
-    constexpr int NACT = G * HW;                     // active threads in the projection
-    const int b = blockIdx.x - p.n_tiles_b;
-    float* U2s = smem;                               // [C][R]
-    float* Vp = U2s + C * R;                         // [G][HW][R]
-    float* V2s = Vp + G * HW * R;                    // [HW][R]
-    load_factor<R>(U2s, p.U_prev + p.u_off[1], C, p.r[1]);
-    __syncthreads();
-    const TX* Xb = A + (int64_t)b * C * HW;
-    if (tid < NACT) {
-      // thread owns position hw = tid % HW and the channels c = tid / HW (mod G)
-      float acc[R];
-#pragma unroll
-      for (int j = 0; j < R; ++j) acc[j] = 0.f;
-      int c = tid / HW;
-#pragma unroll 4
-      for (int e = tid; e < C * HW; e += NACT, c += G) {
-        const float x = to_f(Xb[e]);
-#pragma unroll
-        for (int j = 0; j < R; j += 4) {
-          const float4 u = *reinterpret_cast<const float4*>(U2s + c * R + j);
-          acc[j] = fmaf(x, u.x, acc[j]);
-          acc[j + 1] = fmaf(x, u.y, acc[j + 1]);
-          acc[j + 2] = fmaf(x, u.z, acc[j + 2]);
-          acc[j + 3] = fmaf(x, u.w, acc[j + 3]);
-        }
+    // ---------------- role C: mode 2 on block [C x HWC] of one sample ----------------
+    // S = 7: the whole sample (contiguous, staged by the bulk-copy engine); larger maps: one quarter
+    // of the positions, rows gathered with plain loads (they are only 4-byte aligned).
+    constexpr int NQ = (S == 7) ? 1 : 4;
+    constexpr int HWC = HW / NQ;
+    constexpr int PC = (HWC % 2 == 0) ? HWC + 1 : HWC;     // odd pitch: conflict-free row-per-thread reads
+    constexpr int G = kNT / HWC;
+    constexpr bool kBulkC = kBulk && NQ == 1;
+    const int b = blockIdx.x / NQ, q = blockIdx.x % NQ;
+    float* Xs = smem;                                // [C][PC]
+    float* U2s = Xs + ((C * PC + 3) & ~3);           // [C][R]
+    float* V2s = U2s + C * R;                        // [HWC][R]
+    float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
+    const TX* Xb = A + (int64_t)b * C * HW + q * HWC;
+    if constexpr (kBulkC) {
+      stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
+    } else if constexpr (NQ == 1) {
+      const int n4 = C * HW / 4;
+      for (int idx = tid; idx < n4; idx += kNT) *reinterpret_cast<float4*>(Xs + 4 * idx) = ld4<TX>(Xb + 4 * idx);
+    } else {
+      const int n = C * HWC;
+#pragma unroll 8
+      for (int idx = tid; idx < n; idx += kNT) {
+        const int c = idx / HWC, hw = idx - c * HWC;
+        Xs[c * PC + hw] = to_f(Xb[(int64_t)c * HW + hw]);
       }
-#pragma unroll
-      for (int j = 0; j < R; ++j) Vp[tid * R + j] = acc[j];
     }
-    __syncthreads();
-    for (int idx = tid; idx < HW * R; idx += 256) {
-      float s = 0.f;
-#pragma unroll
-      for (int g = 0; g < G; ++g) s += Vp[g * HW * R + idx];
-      V2s[idx] = s;
+    {
+      const FacDesc fd[1] = {{p.U_prev + p.u_off[1], U2s, C, p.r[1], R}};
+      load_factors<1>(fd);
     }
-    __syncthreads();
+    if constexpr (kBulkC) {
+      if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
+    } else {
+      __syncthreads();
+    }
+    project_channels<HWC, PC, R>(Xs, U2s, Vp, V2s, C);
     // expansion: P2[c,:] = sum_hw X[c,hw] V2[hw,:], one channel row per thread
-    float* P2 = p.Pp[1] + (int64_t)b * C * p.r[1];
-    for (int c = tid; c < C; c += 256) {
-      const TX* row = Xb + (int64_t)c * HW;
+    float* P2 = p.Pp[1] + (int64_t)blockIdx.x * C * p.r[1];
+    for (int c = tid; c < C; c += kNT) {
+      const float* row = Xs + c * PC;
       float acc[R];
 #pragma unroll
       for (int j = 0; j < R; ++j) acc[j] = 0.f;
 #pragma unroll 7
-      for (int hw = 0; hw < HW; ++hw) {
-        const float x = to_f(row[hw]);
-#pragma unroll
-        for (int j = 0; j < R; j += 4) {
-          const float4 v = *reinterpret_cast<const float4*>(V2s + hw * R + j);
-          acc[j] = fmaf(x, v.x, acc[j]);
-          acc[j + 1] = fmaf(x, v.y, acc[j + 1]);
-          acc[j + 2] = fmaf(x, v.z, acc[j + 2]);
-          acc[j + 3] = fmaf(x, v.w, acc[j + 3]);
-        }
-      }
+      for (int hw = 0; hw < HWC; ++hw) fma_row<R>(acc, row[hw], V2s + hw * R);
 #pragma unroll
       for (int j = 0; j < R; ++j)
         if (j < p.r[1]) P2[c * p.r[1] + j] = acc[j];
@@ -261,75 +583,241 @@ __global__ void __launch_bounds__(256) k_sm_pass1(SmPass1Args p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_sm_core: CTA b computes T[b] = A[b] x_2 U2^T x_3 U3^T x_4 U4^T ([r2,r3,r4]); the last CTA to
-// finish sums core[i,:] = sum_b U1[b,i] T[b,:] in sample order.
+// k_sm_reduce: CTA (c, m) sums rows [16 c, 16 c + 16) of the per-tile partials of P_m in fp64 in a
+// fixed order (thread (e, sg) takes the partials s == sg (mod SG); the SG sums meet in shared memory
+// in index order), stores them in fp64 and adds its share of G_m = P_m^T P_m.  A mode whose
+// partials are Gram matrices A_m A_m^T (a <= 16, one CTA) is summed the same way and multiplied by
+// U_m^prev first.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
+  constexpr int RM = 8, RPC = kRedRows;
+  const SmReduceMode M = args.m[blockIdx.y];
+  const int c = blockIdx.x;
+  if (c >= M.nchunk) return;
+  __shared__ double part[kRedNT];
+  __shared__ double Ps[RPC][RM];
+  __shared__ double Gm[RPC * RPC];
+  const int tid = threadIdx.x;
+  const int r = M.r, a = M.a;
+  const int row0 = c * RPC;
+  const int nrow = (a - row0 < RPC) ? (a - row0) : RPC;
+  const int E = M.gram ? a * a : nrow * r;         // <= 256
+  int EP = 32;
+  while (EP < E) EP <<= 1;
+  const int SG = kRedNT / EP;
+  float u_prev = 0.f;
+  if (M.gram && tid < a * r) u_prev = __ldg(M.Uprev + tid);
+  {
+    const int e = tid & (EP - 1), sg = tid / EP;
+    double acc = 0.0;
+    if (e < E) {
+      const float* ptr = M.Pp + (M.gram ? 0 : (int64_t)row0 * r) + e;
+      const int64_t stride = M.gram ? (int64_t)a * a : (int64_t)a * r;
+#pragma unroll 16
+      for (int s = sg; s < M.nsplit; s += SG) acc += (double)__ldcg(ptr + s * stride);
+    }
+    part[tid] = acc;
+  }
+  for (int idx = tid; idx < RPC * RM; idx += kRedNT) Ps[idx / RM][idx % RM] = 0.0;
+  __syncthreads();
+  if (M.gram) {
+    __shared__ float Us[RPC * RM];
+    if (tid < E) {
+      double v = 0.0;
+      for (int sg = 0; sg < SG; ++sg) v += part[sg * EP + tid];
+      Gm[tid] = v;
+    }
+    if (tid < a * r) Us[tid] = u_prev;
+    __syncthreads();
+    if (tid < a * r) {
+      const int k = tid / r, j = tid % r;
+      double v = 0.0;
+      for (int k2 = 0; k2 < a; ++k2) v = fma(Gm[k * a + k2], (double)Us[k2 * r + j], v);
+      M.Pred[tid] = v;
+      Ps[k][j] = v;
+    }
+  } else if (tid < E) {
+    double v = 0.0;
+    for (int sg = 0; sg < SG; ++sg) v += part[sg * EP + tid];
+    M.Pred[(int64_t)row0 * r + tid] = v;
+    Ps[tid / r][tid % r] = v;
+  }
+  __syncthreads();
+  if (tid < r * r) {
+    const int i = tid / r, j = tid % r;
+    double g = 0.0;
+    if (j >= i) {
+#pragma unroll
+      for (int rl = 0; rl < RPC; ++rl) g = fma(Ps[rl][i], Ps[rl][j], g);
+    }
+    M.Gp[((int64_t)c * r + i) * r + j] = g;
+  }
+}
+
+cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st) {
+  double bytes = 0.0;
+  for (int m = 0; m < nd; ++m)
+    bytes += 4.0 * p.m[m].nsplit * p.m[m].a * (p.m[m].gram ? p.m[m].a : p.m[m].r) + 8.0 * p.m[m].a * p.m[m].r;
+  ProfScope prof(ASI_K_QR, st, bytes);
+  dim3 grid((unsigned)max_chunks, (unsigned)nd);
+  k_sm_reduce<<<grid, kRedNT, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// k_sm_core.  Tile t = [all B x J] as in role B of the first pass.
+//   prologue (while the tile is in flight): each thread fetches the fp64 row of P_m it will solve
+//     for; warps 4m..4m+3 sum the Gram shares of mode m and warp 4m factors G_m = R_m^T R_m; then
+//     one thread per needed factor row solves u = p R_m^{-1} -- all of U_1, the tile's own rows of
+//     U_2, all of U_3 and U_4 -- and the owners write them to U_new;
+//   W[i][c,h,w] = sum_b U1[b,i] X[b][c,h,w];  Y[i,j][h,w] = sum_c U2[c,j] W[i][c,h,w];
+//   T[i,j,k,l] = Y x_3 U3^T x_4 U4^T  -> per-tile partial core; the last CTA sums the tiles in order.
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
-__global__ void __launch_bounds__(256) k_sm_core(SmCoreArgs p) {
+__global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
+  constexpr bool kBulk = std::is_same<TX, float>::value;
   constexpr int HW = S * S;
-  constexpr int G = 256 / HW;
-  constexpr int NACT = G * HW;
-  extern __shared__ __align__(16) float smem[];
-  const int tid = threadIdx.x;
-  const int b = blockIdx.x, C = p.C;
-  const int r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
-  float* U2s = smem;                    // [C][R]
-  float* Vp = U2s + C * R;              // [G][HW][R]
-  float* T2 = Vp + G * HW * R;          // [HW][R]      T2[(h,w)][j]
-  float* U3s = T2 + HW * R;             // [S][R]
-  float* U4s = U3s + S * R;             // [S][R]
-  float* T3 = U4s + S * R;              // [R][R][S]    T3[j][k][w]
+  constexpr int CC = (S == 7) ? 4 : 1;
+  constexpr int J = CC * HW;
+  constexpr int PJ = pitch4(J);
+  constexpr int NH = batch_groups(kNT, J);
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_flag;
   __shared__ int s_last;
-  load_factor<R>(U2s, p.U + p.u_off[1], C, r2);
-  load_factor<R>(U3s, p.U + p.u_off[2], S, r3);
-  load_factor<R>(U4s, p.U + p.u_off[3], S, r4);
-  __syncthreads();
-  const TX* Xb = reinterpret_cast<const TX*>(p.act) + (int64_t)b * C * HW;
-  if (tid < NACT) {
-    float acc[R];
+  __shared__ double Gq[4][4][R * R];
+  __shared__ double Gs[4][R][R + 1];
+  __shared__ double Dinv[4][R];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int B = p.B, C = p.C, tile = blockIdx.x;
+  const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
+  float* Xs = smem;                     // [B][PJ]
+  float* U1s = Xs + B * PJ;             // [B][R]
+  float* U2s = U1s + B * R;             // [CC][R]
+  float* U3s = U2s + CC * R;            // [S][R]
+  float* U4s = U3s + S * R;             // [S][R]
+  float* Ws = U4s + S * R;              // [J][R]
+  float* part = Ws + J * R;             // [NH][J][R]
+  float* Ysm = part + NH * J * R;       // [R R][HW]
+  float* T3s = Ysm + R * R * HW;        // [R R][R][S]
+  stage_tile_begin<TX>(reinterpret_cast<const TX*>(p.act) + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ,
+                       &s_bar);
+  // ---- the factor row this thread will solve for: [U1: B rows][U2: CC rows][U3: S][U4: S]
+  const int nrows = B + CC + 2 * S;     // <= kNT (checked when the plan picks this kernel)
+  int rm = 0, rk = 0, rr = 0;
+  float* rdst = nullptr;
+  bool rowner = false;
+  double prow[R];
 #pragma unroll
-    for (int j = 0; j < R; ++j) acc[j] = 0.f;
-    int c = tid / HW;
-#pragma unroll 4
-    for (int e = tid; e < C * HW; e += NACT, c += G) {
-      const float x = to_f(Xb[e]);
+  for (int j = 0; j < R; ++j) prow[j] = 0.0;
+  if (tid < nrows) {
+    if (tid < B) { rm = 0; rk = tid; rdst = U1s + rk * R; rowner = tile == 0; }
+    else if (tid < B + CC) { rm = 1; rk = tile * CC + (tid - B); rdst = U2s + (tid - B) * R; rowner = true; }
+    else if (tid < B + CC + S) { rm = 2; rk = tid - B - CC; rdst = U3s + rk * R; rowner = tile == 0; }
+    else { rm = 3; rk = tid - B - CC - S; rdst = U4s + rk * R; rowner = tile == 0; }
+    rr = p.r[rm];
+    const double* src = p.Pred[rm] + (int64_t)rk * rr;
 #pragma unroll
-      for (int j = 0; j < R; j += 4) {
-        const float4 u = *reinterpret_cast<const float4*>(U2s + c * R + j);
-        acc[j] = fmaf(x, u.x, acc[j]);
-        acc[j + 1] = fmaf(x, u.y, acc[j + 1]);
-        acc[j + 2] = fmaf(x, u.z, acc[j + 2]);
-        acc[j + 3] = fmaf(x, u.w, acc[j + 3]);
-      }
+    for (int j = 0; j < R; ++j)
+      if (j < rr) prow[j] = __ldcg(src + j);
+  }
+  // ---- Gram shares: warp 4m + q sums the chunks == q (mod 4) of mode m
+  {
+    const int m = warp >> 2, q = warp & 3, r = p.r[m];
+    const double* Gp = p.Gp[m];
+    const int nch = p.nchunk[m];
+    for (int e = lane; e < r * r; e += 32) {
+      double g = 0.0;
+#pragma unroll 8
+      for (int cc = q; cc < nch; cc += 4) g += __ldcg(Gp + (int64_t)cc * r * r + e);
+      Gq[m][q][e] = g;
     }
-#pragma unroll
-    for (int j = 0; j < R; ++j) Vp[tid * R + j] = acc[j];
   }
   __syncthreads();
-  for (int idx = tid; idx < HW * R; idx += 256) {
-    float s = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) s += Vp[g * HW * R + idx];
-    T2[idx] = s;
+  if ((warp & 3) == 0) {
+    const int m = warp >> 2, r = p.r[m];
+    for (int e = lane; e < r * r; e += 32)
+      Gs[m][e / r][e % r] = ((Gq[m][0][e] + Gq[m][1][e]) + Gq[m][2][e]) + Gq[m][3][e];
+    __syncwarp();
+    double trace = 0.0;
+    for (int i = 0; i < r; ++i) trace += Gs[m][i][i];
+    const double floor_d = 1e-12 * trace;
+    for (int j = 0; j < r; ++j) {
+      if (lane == 0) {
+        double d = Gs[m][j][j];
+        if (!(d > floor_d)) {
+          if (blockIdx.x == 0) atomicMax(p.status, (int)ASI_ERR_RANK_DEFICIENT);
+          d = (floor_d > 0.0) ? floor_d : 1.0;
+        }
+        const double rjj = sqrt(d);
+        Gs[m][j][j] = rjj;
+        Dinv[m][j] = 1.0 / rjj;
+      }
+      __syncwarp();
+      const double inv = Dinv[m][j];
+      if (lane > j && lane < r) Gs[m][j][lane] *= inv;
+      __syncwarp();
+      for (int e = lane; e < r * r; e += 32) {
+        const int i = e / r, k = e % r;
+        if (i > j && k >= i) Gs[m][i][k] -= Gs[m][j][i] * Gs[m][j][k];
+      }
+      __syncwarp();
+    }
   }
   __syncthreads();
-  // T3[j][k][w] = sum_h T2[(h,w)][j] U3[h][k]
-  for (int idx = tid; idx < r2 * r3 * S; idx += 256) {
-    const int w = idx % S, k = (idx / S) % r3, j = idx / (S * r3);
+  if (tid < nrows) {
+    float* gdst = p.U_new + p.u_off[rm] + (int64_t)rk * rr;
+    double q[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+      float out = 0.f;
+      if (j < rr) {
+        double v = prow[j];
+#pragma unroll
+        for (int i = 0; i < R; ++i)
+          if (i < j) v -= q[i] * Gs[rm][i][j];
+        v *= Dinv[rm][j];
+        q[j] = v;
+        out = (float)v;
+        if (rowner) gdst[j] = out;
+      }
+      rdst[j] = out;
+    }
+  }
+  if constexpr (kBulk) {
+    if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
+  } else {
+    __syncthreads();
+  }
+  project_batch<R>(Xs, PJ, U1s, B, J, part, Ws, tid, kNT, 0);
+  // Y[(i,j)][hw] = sum_cl U2[cl][j] W[cl*HW + hw][i]
+  const int r12 = r1 * r2;
+  for (int idx = tid; idx < r12 * HW; idx += kNT) {
+    const int hw = idx % HW, ij = idx / HW;
+    const int i = ij / r2, j = ij - i * r2;
     float s = 0.f;
 #pragma unroll
-    for (int h = 0; h < S; ++h) s = fmaf(T2[(h * S + w) * R + j], U3s[h * R + k], s);
-    T3[(j * R + k) * S + w] = s;
+    for (int cl = 0; cl < CC; ++cl) s = fmaf(U2s[cl * R + j], Ws[(cl * HW + hw) * R + i], s);
+    Ysm[ij * HW + hw] = s;
   }
   __syncthreads();
-  // T[b][j][k][l] = sum_w T3[j][k][w] U4[w][l]
-  const int n234 = r2 * r3 * r4;
-  for (int idx = tid; idx < n234; idx += 256) {
-    const int l = idx % r4, k = (idx / r4) % r3, j = idx / (r4 * r3);
+  // T3[(i,j)][k][w] = sum_h Y[(i,j)][h,w] U3[h][k]
+  for (int idx = tid; idx < r12 * r3 * S; idx += kNT) {
+    const int w = idx % S, k = (idx / S) % r3, ij = idx / (S * r3);
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < S; ++w) s = fmaf(T3[(j * R + k) * S + w], U4s[w * R + l], s);
-    p.Tb[(int64_t)b * n234 + idx] = s;
+    for (int h = 0; h < S; ++h) s = fmaf(Ysm[ij * HW + h * S + w], U3s[h * R + k], s);
+    T3s[(ij * R + k) * S + w] = s;
+  }
+  __syncthreads();
+  // T[(i,j)][k][l] = sum_w T3[(i,j)][k][w] U4[w][l]
+  const int ce = r12 * r3 * r4;
+  for (int idx = tid; idx < ce; idx += kNT) {
+    const int l = idx % r4, k = (idx / r4) % r3, ij = idx / (r4 * r3);
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < S; ++w) s = fmaf(T3s[(ij * R + k) * S + w], U4s[w * R + l], s);
+    p.Tp[(int64_t)tile * ce + idx] = s;
   }
   __threadfence();
   __syncthreads();
@@ -337,198 +825,247 @@ __global__ void __launch_bounds__(256) k_sm_core(SmCoreArgs p) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const float* U1 = p.U + p.u_off[0];
-  const int r1 = p.r[0];
-  for (int idx = tid; idx < r1 * n234; idx += 256) {
-    const int i = idx / n234, rest = idx % n234;
+  // the last CTA sums the tiles in index order: thread (idx, h) takes the tiles == h (mod nh)
+  const int nh = (ce <= kNT / 4) ? 4 : (ce <= kNT / 2) ? 2 : 1;
+  const int per = kNT / nh;
+  float* fold = part;                   // [nh][ce] (nh > 1 only)
+  for (int idx0 = 0; idx0 < ce; idx0 += per) {
+    const int idx = idx0 + (tid % per), h = tid / per;
     float s = 0.f;
-    for (int bb = 0; bb < p.B; ++bb) s = fmaf(U1[bb * r1 + i], __ldcg(p.Tb + (int64_t)bb * n234 + rest), s);
-    p.core[idx] = s;
+    if (idx < ce) {
+#pragma unroll 32
+      for (int t = h; t < p.n_tiles; t += nh) s += __ldcg(p.Tp + (int64_t)t * ce + idx);
+      if (nh == 1) p.core[idx] = s;
+      else fold[h * ce + idx] = s;
+    }
+  }
+  if (nh > 1) {
+    __syncthreads();
+    for (int idx = tid; idx < ce; idx += kNT) {
+      float s = 0.f;
+      for (int h = 0; h < nh; ++h) s += fold[h * ce + idx];
+      p.core[idx] = s;
+    }
   }
   if (tid == 0) *p.counter = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_sm_wgrad: CTA owns CPB consecutive output channels.
-//   Z3 = core x_3 U3 x_4 U4 (recomputed per CTA, tiny);  Z1 = dY x_1 U1^T on the CTA's channels;
+// k_sm_wgrad: CTA owns cpb consecutive output channels, i.e. the dY tile [B x J], J = cpb*Ho*Wo
+// contiguous values per sample (staged by the bulk-copy engine when fp32).
+//   Z3 = core x_3 U3 x_4 U4 (recomputed per CTA while the tile is in flight);
+//   Z1 = dY x_1 U1^T on the CTA's channels;
 //   Z4[c',j,kh,kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p];  dW = Z4 x_2 U2.
 // ---------------------------------------------------------------------------------------------
+template <int R, int KK>
+__device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const float* __restrict__ Z4s,
+                                                  const float* __restrict__ U2s, int c0) {
+  // thread -> fixed kernel tap t = tid mod kk; it walks the input channels c = tid / kk + k * (nthr / kk)
+  const int kk = (KK > 0) ? KK : p.kh * p.kw;
+  const int r2 = p.r[1];
+  const int cg = p.C / p.groups, og = p.Cout / p.groups;
+  const int cstep = kNT / kk, nthr = cstep * kk;
+  const int tid = threadIdx.x;
+  if (tid >= nthr) return;
+  const int t = tid % kk, cfirst = tid / kk;
+  for (int cl = 0; cl < p.cpb; ++cl) {
+    const int co = c0 + cl;
+    const int g = co / og;
+    float* dw = p.dW + (int64_t)co * cg * kk + t;
+    const float* u2 = U2s + (int64_t)g * cg * R;
+    float z[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) z[j] = (j < r2) ? Z4s[(cl * r2 + j) * kk + t] : 0.f;
+#pragma unroll 4
+    for (int c = cfirst; c < cg; c += cstep) {
+      float v = 0.f;
+#pragma unroll
+      for (int j = 0; j < R; j += 4) {
+        const float4 u = *reinterpret_cast<const float4*>(u2 + c * R + j);
+        v = fmaf(z[j], u.x, v);
+        v = fmaf(z[j + 1], u.y, v);
+        v = fmaf(z[j + 2], u.z, v);
+        v = fmaf(z[j + 3], u.w, v);
+      }
+      dw[(int64_t)c * kk] = v;
+    }
+  }
+}
+
 template <int R, typename TX>
-__global__ void __launch_bounds__(256) k_sm_wgrad(SmWgradArgs p) {
-  extern __shared__ __align__(16) float smem[];
+__global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_flag;
   const int tid = threadIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
   const int H = p.H, W = p.W, HW = H * W, HoWo = p.Ho * p.Wo, kk = p.kh * p.kw;
   const int J = p.cpb * HoWo;                        // dY columns of this CTA, contiguous per sample
+  const int PJ = p.pj;
+  const int NH = batch_groups(kNT, J);
   const int c0 = blockIdx.x * p.cpb;
-  float* U1s = smem;                                 // [B][R]
-  float* Ss = U1s + p.B * R;                         // [r1 r2 r3 r4]
+  const int n_out = p.cpb * r2 * kk;
+  float* Ys = smem;                                  // [B][PJ]
+  float* U1s = Ys + p.B * PJ;                        // [B][R]
+  float* U2s = U1s + p.B * R;                        // [C][R]
+  float* Z1s = U2s + p.C * R;                        // [J][R]
+  float* part = Z1s + J * R;                         // [NH][J][R] (NH > 1 only)
+  float* Ss = part + (NH > 1 ? NH : 0) * J * R;      // [r1 r2 r3 r4]
   float* U3s = Ss + r1 * r2 * r3 * r4;               // [H][r3]
   float* U4s = U3s + H * r3;                         // [W][r4]
   float* Tm = U4s + W * r4;                          // [r1 r2][H][r4]
   float* Z3s = Tm + r1 * r2 * H * r4;                // [r1 r2][H][W]
-  float* Z1s = Z3s + r1 * r2 * HW;                   // [J][R]
-  float* Z4s = Z1s + J * R;                          // [cpb][r2][kk]
-  float* red = Z4s + p.cpb * r2 * kk;                // [nsplit][cpb r2 kk]
+  float* Z4s = Z3s + r1 * r2 * HW;                   // [cpb][r2][kk]
+  float* red = Z4s + n_out;                          // [r1][cpb r2 kk]
 
-  load_factor<R>(U1s, p.U + p.u_off[0], p.B, r1);
-  for (int idx = tid; idx < r1 * r2 * r3 * r4; idx += 256) Ss[idx] = p.core[idx];
-  for (int idx = tid; idx < H * r3; idx += 256) U3s[idx] = p.U[p.u_off[2] + idx];
-  for (int idx = tid; idx < W * r4; idx += 256) U4s[idx] = p.U[p.u_off[3] + idx];
-  __syncthreads();
-
-  // term 1: Z1[j,:] = sum_b dY[b, c0*HoWo + j] U1[b,:]  (thread per column, coalesced per sample)
   const TX* dY = reinterpret_cast<const TX*>(p.dY) + (int64_t)c0 * HoWo;
   const int64_t sstride = (int64_t)p.Cout * HoWo;
-  for (int j = tid; j < J; j += 256) {
-    float acc[R];
-#pragma unroll
-    for (int q = 0; q < R; ++q) acc[q] = 0.f;
-#pragma unroll 8
-    for (int b = 0; b < p.B; ++b) {
-      const float x = to_f(dY[b * sstride + j]);
-#pragma unroll
-      for (int q = 0; q < R; q += 4) {
-        const float4 u = *reinterpret_cast<const float4*>(U1s + b * R + q);
-        acc[q] = fmaf(x, u.x, acc[q]);
-        acc[q + 1] = fmaf(x, u.y, acc[q + 1]);
-        acc[q + 2] = fmaf(x, u.z, acc[q + 2]);
-        acc[q + 3] = fmaf(x, u.w, acc[q + 3]);
-      }
+  const bool bulk = std::is_same<TX, float>::value && p.bulk;
+  if (bulk) {
+    stage_rows(&s_bar, reinterpret_cast<char*>(Ys), reinterpret_cast<const char*>(dY), p.B, (uint32_t)J * 4u,
+               sstride * 4, (uint32_t)PJ * 4u);
+  } else {
+    for (int idx = tid; idx < p.B * J; idx += kNT) {
+      const int b = idx / J, j = idx - b * J;
+      Ys[b * PJ + j] = to_f(dY[b * sstride + j]);
     }
-#pragma unroll
-    for (int q = 0; q < R; ++q) Z1s[j * R + q] = acc[q];
   }
+  {
+    const FacDesc fd[5] = {{p.core, Ss, 1, r1 * r2 * r3 * r4, r1 * r2 * r3 * r4},
+                           {p.U + p.u_off[2], U3s, H, r3, r3},
+                           {p.U + p.u_off[3], U4s, W, r4, r4},
+                           {p.U + p.u_off[0], U1s, p.B, r1, R},
+                           {p.U + p.u_off[1], U2s, p.C, r2, R}};
+    load_factors<5>(fd);
+  }
+  __syncthreads();
   // terms 2-3: Tm[ij][h][l] = sum_k S[ij][k][l] U3[h][k];  Z3[ij][h][w] = sum_l Tm[ij][h][l] U4[w][l]
-  for (int idx = tid; idx < r1 * r2 * H * r4; idx += 256) {
+  for (int idx = tid; idx < r1 * r2 * H * r4; idx += kNT) {
     const int l = idx % r4, h = (idx / r4) % H, ij = idx / (r4 * H);
     float s = 0.f;
     for (int k = 0; k < r3; ++k) s = fmaf(Ss[(ij * r3 + k) * r4 + l], U3s[h * r3 + k], s);
     Tm[idx] = s;
   }
   __syncthreads();
-  for (int idx = tid; idx < r1 * r2 * HW; idx += 256) {
+  for (int idx = tid; idx < r1 * r2 * HW; idx += kNT) {
     const int w = idx % W, h = (idx / W) % H, ij = idx / HW;
     float s = 0.f;
     for (int l = 0; l < r4; ++l) s = fmaf(Tm[(ij * H + h) * r4 + l], U4s[w * r4 + l], s);
     Z3s[idx] = s;
   }
-  __syncthreads();
-  // term 4: thread (o, s): output o = (cl, j, kh, kw), split s of the (i, h') reduction
-  const int n_out = p.cpb * r2 * kk;
-  int nsplit = 256 / n_out;
-  if (nsplit < 1) nsplit = 1;
-  const int n_items = r1 * p.Ho;
-  if (nsplit > n_items) nsplit = n_items;
-  for (int t = tid; t < n_out * nsplit; t += 256) {
-    const int o = t % n_out, s = t / n_out;
+  if (bulk) {
+    if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
+  } else {
+    __syncthreads();
+  }
+  // term 1: Z1[j,:] = sum_b dY[b, c0*HoWo + j] U1[b,:]
+  project_batch<R>(Ys, PJ, U1s, p.B, J, part, Z1s, tid, kNT, 0);
+  // term 4: thread (o, i): output o = (cl, j, kh, kw), pseudo-sample i, over the (h', w') that fall
+  // inside the map; the r1 partial sums meet in order
+  for (int it = tid; it < n_out * r1; it += kNT) {
+    const int o = it % n_out, i = it / n_out;
     const int cl = o / (r2 * kk), j = (o / kk) % r2, tt = o % kk, ky = tt / p.kw, kx = tt % p.kw;
+    // h = ho*sh + ky - ph in [0, H)  <=>  ho in [ho_lo, ho_hi)
+    int ho_lo = (p.ph - ky + p.sh - 1) / p.sh, ho_hi = (H - 1 + p.ph - ky) / p.sh + 1;
+    int wo_lo = (p.pw - kx + p.sw - 1) / p.sw, wo_hi = (W - 1 + p.pw - kx) / p.sw + 1;
+    if (p.ph - ky < 0) ho_lo = 0;
+    if (p.pw - kx < 0) wo_lo = 0;
+    if (ho_hi > p.Ho) ho_hi = p.Ho;
+    if (wo_hi > p.Wo) wo_hi = p.Wo;
     float acc = 0.f;
-    for (int it = s; it < n_items; it += nsplit) {
-      const int i = it / p.Ho, ho = it % p.Ho;
-      const int h = ho * p.sh + ky - p.ph;
-      if (h < 0 || h >= H) continue;
+    for (int ho = ho_lo; ho < ho_hi; ++ho) {
       const float* z1 = Z1s + (cl * HoWo + ho * p.Wo) * R + i;
-      const float* z3 = Z3s + ((i * r2 + j) * H + h) * W;
-      for (int wo = 0; wo < p.Wo; ++wo) {
-        const int w = wo * p.sw + kx - p.pw;
-        if (w >= 0 && w < W) acc = fmaf(z1[wo * R], z3[w], acc);
-      }
+      const float* z3 = Z3s + ((i * r2 + j) * H + ho * p.sh + ky - p.ph) * W + kx - p.pw;
+#pragma unroll 7
+      for (int wo = wo_lo; wo < wo_hi; ++wo) acc = fmaf(z1[wo * R], z3[wo * p.sw], acc);
     }
-    red[s * n_out + o] = acc;
+    red[i * n_out + o] = acc;
   }
   __syncthreads();
-  for (int o = tid; o < n_out; o += 256) {
+  for (int o = tid; o < n_out; o += kNT) {
     float v = 0.f;
-    for (int s = 0; s < nsplit; ++s) v += red[s * n_out + o];
+    for (int i = 0; i < r1; ++i) v += red[i * n_out + o];
     Z4s[o] = v;
   }
   __syncthreads();
   // term 5: dW[c0+cl, c, t] = sum_j Z4[cl][j][t] U2[(g cg + c), j]
-  const int cg = p.C / p.groups, og = p.Cout / p.groups;
-  const float* U2 = p.U + p.u_off[1];
-  for (int cl = 0; cl < p.cpb; ++cl) {
-    const int co = c0 + cl;
-    const int g = co / og;
-    float* dw = p.dW + (int64_t)co * cg * kk;
-    const float* z4 = Z4s + cl * r2 * kk;
-    for (int idx = tid; idx < cg * kk; idx += 256) {
-      const int c = idx / kk, t = idx % kk;
-      const float* u = U2 + (int64_t)(g * cg + c) * r2;
-      float v = 0.f;
-      for (int j = 0; j < r2; ++j) v = fmaf(z4[j * kk + t], __ldg(u + j), v);
-      dw[idx] = v;
-    }
-  }
+  if (kk == 9) wgrad_expand_rows<R, 9>(p, Z4s, U2s, c0);
+  else if (kk == 1) wgrad_expand_rows<R, 1>(p, Z4s, U2s, c0);
+  else wgrad_expand_rows<R, 0>(p, Z4s, U2s, c0);
 }
 
 // ---------------------------------------------------------------------------------------------
 // host-side launchers
 // ---------------------------------------------------------------------------------------------
+int sm_pass1_role_c_ctas(int S, int B) { return (S == 7) ? B : 4 * B; }
+
 size_t sm_pass1_smem(int S, int R, int B, int C) {
-  const int HW = S * S, CC = (S == 7) ? 4 : 1, J = CC * HW, PJ = (J % 32 == 4) ? J : J + 4;
-  const size_t role_b = (size_t)B * PJ + (size_t)B * R + 2 * S * R + (size_t)J * R + 8 * S * R;
-  const int G = 256 / HW;
-  const size_t role_c = (size_t)C * R + (size_t)G * HW * R + (size_t)HW * R;
+  const int HW = S * S, CC = (S == 7) ? 4 : 1, J = CC * HW, PJ = pitch4(J);
+  const int NH1 = batch_groups(kNG, J);
+  const size_t role_b = (size_t)B * PJ + (size_t)B * R + 2 * S * R + (size_t)J * R +
+                        (NH1 > 1 ? (size_t)NH1 * J * R : 0) + 8 * 32;
+  const int HWC = (S == 7) ? HW : HW / 4;
+  const int PC = (HWC % 2 == 0) ? HWC + 1 : HWC;
+  const int G = kNT / HWC;
+  const size_t vp = (C >= (G - 1) * HWC) ? 0 : (size_t)(G - 1) * HWC * R;
+  const size_t role_c = (size_t)((C * PC + 3) & ~3) + (size_t)C * R + (size_t)HWC * R + vp;
   return 4 * (role_b > role_c ? role_b : role_c);
 }
 
-size_t sm_core_smem(int S, int R, int C) {
-  const int HW = S * S, G = 256 / HW;
-  return 4 * ((size_t)C * R + (size_t)G * HW * R + (size_t)HW * R + 2 * S * R + (size_t)R * R * S);
+size_t sm_core_smem(int S, int R, int B) {
+  const int HW = S * S, CC = (S == 7) ? 4 : 1, J = CC * HW, PJ = pitch4(J);
+  const int NH = batch_groups(kNT, J);
+  return 4 * ((size_t)B * PJ + (size_t)B * R + (size_t)CC * R + 2 * S * R + (size_t)J * R + (size_t)NH * J * R +
+              (size_t)R * R * HW + (size_t)R * R * R * S);
 }
+
+int sm_core_max_rows() { return kNT; }
+
+int sm_wgrad_pitch(int J) { return pitch4(J); }
 
 size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
   const int HW = p.H * p.W, J = p.cpb * p.Ho * p.Wo, kk = p.kh * p.kw;
   const int n_out = p.cpb * r2 * kk;
-  int nsplit = 256 / n_out;
-  if (nsplit < 1) nsplit = 1;
-  size_t n = (size_t)p.B * R + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
-             (size_t)r1 * r2 * p.H * r4 + (size_t)r1 * r2 * HW + (size_t)J * R + n_out +
-             (size_t)nsplit * n_out;
+  const int NH = batch_groups(kNT, J);
+  size_t n = (size_t)p.B * pitch4(J) + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
+             (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
+             (size_t)r1 * r2 * p.H * r4 + (size_t)r1 * r2 * HW + n_out + (size_t)r1 * n_out;
   return 4 * n + 64;
+}
+
+template <typename K>
+static cudaError_t opt_in_smem(K kernel, bool* done) {
+  if (*done) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e == cudaSuccess) *done = true;
+  return e;
 }
 
 template <int S, int R, typename TX>
 static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
-  const size_t smem = sm_pass1_smem(S, R, p.B, p.C);
   static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_sm_pass1<S, R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kMaxDynSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  k_sm_pass1<S, R, TX><<<p.n_tiles_b + p.B, 256, smem, st>>>(p);
+  cudaError_t e = opt_in_smem(k_sm_pass1<S, R, TX>, &attr_done);
+  if (e != cudaSuccess) return e;
+  k_sm_pass1<S, R, TX><<<p.n_tiles_b + sm_pass1_role_c_ctas(S, p.B), kNT, sm_pass1_smem(S, R, p.B, p.C), st>>>(p);
   return cudaGetLastError();
 }
 
 template <int S, int R, typename TX>
 static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
-  const size_t smem = sm_core_smem(S, R, p.C);
   static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_sm_core<S, R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kMaxDynSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  k_sm_core<S, R, TX><<<p.B, 256, smem, st>>>(p);
+  cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &attr_done);
+  if (e != cudaSuccess) return e;
+  k_sm_core<S, R, TX><<<p.n_tiles, kNT, sm_core_smem(S, R, p.B), st>>>(p);
   return cudaGetLastError();
 }
 
 template <int R, typename TX>
 static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
-  const size_t smem = sm_wgrad_smem(p, R);
   static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(k_sm_wgrad<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kMaxDynSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  k_sm_wgrad<R, TX><<<p.Cout / p.cpb, 256, smem, st>>>(p);
+  cudaError_t e = opt_in_smem(k_sm_wgrad<R, TX>, &attr_done);
+  if (e != cudaSuccess) return e;
+  k_sm_wgrad<R, TX><<<p.Cout / p.cpb, kNT, sm_wgrad_smem(p, R), st>>>(p);
   return cudaGetLastError();
 }
 
@@ -549,7 +1086,8 @@ static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st) {
   const size_t eb = bf16 ? 2 : 4;
   double bytes = (double)p.B * p.C * S * S * eb;
-  bytes += 4.0 * ((double)p.n_tiles_b * (p.B * p.r[0] + S * p.r[2] + S * p.r[3]) + (double)p.B * p.C * p.r[1]);
+  const double m34 = (S == 7) ? 2.0 * S * S : (double)S * (p.r[2] + p.r[3]);
+  bytes += 4.0 * ((double)p.n_tiles_b * (p.B * p.r[0] + m34) + (double)p.B * p.C * p.r[1]);
   ProfScope prof(ASI_K_SM_PASS1, st, bytes);
   ASI_DISPATCH_SR(launch_pass1_t, p);
 }

@@ -86,9 +86,9 @@ def test_fused_small_map_kernels(case):
                      rho=tuple(_rho(r) for r in ranks), bf16=bf16,
                      gen_ranks=tuple(min(d, max(r + 2, 4)) for d, r in zip(dims, ranks)))
     run = make_runner(L, bf16=bf16)
-    assert run.plan.launch_count(0) == 4 and run.plan.launch_count(1) == 1   # fused path chosen
+    assert run.plan.launch_count(0) == 3 and run.plan.launch_count(1) == 1   # fused path chosen
     gen = make_runner(L, bf16=bf16, generic_only=True)
-    assert gen.plan.launch_count(0) > 4
+    assert gen.plan.launch_count(0) > 3
     U_prev = st.u_prev0()
     for t in range(2):
         A, dY = st.next()
