@@ -121,6 +121,34 @@ asi_status_t asi_compress(const asi_plan_t* plan, const void* act, const float* 
 asi_status_t asi_init_factors(const asi_plan_t* plan, const void* act, const float* omega,
                               float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
 
+/* asi_compress for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a deployment convenience, not part of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a training-loop hook that must
+ * not disturb the framework's caching allocator, a latency-critical loop in which an allocation
+ * (which synchronises the device) is not acceptable, or a process whose device-memory budget was
+ * fixed at start-up.  Such a caller still owns act, U_prev, U_new and core, but has nowhere to
+ * get the scratch workspace from.
+ *
+ * This entry point computes exactly what asi_compress computes, with the workspace taken from an
+ * array of ASI_STATIC_WS_MAX_BYTES that is part of the library image: every GPU that loads the
+ * library holds that array until the process exits.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ *   - A plan whose compress_ws_bytes exceeds ASI_STATIC_WS_MAX_BYTES is refused with
+ *     ASI_ERR_WORKSPACE and nothing is enqueued (asi_last_cuda_error() then holds the two sizes).
+ *   - The first call on each device looks up the array's device address (one runtime query, with
+ *     that device current).  Make that first call before any stream capture begins.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call left in
+ *     it.  The words that must start at zero (status word, completion counters) are cleared by the
+ *     call itself.  Two calls whose GPU work overlaps -- different streams, or several host threads
+ *     -- race on the array: keep them on one stream or order them with events.
+ *   - The device status word sits inside the shared array, so asi_poll_status cannot be used with
+ *     this variant: a rank-deficient iterate is not reported.  Use asi_compress with a workspace
+ *     of your own when you need that check. */
+#define ASI_STATIC_WS_MAX_BYTES (4u << 20)
+asi_status_t asi_compress_static_ws(const asi_plan_t* plan, const void* act, const float* U_prev,
+                                    float* U_new, float* core, void* stream);
+
 /* Weight gradient of a conv2d layer from the compressed activation, in the
  * order the five terms of C_ASI fix (appendix "Speedup"):
  *   Z1 = dY x_1 U_1^T;  Z3 = core x_3 U_3 x_4 U_4;

@@ -25,9 +25,11 @@ ASI_ERR_TIMEOUT = 7
 ASI_F32, ASI_BF16 = 0, 1
 ASI_CONV2D, ASI_LINEAR = 0, 1
 ASI_MAX_MODES = 4
+ASI_STATIC_WS_MAX_BYTES = 4 << 20
 
 EXPORTS = (
-    "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_init_factors",
+    "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
+    "asi_init_factors",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
     "asi_profile_end", "asi_last_cuda_error",
@@ -75,6 +77,7 @@ def lib():
     L.asi_plan_destroy.argtypes = [vp]
     L.asi_plan_query.argtypes = [vp, C.POINTER(PlanInfo)]
     L.asi_compress.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_compress_static_ws.argtypes = [vp, vp, vp, vp, vp, vp]
     L.asi_init_factors.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_linear_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
@@ -92,7 +95,7 @@ def lib():
     L.asi_last_cuda_error.restype = C.c_char_p
     L.asi_status_string.argtypes = [i32]
     L.asi_status_string.restype = C.c_char_p
-    for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress",
+    for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
                  "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
                  "asi_poll_status"):
         getattr(L, name).restype = i32
@@ -165,6 +168,11 @@ class Plan:
     def compress(self, act, U_prev, U_new, core, ws, ws_bytes, stream=0):
         _check(lib().asi_compress(self._h, act, U_prev, U_new, core, ws, ws_bytes, stream),
                "asi_compress")
+
+    def compress_static_ws(self, act, U_prev, U_new, core, stream=0):
+        """asi_compress with the library's built-in scratch array (no workspace argument)."""
+        _check(lib().asi_compress_static_ws(self._h, act, U_prev, U_new, core, stream),
+               "asi_compress_static_ws")
 
     def init_factors(self, act, omega, U_new, core, ws, ws_bytes, stream=0):
         _check(lib().asi_init_factors(self._h, act, omega, U_new, core, ws, ws_bytes, stream),

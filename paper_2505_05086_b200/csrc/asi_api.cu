@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "asi_internal.h"
@@ -473,6 +474,43 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     if (s != ASI_OK) return s;
   }
   return finish_compress(pl, act, U_new, core, w, nullptr, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// asi_compress with the workspace in the library image, for callers that may not allocate.
+// g_static_ws names the array only in device code; host code must ask the runtime for its device
+// address (once per device, with that device current) and hand that address to the kernels.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_ws[ASI_STATIC_WS_MAX_BYTES];
+
+asi_status_t asi_compress_static_ws(const asi_plan_t* pl, const void* act, const float* U_prev,
+                                    float* U_new, float* core, void* stream) {
+  constexpr int kMaxDevices = 64;
+  static void* addr_of_device[kMaxDevices] = {};
+  static std::mutex setup_lock;
+  if (!pl) return ASI_ERR_INVALID_ARG;
+  if (pl->compress_ws > (size_t)ASI_STATIC_WS_MAX_BYTES) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err),
+             "asi_compress_static_ws: the plan needs %zu bytes of scratch, the built-in array holds %u",
+             pl->compress_ws, (unsigned)ASI_STATIC_WS_MAX_BYTES);
+    return ASI_ERR_WORKSPACE;
+  }
+  int dev = -1;
+  ASI_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ASI_ERR_UNSUPPORTED;
+  void* ws = nullptr;
+  {
+    std::lock_guard<std::mutex> guard(setup_lock);
+    if (!addr_of_device[dev]) {
+      void* p = nullptr;
+      ASI_CUDA(cudaGetSymbolAddress(&p, g_static_ws));
+      addr_of_device[dev] = p;
+    }
+    ws = addr_of_device[dev];
+  }
+  // asi_compress clears the status word and the completion counters itself; everything else in the
+  // array is written before it is read.
+  return asi_compress(pl, act, U_prev, U_new, core, ws, (size_t)ASI_STATIC_WS_MAX_BYTES, stream);
 }
 
 asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float* omega, float* U_new,
