@@ -50,16 +50,21 @@ void choose_kernels(asi_plan* pl) {
   if (B <= 4096 && H <= 64 && W <= 64) {
     const int Cout = pl->d.cout;
     const int64_t HoWo = pl->Ho * pl->Wo;
-    // channels per CTA: the smallest count that makes a staged row a multiple of 16 bytes
-    int cpb = 1;
-    while (cpb < 4 && ((cpb * HoWo * 4) % 16 != 0 || Cout % cpb != 0)) cpb *= 2;
-    const bool rows_ok = (cpb * HoWo * 4) % 16 == 0 && Cout % cpb == 0;
-    if (!rows_ok) cpb = 1;
+    // channels per CTA: the smallest count that makes a staged row a multiple of 16 bytes (rows can
+    // then be staged by the bulk-copy engine); failing that, the smallest that makes it even
+    int cpb = 0;
+    bool rows_ok = false;
+    for (int c = 1; c <= 4 && !cpb; c *= 2)
+      if (Cout % c == 0 && (c * HoWo * 4) % 16 == 0) { cpb = c; rows_ok = true; }
+    for (int c = 1; c <= 2 && !cpb; c *= 2)
+      if (Cout % c == 0 && (c * HoWo) % 2 == 0) cpb = c;
+    if (!cpb) return;
     SmWgradArgs a;
     std::memset(&a, 0, sizeof(a));
     for (int m = 0; m < 4; ++m) a.r[m] = pl->r[m];
     a.B = (int)B; a.C = (int)C; a.Cout = Cout; a.H = (int)H; a.W = (int)W;
     a.Ho = (int)pl->Ho; a.Wo = (int)pl->Wo; a.kh = pl->d.kh; a.kw = pl->d.kw; a.cpb = cpb;
+    a.ph = pl->d.pad_h; a.pw = pl->d.pad_w;
     if (sm_wgrad_smem(a, R) <= kSmemLimit) {
       pl->fast_wgrad = true;
       pl->cpb = cpb;

@@ -153,9 +153,11 @@ __device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char
   }
 }
 
-// Small read-only arrays a CTA keeps in shared memory (factors, the core).  All of them are fetched
-// in ONE batch: every thread first issues the loads of all its elements, then stores them, so the
-// prologue costs a single global-memory round trip.  Element (k, j) of array i, j < r_dst:
+// Small read-only arrays a CTA keeps in shared memory (factors, the core).  fac_issue() starts one
+// 4-byte asynchronous copy (cp.async) per element -- a compact loop, no registers held -- and
+// fac_wait() waits for this thread's copies; a __syncthreads() after it publishes them.  Whatever a
+// kernel does in between overlaps the single round trip, and these small loads are ahead of its bulk
+// traffic in the memory system.  Element (k, j) of array i, j < r_dst:
 // dst[k*r_dst + j] = j < r_src ? src[k*r_src + j] : 0.
 struct FacDesc {
   const float* src;
@@ -163,41 +165,41 @@ struct FacDesc {
   int rows, r_src, r_dst;
 };
 template <int NF>
-__device__ __forceinline__ void load_factors(const FacDesc (&f)[NF]) {
-  constexpr int MAXI = 8;
-  int n[NF], total = 0;
+__device__ __forceinline__ void fac_issue(const FacDesc (&f)[NF]) {
+  int total = 0;
 #pragma unroll
-  for (int i = 0; i < NF; ++i) {
-    n[i] = f[i].rows * f[i].r_dst;
-    total += n[i];
-  }
-  for (int base = 0; base < total; base += kNT * MAXI) {
-    float v[MAXI];
-    float* d[MAXI];
+  for (int i = 0; i < NF; ++i) total += f[i].rows * f[i].r_dst;
+#pragma unroll 1
+  for (int idx0 = threadIdx.x; idx0 < total; idx0 += kNT) {
+    int idx = idx0;
+    const float* src = f[0].src;
+    float* dst = f[0].dst;
+    int fill = 0;
 #pragma unroll
-    for (int k = 0; k < MAXI; ++k) {
-      int idx = base + k * kNT + (int)threadIdx.x;
-      v[k] = 0.f;
-      d[k] = nullptr;
-      if (idx < total) {
-#pragma unroll
-        for (int i = 0; i < NF; ++i) {
-          if (d[k] == nullptr) {
-            if (idx < n[i]) {
-              const int row = idx / f[i].r_dst, j = idx - row * f[i].r_dst;
-              d[k] = f[i].dst + idx;
-              if (j < f[i].r_src) v[k] = __ldg(f[i].src + row * f[i].r_src + j);
-            } else {
-              idx -= n[i];
-            }
+    for (int i = 0; i < NF; ++i) {
+      const int n = f[i].rows * f[i].r_dst;
+      if (idx >= 0 && idx < n) {
+        dst = f[i].dst + idx;
+        if (f[i].r_src == f[i].r_dst) {
+          src = f[i].src + idx;
+          fill = 4;
+        } else {
+          const int row = idx / f[i].r_dst, j = idx - row * f[i].r_dst;
+          if (j < f[i].r_src) {
+            src = f[i].src + row * f[i].r_src + j;
+            fill = 4;
           }
         }
+        idx = -1;
+      } else if (idx >= 0) {
+        idx -= n;
       }
     }
-#pragma unroll
-    for (int k = 0; k < MAXI; ++k)
-      if (d[k] != nullptr) *d[k] = v[k];
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(fill) : "memory");
   }
+}
+__device__ __forceinline__ void fac_wait() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
 }
 
 template <int R>
@@ -211,6 +213,27 @@ __device__ __forceinline__ void fma_row(float (&acc)[R], float x, const float* _
     acc[j + 3] = fmaf(x, v.w, acc[j + 3]);
   }
 }
+
+// Programmatic dependent launch: the reduce and core kernels are launched with the
+// programmatic-stream-serialization attribute, so their CTAs may start (and do whatever does not
+// depend on the previous kernel, e.g. stage their activation tile) once every CTA of the previous
+// kernel has passed pdl_launch_dependents(); pdl_wait() then blocks until that kernel has finished
+// and its writes are visible.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Division of a small index (n < 2^21) by a run-time divisor through one reciprocal: the integer
+// division sequence costs ~150 cycles of latency, which dominates the short index loops below.
+struct FDiv {
+  float inv;
+  int d;
+  __device__ __forceinline__ explicit FDiv(int d_) : inv(1.0f / (float)d_), d(d_) {}
+  __device__ __forceinline__ int div(int n) const { return __float2int_rd(((float)n + 0.5f) * inv); }
+  __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
+    q = div(n);
+    r = n - q * d;
+  }
+};
 
 __device__ __forceinline__ void bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -247,7 +270,7 @@ __device__ __forceinline__ int scatter_base(int lane) {
 
 // Number of interleaved sample groups project_batch uses for a tile of J columns on nthr threads.
 __host__ __device__ constexpr int batch_groups(int nthr, int J) {
-  const int items = (J % 2 == 0) ? J / 2 : J;
+  const int items = J / 2;
   int nh = nthr / items;
   return nh < 1 ? 1 : (nh > 4 ? 4 : nh);
 }
@@ -262,41 +285,31 @@ __device__ __forceinline__ void project_batch(const float* __restrict__ Xs, int 
                                               float* __restrict__ part, float* __restrict__ out, int t,
                                               int nthr, int bar) {
   const int NH = batch_groups(nthr, J);
-  if ((J & 1) == 0) {
-    const int J2 = J >> 1;
-    for (int it = t; it < NH * J2; it += nthr) {
-      const int h = it / J2, jp = it - h * J2;
-      float a0[R], a1[R];
+  const int J2 = J >> 1;                             // J is even
+  const FDiv dJ2(J2);
+#pragma unroll 1
+  for (int it = t; it < NH * J2; it += nthr) {
+    int h, jp;
+    dJ2.divmod(it, h, jp);
+    float a0[R], a1[R];
 #pragma unroll
-      for (int q = 0; q < R; ++q) a0[q] = a1[q] = 0.f;
-#pragma unroll 8
-      for (int b = h; b < B; b += NH) {
-        const float2 x = *reinterpret_cast<const float2*>(Xs + b * PJ + 2 * jp);
-        fma_row<R>(a0, x.x, Us + b * R);
-        fma_row<R>(a1, x.y, Us + b * R);
-      }
-      float* dst = (NH > 1 ? part + h * J * R : out) + 2 * jp * R;
-#pragma unroll
-      for (int q = 0; q < R; q += 4) {
-        *reinterpret_cast<float4*>(dst + q) = make_float4(a0[q], a0[q + 1], a0[q + 2], a0[q + 3]);
-        *reinterpret_cast<float4*>(dst + R + q) = make_float4(a1[q], a1[q + 1], a1[q + 2], a1[q + 3]);
-      }
+    for (int q = 0; q < R; ++q) a0[q] = a1[q] = 0.f;
+#pragma unroll 4
+    for (int b = h; b < B; b += NH) {
+      const float2 x = *reinterpret_cast<const float2*>(Xs + b * PJ + 2 * jp);
+      fma_row<R>(a0, x.x, Us + b * R);
+      fma_row<R>(a1, x.y, Us + b * R);
     }
-  } else {
-    for (int it = t; it < NH * J; it += nthr) {
-      const int h = it / J, j = it - h * J;
-      float acc[R];
+    float* dst = (NH > 1 ? part + h * J * R : out) + 2 * jp * R;
 #pragma unroll
-      for (int q = 0; q < R; ++q) acc[q] = 0.f;
-#pragma unroll 8
-      for (int b = h; b < B; b += NH) fma_row<R>(acc, Xs[b * PJ + j], Us + b * R);
-      float* dst = (NH > 1 ? part + h * J * R : out) + j * R;
-#pragma unroll
-      for (int q = 0; q < R; ++q) dst[q] = acc[q];
+    for (int q = 0; q < R; q += 4) {
+      *reinterpret_cast<float4*>(dst + q) = make_float4(a0[q], a0[q + 1], a0[q + 2], a0[q + 3]);
+      *reinterpret_cast<float4*>(dst + R + q) = make_float4(a1[q], a1[q + 1], a1[q + 2], a1[q + 3]);
     }
   }
   if (NH > 1) {
     bar_sync(bar, nthr);
+#pragma unroll 1
     for (int idx = t; idx < J * R; idx += nthr) {
       float s = 0.f;
       for (int h = 0; h < NH; ++h) s += part[h * J * R + idx];
@@ -384,6 +397,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
   const int B = p.B, C = p.C;
 
   if (blockIdx.x == 0 && tid < 9) p.status[tid == 0 ? 0 : 15 + tid] = 0;   // status word, counters 16..23
+  pdl_launch_dependents();
 
   constexpr int kNQ = (S == 7) ? 1 : 4;             // role-C CTAs per sample
   if ((int)blockIdx.x >= B * kNQ) {
@@ -396,12 +410,13 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* V1s = U4s + S * R;                        // [J][R]
     float* part = V1s + J * R;                       // [NH1][J][R] (NH1 > 1 only)
     float* red = part + (NH1 > 1 ? NH1 : 0) * J * R; // [8][32]
-    stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
     {
       const FacDesc fd[3] = {{p.U_prev + p.u_off[0], U1s, B, p.r[0], R},
                              {p.U_prev + p.u_off[2], U3s, S, p.r[2], R},
                              {p.U_prev + p.u_off[3], U4s, S, p.r[3], R}};
-      load_factors<3>(fd);
+      fac_issue<3>(fd);
+      stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
+      fac_wait();
     }
     if constexpr (kBulk) {
       if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
@@ -543,6 +558,8 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* V2s = U2s + C * R;                        // [HWC][R]
     float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
     const TX* Xb = A + (int64_t)b * C * HW + q * HWC;
+    const FacDesc fdc[1] = {{p.U_prev + p.u_off[1], U2s, C, p.r[1], R}};
+    fac_issue<1>(fdc);
     if constexpr (kBulkC) {
       stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
     } else if constexpr (NQ == 1) {
@@ -550,16 +567,13 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
       for (int idx = tid; idx < n4; idx += kNT) *reinterpret_cast<float4*>(Xs + 4 * idx) = ld4<TX>(Xb + 4 * idx);
     } else {
       const int n = C * HWC;
-#pragma unroll 8
+#pragma unroll 4
       for (int idx = tid; idx < n; idx += kNT) {
         const int c = idx / HWC, hw = idx - c * HWC;
         Xs[c * PC + hw] = to_f(Xb[(int64_t)c * HW + hw]);
       }
     }
-    {
-      const FacDesc fd[1] = {{p.U_prev + p.u_off[1], U2s, C, p.r[1], R}};
-      load_factors<1>(fd);
-    }
+    fac_wait();
     if constexpr (kBulkC) {
       if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
     } else {
@@ -593,7 +607,9 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   constexpr int RM = 8, RPC = kRedRows;
   const SmReduceMode M = args.m[blockIdx.y];
   const int c = blockIdx.x;
+  pdl_launch_dependents();
   if (c >= M.nchunk) return;
+  pdl_wait();                                      // the partials come from the previous kernel
   __shared__ double part[kRedNT];
   __shared__ double Ps[RPC][RM];
   __shared__ double Gm[RPC * RPC];
@@ -602,18 +618,19 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   const int row0 = c * RPC;
   const int nrow = (a - row0 < RPC) ? (a - row0) : RPC;
   const int E = M.gram ? a * a : nrow * r;         // <= 256
+  const FDiv dr(r);
   int EP = 32;
   while (EP < E) EP <<= 1;
   const int SG = kRedNT / EP;
   float u_prev = 0.f;
   if (M.gram && tid < a * r) u_prev = __ldg(M.Uprev + tid);
   {
-    const int e = tid & (EP - 1), sg = tid / EP;
+    const int e = tid & (EP - 1), sg = tid >> (31 - __clz(EP));
     double acc = 0.0;
     if (e < E) {
       const float* ptr = M.Pp + (M.gram ? 0 : (int64_t)row0 * r) + e;
       const int64_t stride = M.gram ? (int64_t)a * a : (int64_t)a * r;
-#pragma unroll 16
+#pragma unroll 8
       for (int s = sg; s < M.nsplit; s += SG) acc += (double)__ldcg(ptr + s * stride);
     }
     part[tid] = acc;
@@ -630,7 +647,8 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
     if (tid < a * r) Us[tid] = u_prev;
     __syncthreads();
     if (tid < a * r) {
-      const int k = tid / r, j = tid % r;
+      int k, j;
+      dr.divmod(tid, k, j);
       double v = 0.0;
       for (int k2 = 0; k2 < a; ++k2) v = fma(Gm[k * a + k2], (double)Us[k2 * r + j], v);
       M.Pred[tid] = v;
@@ -640,18 +658,38 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
     double v = 0.0;
     for (int sg = 0; sg < SG; ++sg) v += part[sg * EP + tid];
     M.Pred[(int64_t)row0 * r + tid] = v;
-    Ps[tid / r][tid % r] = v;
+    int k, j;
+    dr.divmod(tid, k, j);
+    Ps[k][j] = v;
   }
   __syncthreads();
   if (tid < r * r) {
-    const int i = tid / r, j = tid % r;
+    int i, j;
+    dr.divmod(tid, i, j);
     double g = 0.0;
     if (j >= i) {
-#pragma unroll
+#pragma unroll 4
       for (int rl = 0; rl < RPC; ++rl) g = fma(Ps[rl][i], Ps[rl][j], g);
     }
     M.Gp[((int64_t)c * r + i) * r + j] = g;
   }
+}
+
+// <<<>>> with the programmatic-stream-serialization attribute
+template <typename Arg>
+static cudaError_t launch_dependent(void (*kernel)(Arg), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    const Arg& arg) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, arg);
 }
 
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st) {
@@ -660,8 +698,7 @@ cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cuda
     bytes += 4.0 * p.m[m].nsplit * p.m[m].a * (p.m[m].gram ? p.m[m].a : p.m[m].r) + 8.0 * p.m[m].a * p.m[m].r;
   ProfScope prof(ASI_K_QR, st, bytes);
   dim3 grid((unsigned)max_chunks, (unsigned)nd);
-  k_sm_reduce<<<grid, kRedNT, 0, st>>>(p);
-  return cudaGetLastError();
+  return launch_dependent(k_sm_reduce, grid, dim3(kRedNT), 0, st, p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -702,6 +739,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   float* T3s = Ysm + R * R * HW;        // [R R][R][S]
   stage_tile_begin<TX>(reinterpret_cast<const TX*>(p.act) + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ,
                        &s_bar);
+  pdl_wait();                           // P_m and the Gram shares come from the reduction kernel
   // ---- the factor row this thread will solve for: [U1: B rows][U2: CC rows][U3: S][U4: S]
   const int nrows = B + CC + 2 * S;     // <= kNT (checked when the plan picks this kernel)
   int rm = 0, rk = 0, rr = 0;
@@ -735,32 +773,34 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   }
   __syncthreads();
   if ((warp & 3) == 0) {
+    // right-looking Cholesky G = R^T R on one warp; lane owns entries e0 = lane and e1 = lane + 32
     const int m = warp >> 2, r = p.r[m];
-    for (int e = lane; e < r * r; e += 32)
-      Gs[m][e / r][e % r] = ((Gq[m][0][e] + Gq[m][1][e]) + Gq[m][2][e]) + Gq[m][3][e];
+    const int e0 = lane, e1 = lane + 32;
+    const int i0 = e0 / r, k0 = e0 - i0 * r, i1 = e1 / r, k1 = e1 - i1 * r;
+    const bool in0 = e0 < r * r, in1 = e1 < r * r;
+    if (in0) Gs[m][i0][k0] = ((Gq[m][0][e0] + Gq[m][1][e0]) + Gq[m][2][e0]) + Gq[m][3][e0];
+    if (in1) Gs[m][i1][k1] = ((Gq[m][0][e1] + Gq[m][1][e1]) + Gq[m][2][e1]) + Gq[m][3][e1];
     __syncwarp();
     double trace = 0.0;
     for (int i = 0; i < r; ++i) trace += Gs[m][i][i];
     const double floor_d = 1e-12 * trace;
     for (int j = 0; j < r; ++j) {
-      if (lane == 0) {
-        double d = Gs[m][j][j];
-        if (!(d > floor_d)) {
-          if (blockIdx.x == 0) atomicMax(p.status, (int)ASI_ERR_RANK_DEFICIENT);
-          d = (floor_d > 0.0) ? floor_d : 1.0;
-        }
-        const double rjj = sqrt(d);
-        Gs[m][j][j] = rjj;
-        Dinv[m][j] = 1.0 / rjj;
+      double d = Gs[m][j][j];
+      if (!(d > floor_d)) {
+        if (blockIdx.x == 0 && lane == 0) atomicMax(p.status, (int)ASI_ERR_RANK_DEFICIENT);
+        d = (floor_d > 0.0) ? floor_d : 1.0;
+      }
+      const double inv = rsqrt(d);
+      __syncwarp();
+      if (lane == j) {
+        Gs[m][j][j] = d * inv;
+        Dinv[m][j] = inv;
+      } else if (lane > j && lane < r) {
+        Gs[m][j][lane] *= inv;
       }
       __syncwarp();
-      const double inv = Dinv[m][j];
-      if (lane > j && lane < r) Gs[m][j][lane] *= inv;
-      __syncwarp();
-      for (int e = lane; e < r * r; e += 32) {
-        const int i = e / r, k = e % r;
-        if (i > j && k >= i) Gs[m][i][k] -= Gs[m][j][i] * Gs[m][j][k];
-      }
+      if (in0 && i0 > j && k0 >= i0) Gs[m][i0][k0] -= Gs[m][j][i0] * Gs[m][j][k0];
+      if (in1 && i1 > j && k1 >= i1) Gs[m][i1][k1] -= Gs[m][j][i1] * Gs[m][j][k1];
       __syncwarp();
     }
   }
@@ -792,9 +832,11 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   project_batch<R>(Xs, PJ, U1s, B, J, part, Ws, tid, kNT, 0);
   // Y[(i,j)][hw] = sum_cl U2[cl][j] W[cl*HW + hw][i]
   const int r12 = r1 * r2;
+  const FDiv d_r2(r2), d_r3(r3), d_r4(r4);
   for (int idx = tid; idx < r12 * HW; idx += kNT) {
     const int hw = idx % HW, ij = idx / HW;
-    const int i = ij / r2, j = ij - i * r2;
+    int i, j;
+    d_r2.divmod(ij, i, j);
     float s = 0.f;
 #pragma unroll
     for (int cl = 0; cl < CC; ++cl) s = fmaf(U2s[cl * R + j], Ws[(cl * HW + hw) * R + i], s);
@@ -803,7 +845,9 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __syncthreads();
   // T3[(i,j)][k][w] = sum_h Y[(i,j)][h,w] U3[h][k]
   for (int idx = tid; idx < r12 * r3 * S; idx += kNT) {
-    const int w = idx % S, k = (idx / S) % r3, ij = idx / (S * r3);
+    const int w = idx % S;
+    int ij, k;
+    d_r3.divmod(idx / S, ij, k);
     float s = 0.f;
 #pragma unroll
     for (int h = 0; h < S; ++h) s = fmaf(Ysm[ij * HW + h * S + w], U3s[h * R + k], s);
@@ -813,7 +857,9 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   // T[(i,j)][k][l] = sum_w T3[(i,j)][k][w] U4[w][l]
   const int ce = r12 * r3 * r4;
   for (int idx = tid; idx < ce; idx += kNT) {
-    const int l = idx % r4, k = (idx / r4) % r3, ij = idx / (r4 * r3);
+    int t34, l, ij, k;
+    d_r4.divmod(idx, t34, l);
+    d_r3.divmod(t34, ij, k);
     float s = 0.f;
 #pragma unroll
     for (int w = 0; w < S; ++w) s = fmaf(T3s[(ij * R + k) * S + w], U4s[w * R + l], s);
@@ -825,16 +871,26 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // the last CTA sums the tiles in index order: thread (idx, h) takes the tiles == h (mod nh)
+  // the last CTA sums the tiles in index order: thread (idx, h) takes the tiles == h (mod nh), 32
+  // loads in flight at a time
   const int nh = (ce <= kNT / 4) ? 4 : (ce <= kNT / 2) ? 2 : 1;
   const int per = kNT / nh;
   float* fold = part;                   // [nh][ce] (nh > 1 only)
   for (int idx0 = 0; idx0 < ce; idx0 += per) {
-    const int idx = idx0 + (tid % per), h = tid / per;
+    const int idx = idx0 + (tid & (per - 1)), h = tid >> (31 - __clz(per));
     float s = 0.f;
     if (idx < ce) {
-#pragma unroll 32
-      for (int t = h; t < p.n_tiles; t += nh) s += __ldcg(p.Tp + (int64_t)t * ce + idx);
+      const float* src = p.Tp + idx;
+      for (int t0 = h; t0 < p.n_tiles; t0 += 32 * nh) {
+        float v[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          const int t = t0 + k * nh;
+          v[k] = (t < p.n_tiles) ? __ldcg(src + (int64_t)t * ce) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < 32; ++k) s += v[k];
+      }
       if (nh == 1) p.core[idx] = s;
       else fold[h * ce + idx] = s;
     }
@@ -857,17 +913,18 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
 //   Z1 = dY x_1 U1^T on the CTA's channels;
 //   Z4[c',j,kh,kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p];  dW = Z4 x_2 U2.
 // ---------------------------------------------------------------------------------------------
-template <int R, int KK>
+template <int R>
 __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const float* __restrict__ Z4s,
                                                   const float* __restrict__ U2s, int c0) {
   // thread -> fixed kernel tap t = tid mod kk; it walks the input channels c = tid / kk + k * (nthr / kk)
-  const int kk = (KK > 0) ? KK : p.kh * p.kw;
+  const int kk = p.kh * p.kw;
   const int r2 = p.r[1];
   const int cg = p.C / p.groups, og = p.Cout / p.groups;
   const int cstep = kNT / kk, nthr = cstep * kk;
   const int tid = threadIdx.x;
   if (tid >= nthr) return;
   const int t = tid % kk, cfirst = tid / kk;
+#pragma unroll 1
   for (int cl = 0; cl < p.cpb; ++cl) {
     const int co = c0 + cl;
     const int g = co / og;
@@ -914,43 +971,52 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   float* U3s = Ss + r1 * r2 * r3 * r4;               // [H][r3]
   float* U4s = U3s + H * r3;                         // [W][r4]
   float* Tm = U4s + W * r4;                          // [r1 r2][H][r4]
-  float* Z3s = Tm + r1 * r2 * H * r4;                // [r1 r2][H][W]
-  float* Z4s = Z3s + r1 * r2 * HW;                   // [cpb][r2][kk]
+  const int Hp = H + 2 * p.ph, Wp = W + 2 * p.pw;    // Z3 is kept zero-padded: term 4 needs no bounds logic
+  float* Z3s = Tm + r1 * r2 * H * r4;                // [r1 r2][Hp][Wp]
+  float* Z4s = Z3s + r1 * r2 * Hp * Wp;              // [cpb][r2][kk]
   float* red = Z4s + n_out;                          // [r1][cpb r2 kk]
 
   const TX* dY = reinterpret_cast<const TX*>(p.dY) + (int64_t)c0 * HoWo;
   const int64_t sstride = (int64_t)p.Cout * HoWo;
   const bool bulk = std::is_same<TX, float>::value && p.bulk;
-  if (bulk) {
-    stage_rows(&s_bar, reinterpret_cast<char*>(Ys), reinterpret_cast<const char*>(dY), p.B, (uint32_t)J * 4u,
-               sstride * 4, (uint32_t)PJ * 4u);
-  } else {
-    for (int idx = tid; idx < p.B * J; idx += kNT) {
-      const int b = idx / J, j = idx - b * J;
-      Ys[b * PJ + j] = to_f(dY[b * sstride + j]);
-    }
-  }
   {
     const FacDesc fd[5] = {{p.core, Ss, 1, r1 * r2 * r3 * r4, r1 * r2 * r3 * r4},
                            {p.U + p.u_off[2], U3s, H, r3, r3},
                            {p.U + p.u_off[3], U4s, W, r4, r4},
                            {p.U + p.u_off[0], U1s, p.B, r1, R},
                            {p.U + p.u_off[1], U2s, p.C, r2, R}};
-    load_factors<5>(fd);
+    fac_issue<5>(fd);
+    if (bulk) {
+      stage_rows(&s_bar, reinterpret_cast<char*>(Ys), reinterpret_cast<const char*>(dY), p.B, (uint32_t)J * 4u,
+                 sstride * 4, (uint32_t)PJ * 4u);
+    } else {
+      for (int idx = tid; idx < p.B * J; idx += kNT) {
+        const int b = idx / J, j = idx - b * J;
+        Ys[b * PJ + j] = to_f(dY[b * sstride + j]);
+      }
+    }
+    fac_wait();
   }
   __syncthreads();
   // terms 2-3: Tm[ij][h][l] = sum_k S[ij][k][l] U3[h][k];  Z3[ij][h][w] = sum_l Tm[ij][h][l] U4[w][l]
+  const FDiv d_r4(r4), d_H(H), d_Wp(Wp), d_Hp(Hp), d_nout(n_out), d_kk(kk), d_r2(r2), d_kw(p.kw);
   for (int idx = tid; idx < r1 * r2 * H * r4; idx += kNT) {
-    const int l = idx % r4, h = (idx / r4) % H, ij = idx / (r4 * H);
+    int t0, l, ij, h;
+    d_r4.divmod(idx, t0, l);
+    d_H.divmod(t0, ij, h);
     float s = 0.f;
     for (int k = 0; k < r3; ++k) s = fmaf(Ss[(ij * r3 + k) * r4 + l], U3s[h * r3 + k], s);
     Tm[idx] = s;
   }
   __syncthreads();
-  for (int idx = tid; idx < r1 * r2 * HW; idx += kNT) {
-    const int w = idx % W, h = (idx / W) % H, ij = idx / HW;
+  for (int idx = tid; idx < r1 * r2 * Hp * Wp; idx += kNT) {
+    int t0, wp, ij, hp;
+    d_Wp.divmod(idx, t0, wp);
+    d_Hp.divmod(t0, ij, hp);
+    const int h = hp - p.ph, w = wp - p.pw;
     float s = 0.f;
-    for (int l = 0; l < r4; ++l) s = fmaf(Tm[(ij * H + h) * r4 + l], U4s[w * r4 + l], s);
+    if (h >= 0 && h < H && w >= 0 && w < W)
+      for (int l = 0; l < r4; ++l) s = fmaf(Tm[(ij * H + h) * r4 + l], U4s[w * r4 + l], s);
     Z3s[idx] = s;
   }
   if (bulk) {
@@ -960,24 +1026,23 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   }
   // term 1: Z1[j,:] = sum_b dY[b, c0*HoWo + j] U1[b,:]
   project_batch<R>(Ys, PJ, U1s, p.B, J, part, Z1s, tid, kNT, 0);
-  // term 4: thread (o, i): output o = (cl, j, kh, kw), pseudo-sample i, over the (h', w') that fall
-  // inside the map; the r1 partial sums meet in order
+  // term 4: thread (o, i): output o = (cl, j, kh, kw), pseudo-sample i.  Lanes of a warp share (cl, i)
+  // and differ in (j, kh, kw): the Z1 operand is a broadcast, the Z3 operands are a few words apart.
+  // The r1 partial sums meet in order.
   for (int it = tid; it < n_out * r1; it += kNT) {
-    const int o = it % n_out, i = it / n_out;
-    const int cl = o / (r2 * kk), j = (o / kk) % r2, tt = o % kk, ky = tt / p.kw, kx = tt % p.kw;
-    // h = ho*sh + ky - ph in [0, H)  <=>  ho in [ho_lo, ho_hi)
-    int ho_lo = (p.ph - ky + p.sh - 1) / p.sh, ho_hi = (H - 1 + p.ph - ky) / p.sh + 1;
-    int wo_lo = (p.pw - kx + p.sw - 1) / p.sw, wo_hi = (W - 1 + p.pw - kx) / p.sw + 1;
-    if (p.ph - ky < 0) ho_lo = 0;
-    if (p.pw - kx < 0) wo_lo = 0;
-    if (ho_hi > p.Ho) ho_hi = p.Ho;
-    if (wo_hi > p.Wo) wo_hi = p.Wo;
+    int i, o, t0, tt, cl, j, ky, kx;
+    d_nout.divmod(it, i, o);
+    d_kk.divmod(o, t0, tt);
+    d_r2.divmod(t0, cl, j);
+    d_kw.divmod(tt, ky, kx);
+    const float* z1 = Z1s + cl * HoWo * R + i;
+    const float* z3 = Z3s + ((i * r2 + j) * Hp + ky) * Wp + kx;
     float acc = 0.f;
-    for (int ho = ho_lo; ho < ho_hi; ++ho) {
-      const float* z1 = Z1s + (cl * HoWo + ho * p.Wo) * R + i;
-      const float* z3 = Z3s + ((i * r2 + j) * H + ho * p.sh + ky - p.ph) * W + kx - p.pw;
+    for (int ho = 0; ho < p.Ho; ++ho) {
+      const float* z1r = z1 + ho * p.Wo * R;
+      const float* z3r = z3 + ho * p.sh * Wp;
 #pragma unroll 7
-      for (int wo = wo_lo; wo < wo_hi; ++wo) acc = fmaf(z1[wo * R], z3[wo * p.sw], acc);
+      for (int wo = 0; wo < p.Wo; ++wo) acc = fmaf(z1r[wo * R], z3r[wo * p.sw], acc);
     }
     red[i * n_out + o] = acc;
   }
@@ -989,9 +1054,7 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   }
   __syncthreads();
   // term 5: dW[c0+cl, c, t] = sum_j Z4[cl][j][t] U2[(g cg + c), j]
-  if (kk == 9) wgrad_expand_rows<R, 9>(p, Z4s, U2s, c0);
-  else if (kk == 1) wgrad_expand_rows<R, 1>(p, Z4s, U2s, c0);
-  else wgrad_expand_rows<R, 0>(p, Z4s, U2s, c0);
+  wgrad_expand_rows<R>(p, Z4s, U2s, c0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1030,7 +1093,8 @@ size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   const int NH = batch_groups(kNT, J);
   size_t n = (size_t)p.B * pitch4(J) + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
              (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
-             (size_t)r1 * r2 * p.H * r4 + (size_t)r1 * r2 * HW + n_out + (size_t)r1 * n_out;
+             (size_t)r1 * r2 * p.H * r4 + (size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + n_out +
+             (size_t)r1 * n_out;
   return 4 * n + 64;
 }
 
@@ -1056,8 +1120,7 @@ static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
   static bool attr_done = false;
   cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &attr_done);
   if (e != cudaSuccess) return e;
-  k_sm_core<S, R, TX><<<p.n_tiles, kNT, sm_core_smem(S, R, p.B), st>>>(p);
-  return cudaGetLastError();
+  return launch_dependent(k_sm_core<S, R, TX>, dim3(p.n_tiles), dim3(kNT), sm_core_smem(S, R, p.B), st, p);
 }
 
 template <int R, typename TX>
