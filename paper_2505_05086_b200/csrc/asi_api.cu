@@ -24,6 +24,7 @@ void set_mode_views(asi_plan* pl) {
   }
 }
 
+// dynamic shared memory a fused kernel may ask for: 227 KB per CTA minus up to ~17 KB of static arrays
 constexpr size_t kSmemLimit = 208 * 1024;
 
 // Which fused kernels cover this layer (decided once, at plan creation).
@@ -99,10 +100,10 @@ void layout_compress(asi_plan* pl) {
     pl->nchunk[m] = (int)((v.a + qr_rows - 1) / qr_rows);
     pl->off_Pp[m] = off;
     size_t pp_elems = (size_t)ns * v.a * v.r;
-    if (pl->fast_compress && pl->fast_S == 7 && m >= 2) pp_elems = std::max(pp_elems, (size_t)ns * v.a * v.a);
+    if (pl->fast_compress && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) pp_elems = std::max(pp_elems, (size_t)ns * v.a * v.a);
     off = align_up(off + pp_elems * 4, 256);
     pl->off_Pred[m] = off;
-    off = align_up(off + (size_t)v.a * v.r * 8, 256);
+    off = align_up(off + (size_t)v.a * std::max<int64_t>(v.r, (pl->fast_compress && m >= 2) ? v.a : 0) * 8, 256);
     pl->off_Gp[m] = off;
     off = align_up(off + (size_t)pl->nchunk[m] * v.r * v.r * 8, 256);
   }
@@ -178,7 +179,7 @@ thread_local char g_cuda_err[256] = "";
   } while (0)
 
 // U_m^{new} = Orthogonalize(P_m) for all modes given the split partials.
-// gram_U_prev != nullptr: the partials of modes 3 and 4 of a 7x7 map are Gram matrices A_m A_m^T
+// gram_U_prev != nullptr: the partials of modes 3 and 4 of a 7x7 or 14x14 map are Gram matrices A_m A_m^T
 // (written by the fused first pass) and P_m = G_m U_m^prev is formed during the reduction.
 asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const float* gram_U_prev,
                                cudaStream_t st) {
@@ -195,9 +196,10 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
       ra.m[m].r = pl->r[m];
       ra.m[m].nsplit = pl->nsplit[m];
       ra.m[m].nchunk = pl->nchunk[m];
-      if (gram_U_prev && pl->fast_S == 7 && m >= 2) {
+      if (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) {
         ra.m[m].gram = 1;
-        ra.m[m].Uprev = gram_U_prev + pl->u_off[m];
+        ra.m[m].nchunk = (int)((pl->dims[m] * pl->dims[m] + 24) / 25);   // ~25 Gram elements per CTA
+        max_chunks = std::max(max_chunks, ra.m[m].nchunk);
       }
     }
     ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
@@ -229,6 +231,7 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     SmCoreArgs c;
     c.act = act;
     c.U_new = U_new;
+    c.U_prev = gram_U_prev;
     c.Tp = reinterpret_cast<float*>(w + pl->off_T[0]);
     c.core = core;
     c.status = reinterpret_cast<int*>(w);
@@ -237,6 +240,7 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
       c.Pred[m] = reinterpret_cast<const double*>(w + pl->off_Pred[m]);
       c.Gp[m] = reinterpret_cast<const double*>(w + pl->off_Gp[m]);
       c.nchunk[m] = pl->nchunk[m];
+      c.gram[m] = (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) ? 1 : 0;
       c.u_off[m] = pl->u_off[m];
       c.r[m] = pl->r[m];
     }

@@ -81,9 +81,8 @@ struct SmPass1Args {
 // G_m = P_m^T P_m.
 struct SmReduceMode {
   const float* Pp;     // [nsplit][a][r], or [nsplit][a][a] Gram matrices A_m A_m^T when gram != 0
-  double* Pred;        // [a][r]
+  double* Pred;        // [a][r], or [a][a] (the summed Gram matrix) when gram != 0
   double* Gp;          // [nchunk][r][r]
-  const float* Uprev;  // [a][r] previous factor (gram modes only)
   int a, r, nsplit, nchunk, gram;
 };
 struct SmReduceArgs {
@@ -95,6 +94,8 @@ struct SmCoreArgs {
   const double* Pred[ASI_MAX_MODES];
   const double* Gp[ASI_MAX_MODES];
   int nchunk[ASI_MAX_MODES];
+  int gram[ASI_MAX_MODES];      // != 0: Pred[m] holds G_m = A_m A_m^T (a x a), P_m = G_m U_prev is formed here
+  const float* U_prev;
   float* U_new;
   float* Tp;                    // [n_tiles][core_elems] per-tile partial cores
   float* core;

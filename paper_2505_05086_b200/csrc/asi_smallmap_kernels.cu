@@ -30,9 +30,6 @@ namespace {
 constexpr int kNT = 512;             // threads per CTA of the tile kernels
 constexpr int kNG = 256;             // threads of one half (warp-specialised phases)
 constexpr int kRedNT = 256;          // threads per CTA of the partial-reduction kernel
-// Opt-in dynamic shared memory ceiling of the fused kernels (plans only pick them when the
-// layer needs less); leaves room for static shared memory under the 227 KB per-CTA limit.
-constexpr int kMaxDynSmem = 214 * 1024;
 
 __host__ __device__ constexpr int pitch4(int J) {      // >= J, multiple of 4, == 4 (mod 32)
   int p = (J + 3) / 4 * 4;
@@ -384,6 +381,7 @@ template <int S, int R, typename TX>
 __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
   constexpr bool kBulk = std::is_same<TX, float>::value;
   constexpr bool kGram = (S == 7);                   // modes 3, 4 as Gram matrices A_m A_m^T (7 x 7)
+  constexpr bool kGram14 = (S == 14);                // ... as 14 x 14 Gram matrices in four 7 x 7 blocks
   constexpr int HW = S * S;
   constexpr int CC = (S == 7) ? 4 : 1;               // channels per role-B tile
   constexpr int J = CC * HW;                         // contiguous elements per sample in a tile
@@ -489,8 +487,78 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
         }
         bar_sync(2, kNG);
       }
+    } else if constexpr (kGram14) {
+      // ---- half 1, S = 14: G_m = A_m A_m^T for m = 3, 4 in 7 x 7 blocks.  With a = rows 0..6 and
+      // b = rows 7..13 of a fiber, warp role 0 accumulates the upper triangle of a a^T, role 1 that of
+      // b b^T, role 2 the block a b[0..3]^T and role 3 the block a b[4..6]^T (<= 28 accumulators each).
+      // A unit is a quarter of a plane (fibers == part mod 4), so the lanes of a warp hit 32 banks.
+      constexpr int NACC = 32;
+      const int role = wg & 3;
+      const int u0 = (wg >> 2) * 32 + lane;
+      const int nunits = B * CC * 4;
+#pragma unroll 1
+      for (int mode = 2; mode <= 3; ++mode) {
+        const int es = (mode == 2) ? S : 1;
+        const int cs = (mode == 2) ? 1 : S;
+        float* Gm = p.Pp[mode] + (int64_t)tile * HW;
+        float acc[NACC];
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
+        for (int un = u0; un < nunits; un += 64) {
+          const int pl = un >> 2, part_ = un & 3;
+          const float* base = Xs + (pl / CC) * PJ + (pl % CC) * HW;
+#pragma unroll 1
+          for (int col = part_; col < S; col += 4) {
+            const float* colp = base + col * cs;
+            if (role < 2) {
+              const float* q = colp + role * 7 * es;
+              float x[7];
+#pragma unroll
+              for (int k = 0; k < 7; ++k) x[k] = q[k * es];
+#pragma unroll
+              for (int k = 0; k < 7; ++k)
+#pragma unroll
+                for (int k2 = k; k2 < 7; ++k2) acc[tri_index(7, k, k2)] = fmaf(x[k], x[k2], acc[tri_index(7, k, k2)]);
+            } else if (role == 2) {
+              float xa[7], xb[4];
+#pragma unroll
+              for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) xb[k] = colp[(7 + k) * es];
+#pragma unroll
+              for (int k = 0; k < 7; ++k)
+#pragma unroll
+                for (int k2 = 0; k2 < 4; ++k2) acc[k * 4 + k2] = fmaf(xa[k], xb[k2], acc[k * 4 + k2]);
+            } else {
+              float xa[7], xb[3];
+#pragma unroll
+              for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
+#pragma unroll
+              for (int k = 0; k < 3; ++k) xb[k] = colp[(11 + k) * es];
+#pragma unroll
+              for (int k = 0; k < 7; ++k)
+#pragma unroll
+                for (int k2 = 0; k2 < 3; ++k2) acc[k * 3 + k2] = fmaf(xa[k], xb[k2], acc[k * 3 + k2]);
+            }
+          }
+        }
+        warp_reduce_scatter<NACC>(acc, lane);
+        red[wg * 32 + scatter_base<NACC>(lane)] = acc[0];
+        bar_sync(2, kNG);
+        for (int o = t; o < HW; o += kNG) {
+          const int k = o / S, k2 = o % S;
+          const int lo = k < k2 ? k : k2, hi = k < k2 ? k2 : k;
+          int rl, e;
+          if (hi < 7) { rl = 0; e = tri_index(7, lo, hi); }
+          else if (lo >= 7) { rl = 1; e = tri_index(7, lo - 7, hi - 7); }
+          else if (hi < 11) { rl = 2; e = lo * 4 + (hi - 7); }
+          else { rl = 3; e = lo * 3 + (hi - 11); }
+          Gm[o] = red[rl * 32 + e] + red[(rl + 4) * 32 + e];
+        }
+        bar_sync(2, kNG);
+      }
     } else {
-      // ---- half 1, S > 7: P_m = A_m (A_m^T U_m^prev) for m = 3, 4.  A unit is a quarter of a plane
+      // ---- half 1, other sizes: P_m = A_m (A_m^T U_m^prev) for m = 3, 4.  A unit is a quarter of a plane
       // (columns == part mod 4); unit -> thread so that the 32 lanes of a warp touch 32 different
       // banks.  Each thread owns 2 columns of the factor; warp w serves column pair w mod JH.
       constexpr int TPP = 4, JT = 2, JH = R / JT, NACC = 32;
@@ -566,11 +634,19 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
       const int n4 = C * HW / 4;
       for (int idx = tid; idx < n4; idx += kNT) *reinterpret_cast<float4*>(Xs + 4 * idx) = ld4<TX>(Xb + 4 * idx);
     } else {
+      // rows of a quarter are only 4-byte aligned: one 4-byte asynchronous copy per element (fp32),
+      // all of a thread's copies in flight at once
       const int n = C * HWC;
-#pragma unroll 4
+#pragma unroll 1
       for (int idx = tid; idx < n; idx += kNT) {
         const int c = idx / HWC, hw = idx - c * HWC;
-        Xs[c * PC + hw] = to_f(Xb[(int64_t)c * HW + hw]);
+        if constexpr (kBulk) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(Xs + c * PC + hw)),
+                       "l"(Xb + (int64_t)c * HW + hw)
+                       : "memory");
+        } else {
+          Xs[c * PC + hw] = to_f(Xb[(int64_t)c * HW + hw]);
+        }
       }
     }
     fac_wait();
@@ -599,9 +675,9 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
 // ---------------------------------------------------------------------------------------------
 // k_sm_reduce: CTA (c, m) sums rows [16 c, 16 c + 16) of the per-tile partials of P_m in fp64 in a
 // fixed order (thread (e, sg) takes the partials s == sg (mod SG); the SG sums meet in shared memory
-// in index order), stores them in fp64 and adds its share of G_m = P_m^T P_m.  A mode whose
-// partials are Gram matrices A_m A_m^T (a <= 16, one CTA) is summed the same way and multiplied by
-// U_m^prev first.
+// in index order), stores them in fp64 and adds its share of P_m^T P_m.  A mode whose partials are
+// Gram matrices A_m A_m^T (a <= 16) is summed the same way, a slice of the a x a elements per CTA,
+// and left in fp64 for the core kernel.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   constexpr int RM = 8, RPC = kRedRows;
@@ -612,24 +688,24 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   pdl_wait();                                      // the partials come from the previous kernel
   __shared__ double part[kRedNT];
   __shared__ double Ps[RPC][RM];
-  __shared__ double Gm[RPC * RPC];
   const int tid = threadIdx.x;
   const int r = M.r, a = M.a;
+  // a Gram mode: CTA c sums elements [c*per, c*per + per) of G_m = A_m A_m^T over the tiles;
+  // otherwise rows [16 c, 16 c + 16) of P_m
+  const int per = M.gram ? (a * a + M.nchunk - 1) / M.nchunk : 0;
+  const int first = M.gram ? c * per : c * RPC * r;
   const int row0 = c * RPC;
   const int nrow = (a - row0 < RPC) ? (a - row0) : RPC;
-  const int E = M.gram ? a * a : nrow * r;         // <= 256
-  const FDiv dr(r);
+  const int E = M.gram ? ((a * a - first < per) ? a * a - first : per) : nrow * r;   // <= 128
+  const int64_t stride = M.gram ? (int64_t)a * a : (int64_t)a * r;
   int EP = 32;
   while (EP < E) EP <<= 1;
   const int SG = kRedNT / EP;
-  float u_prev = 0.f;
-  if (M.gram && tid < a * r) u_prev = __ldg(M.Uprev + tid);
   {
     const int e = tid & (EP - 1), sg = tid >> (31 - __clz(EP));
     double acc = 0.0;
     if (e < E) {
-      const float* ptr = M.Pp + (M.gram ? 0 : (int64_t)row0 * r) + e;
-      const int64_t stride = M.gram ? (int64_t)a * a : (int64_t)a * r;
+      const float* ptr = M.Pp + first + e;
 #pragma unroll 8
       for (int s = sg; s < M.nsplit; s += SG) acc += (double)__ldcg(ptr + s * stride);
     }
@@ -637,33 +713,21 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   }
   for (int idx = tid; idx < RPC * RM; idx += kRedNT) Ps[idx / RM][idx % RM] = 0.0;
   __syncthreads();
-  if (M.gram) {
-    __shared__ float Us[RPC * RM];
-    if (tid < E) {
-      double v = 0.0;
-      for (int sg = 0; sg < SG; ++sg) v += part[sg * EP + tid];
-      Gm[tid] = v;
-    }
-    if (tid < a * r) Us[tid] = u_prev;
-    __syncthreads();
-    if (tid < a * r) {
-      int k, j;
-      dr.divmod(tid, k, j);
-      double v = 0.0;
-      for (int k2 = 0; k2 < a; ++k2) v = fma(Gm[k * a + k2], (double)Us[k2 * r + j], v);
-      M.Pred[tid] = v;
-      Ps[k][j] = v;
-    }
-  } else if (tid < E) {
+  if (tid < E) {
     double v = 0.0;
     for (int sg = 0; sg < SG; ++sg) v += part[sg * EP + tid];
-    M.Pred[(int64_t)row0 * r + tid] = v;
-    int k, j;
-    dr.divmod(tid, k, j);
-    Ps[k][j] = v;
+    M.Pred[first + tid] = v;                       // P_m rows, or G_m elements for a Gram mode
+    if (!M.gram) {
+      const FDiv dr(r);
+      int k, j;
+      dr.divmod(tid, k, j);
+      Ps[k][j] = v;
+    }
   }
+  if (M.gram) return;                              // the core kernel forms P_m = G_m U_m^prev itself
   __syncthreads();
   if (tid < r * r) {
+    const FDiv dr(r);
     int i, j;
     dr.divmod(tid, i, j);
     double g = 0.0;
@@ -725,6 +789,8 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __shared__ double Gq[4][4][R * R];
   __shared__ double Gs[4][R][R + 1];
   __shared__ double Dinv[4][R];
+  __shared__ double Gfull[2][S * S];    // A_m A_m^T of a Gram mode (m = 3, 4)
+  __shared__ double Pm[2][S][R];        // and its P_m = G_m U_m^prev
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, C = p.C, tile = blockIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
@@ -754,21 +820,28 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     else if (tid < B + CC + S) { rm = 2; rk = tid - B - CC; rdst = U3s + rk * R; rowner = tile == 0; }
     else { rm = 3; rk = tid - B - CC - S; rdst = U4s + rk * R; rowner = tile == 0; }
     rr = p.r[rm];
-    const double* src = p.Pred[rm] + (int64_t)rk * rr;
+    if (!p.gram[rm]) {
+      const double* src = p.Pred[rm] + (int64_t)rk * rr;
 #pragma unroll
-    for (int j = 0; j < R; ++j)
-      if (j < rr) prow[j] = __ldcg(src + j);
+      for (int j = 0; j < R; ++j)
+        if (j < rr) prow[j] = __ldcg(src + j);
+    }
   }
   // ---- Gram shares: warp 4m + q sums the chunks == q (mod 4) of mode m
   {
     const int m = warp >> 2, q = warp & 3, r = p.r[m];
-    const double* Gp = p.Gp[m];
-    const int nch = p.nchunk[m];
-    for (int e = lane; e < r * r; e += 32) {
-      double g = 0.0;
+    if (!p.gram[m]) {
+      const double* Gp = p.Gp[m];
+      const int nch = p.nchunk[m];
+      for (int e = lane; e < r * r; e += 32) {
+        double g = 0.0;
 #pragma unroll 8
-      for (int cc = q; cc < nch; cc += 4) g += __ldcg(Gp + (int64_t)cc * r * r + e);
-      Gq[m][q][e] = g;
+        for (int cc = q; cc < nch; cc += 4) g += __ldcg(Gp + (int64_t)cc * r * r + e);
+        Gq[m][q][e] = g;
+      }
+    } else {
+      // Gram mode (m = 2, 3; a = S): the four warps fetch G_m = A_m A_m^T
+      for (int e = q * 32 + lane; e < S * S; e += 128) Gfull[m - 2][e] = __ldcg(p.Pred[m] + e);
     }
   }
   __syncthreads();
@@ -778,8 +851,30 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     const int e0 = lane, e1 = lane + 32;
     const int i0 = e0 / r, k0 = e0 - i0 * r, i1 = e1 / r, k1 = e1 - i1 * r;
     const bool in0 = e0 < r * r, in1 = e1 < r * r;
-    if (in0) Gs[m][i0][k0] = ((Gq[m][0][e0] + Gq[m][1][e0]) + Gq[m][2][e0]) + Gq[m][3][e0];
-    if (in1) Gs[m][i1][k1] = ((Gq[m][0][e1] + Gq[m][1][e1]) + Gq[m][2][e1]) + Gq[m][3][e1];
+    if (!p.gram[m]) {
+      if (in0) Gs[m][i0][k0] = ((Gq[m][0][e0] + Gq[m][1][e0]) + Gq[m][2][e0]) + Gq[m][3][e0];
+      if (in1) Gs[m][i1][k1] = ((Gq[m][0][e1] + Gq[m][1][e1]) + Gq[m][2][e1]) + Gq[m][3][e1];
+    } else {
+      // P_m = G_m U_m^prev (Algorithm 1: A_m (A_m^T U)), then its Gram matrix
+      const float* Up = p.U_prev + p.u_off[m];
+      for (int e = lane; e < S * r; e += 32) {
+        const int k = e / r, j = e - k * r;
+        double v = 0.0;
+        for (int k2 = 0; k2 < S; ++k2) v = fma(Gfull[m - 2][k * S + k2], (double)__ldg(Up + k2 * r + j), v);
+        Pm[m - 2][k][j] = v;
+      }
+      __syncwarp();
+      if (in0 && k0 >= i0) {
+        double g = 0.0;
+        for (int k = 0; k < S; ++k) g = fma(Pm[m - 2][k][i0], Pm[m - 2][k][k0], g);
+        Gs[m][i0][k0] = g;
+      }
+      if (in1 && k1 >= i1) {
+        double g = 0.0;
+        for (int k = 0; k < S; ++k) g = fma(Pm[m - 2][k][i1], Pm[m - 2][k][k1], g);
+        Gs[m][i1][k1] = g;
+      }
+    }
     __syncwarp();
     double trace = 0.0;
     for (int i = 0; i < r; ++i) trace += Gs[m][i][i];
@@ -812,7 +907,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     for (int j = 0; j < R; ++j) {
       float out = 0.f;
       if (j < rr) {
-        double v = prow[j];
+        double v = p.gram[rm] ? Pm[rm - 2][rk][j] : prow[j];
 #pragma unroll
         for (int i = 0; i < R; ++i)
           if (i < j) v -= q[i] * Gs[rm][i][j];
@@ -1098,37 +1193,41 @@ size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   return 4 * n + 64;
 }
 
+// Raises the kernel's dynamic shared memory limit to `need` bytes when it is below that.
 template <typename K>
-static cudaError_t opt_in_smem(K kernel, bool* done) {
-  if (*done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
-  if (e == cudaSuccess) *done = true;
+static cudaError_t opt_in_smem(K kernel, size_t* granted, size_t need) {
+  if (need <= *granted) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+  if (e == cudaSuccess) *granted = need;
   return e;
 }
 
 template <int S, int R, typename TX>
 static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
-  static bool attr_done = false;
-  cudaError_t e = opt_in_smem(k_sm_pass1<S, R, TX>, &attr_done);
+  static size_t granted = 48 * 1024;
+  const size_t smem = sm_pass1_smem(S, R, p.B, p.C);
+  cudaError_t e = opt_in_smem(k_sm_pass1<S, R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
-  k_sm_pass1<S, R, TX><<<p.n_tiles_b + sm_pass1_role_c_ctas(S, p.B), kNT, sm_pass1_smem(S, R, p.B, p.C), st>>>(p);
+  k_sm_pass1<S, R, TX><<<p.n_tiles_b + sm_pass1_role_c_ctas(S, p.B), kNT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 template <int S, int R, typename TX>
 static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
-  static bool attr_done = false;
-  cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &attr_done);
+  static size_t granted = 48 * 1024;
+  const size_t smem = sm_core_smem(S, R, p.B);
+  cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
-  return launch_dependent(k_sm_core<S, R, TX>, dim3(p.n_tiles), dim3(kNT), sm_core_smem(S, R, p.B), st, p);
+  return launch_dependent(k_sm_core<S, R, TX>, dim3(p.n_tiles), dim3(kNT), smem, st, p);
 }
 
 template <int R, typename TX>
 static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
-  static bool attr_done = false;
-  cudaError_t e = opt_in_smem(k_sm_wgrad<R, TX>, &attr_done);
+  static size_t granted = 48 * 1024;
+  const size_t smem = sm_wgrad_smem(p, R);
+  cudaError_t e = opt_in_smem(k_sm_wgrad<R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
-  k_sm_wgrad<R, TX><<<p.Cout / p.cpb, kNT, sm_wgrad_smem(p, R), st>>>(p);
+  k_sm_wgrad<R, TX><<<p.Cout / p.cpb, kNT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -1149,7 +1248,7 @@ static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st) {
   const size_t eb = bf16 ? 2 : 4;
   double bytes = (double)p.B * p.C * S * S * eb;
-  const double m34 = (S == 7) ? 2.0 * S * S : (double)S * (p.r[2] + p.r[3]);
+  const double m34 = (S == 7 || S == 14) ? 2.0 * S * S : (double)S * (p.r[2] + p.r[3]);
   bytes += 4.0 * ((double)p.n_tiles_b * (p.B * p.r[0] + m34) + (double)p.B * p.C * p.r[1]);
   ProfScope prof(ASI_K_SM_PASS1, st, bytes);
   ASI_DISPATCH_SR(launch_pass1_t, p);
