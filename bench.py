@@ -230,6 +230,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2505_05086_b200 import binding
+    from paper_2505_05086_b200.replicas import job_throughput
     from paper_2505_05086_b200.runner import LayerRunner
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -333,11 +334,7 @@ def run_ours(args):
     for r in runners:
         if not r.ok():
             raise SystemExit("device status: the timed loop reported an error (rank-deficient iterate or timeout)")
-    t = torch.tensor([ms], device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
-    value = world * nl * args.steps / (ms * 1e-3)
+    value, ms = job_throughput(nl * args.steps, ms, dev)       # max over ranks, whole-job aggregate
 
     if args.timed_only:
         if rank == 0:
@@ -387,13 +384,10 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-    t = torch.tensor([ms_e2e], device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_e2e = float(t.item())
+    e2e_value, ms_e2e = job_throughput(nl * k_e2e, ms_e2e, dev)
     h2d = sum((r.plan.info.act_elems + r.plan.info.dy_elems) * elem + r.plan.info.u_elems * 4 for r in runners)
     d2h = sum((r.plan.info.u_elems + r.plan.info.core_elems + r.plan.info.dw_elems) * 4 for r in runners)
-    e2e = {"value": world * nl * k_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h), "steps": k_e2e}
 
     # ---- per-kernel timing for the roofline ---------------------------------------------------
