@@ -65,7 +65,7 @@ void choose_kernels(asi_plan* pl) {
     for (int m = 0; m < 4; ++m) a.r[m] = pl->r[m];
     a.B = (int)B; a.C = (int)C; a.Cout = Cout; a.H = (int)H; a.W = (int)W;
     a.Ho = (int)pl->Ho; a.Wo = (int)pl->Wo; a.kh = pl->d.kh; a.kw = pl->d.kw; a.cpb = cpb;
-    a.ph = pl->d.pad_h; a.pw = pl->d.pad_w;
+    a.ph = pl->d.pad_h; a.pw = pl->d.pad_w; a.groups = pl->d.groups;
     if (sm_wgrad_smem(a, R) <= kSmemLimit) {
       pl->fast_wgrad = true;
       pl->cpb = cpb;
@@ -127,7 +127,9 @@ void layout_compress(asi_plan* pl) {
   }
   if (pl->fast_compress) {
     tmax[0] = (int64_t)pl->n_tiles_b * pl->core_elems;          // per-tile partial cores
-    tmax[1] = 0;
+    pl->fold_gs = 8;                                             // tiles per group of the two-level sum
+    while ((pl->n_tiles_b + pl->fold_gs - 1) / pl->fold_gs > 192) pl->fold_gs *= 2;
+    tmax[1] = (int64_t)((pl->n_tiles_b + pl->fold_gs - 1) / pl->fold_gs) * pl->core_elems;
   }
   for (int t = 0; t < 2; ++t) {
     pl->off_T[t] = off;
@@ -236,6 +238,9 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     c.core = core;
     c.status = reinterpret_cast<int*>(w);
     c.counter = reinterpret_cast<int*>(w) + 16;
+    c.gcount = reinterpret_cast<int*>(w) + 64;
+    c.gs = pl->fold_gs;
+    c.Tg = reinterpret_cast<float*>(w + pl->off_T[1]);
     for (int m = 0; m < 4; ++m) {
       c.Pred[m] = reinterpret_cast<const double*>(w + pl->off_Pred[m]);
       c.Gp[m] = reinterpret_cast<const double*>(w + pl->off_Gp[m]);
@@ -565,6 +570,8 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
     g.bulk = pl->wgrad_bulk ? 1 : 0;
     if (g.bulk && (reinterpret_cast<uintptr_t>(dY) & 15u)) return ASI_ERR_INVALID_ARG;
     g.status = reinterpret_cast<int*>(w);
+    g.bulk_store = (((pl->dims[1] / pl->d.groups) * pl->d.kh * pl->d.kw) % 4 == 0 &&
+                    (reinterpret_cast<uintptr_t>(dW) & 15u) == 0) ? 1 : 0;
     ASI_CUDA(launch_sm_wgrad(g, pl->fast_R, pl->bf16, st));
     return ASI_OK;
   }

@@ -18,7 +18,7 @@ struct ModeView {
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr int kStatusBytes = 256;
+constexpr int kStatusBytes = 1024;    // status word (int 0), completion counters (ints 16..255)
 constexpr int kQRRows = 64;          // rows per CTA in the orthonormalisation kernels
 constexpr int kExpandKC = 32;        // rows of P per CTA in the expand kernel
 
@@ -72,7 +72,7 @@ struct SmPass1Args {
   const void* act;
   const float* U_prev;
   float* Pp[ASI_MAX_MODES];     // per-mode partials [nsplit][a_m][r_m]
-  int* status;                  // status word (int 0) and completion counters (ints 16..23) of the workspace
+  int* status;                  // status word (int 0) and completion counters (ints 16..255) of the workspace
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
   int B, C, n_tiles_b;
@@ -98,9 +98,12 @@ struct SmCoreArgs {
   const float* U_prev;
   float* U_new;
   float* Tp;                    // [n_tiles][core_elems] per-tile partial cores
+  float* Tg;                    // [ceil(n_tiles / gs)][core_elems] per-group partial cores
   float* core;
   int* status;
   int* counter;                 // zero on entry, zero again on exit
+  int* gcount;                  // one counter per group of gs tiles, same convention
+  int gs;
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
   int B, C, n_tiles;
@@ -116,6 +119,7 @@ struct SmWgradArgs {
   int B, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups, cpb;
   int pj;                       // row pitch (floats) of the staged dY tile
   int bulk;                     // 1: rows staged by the bulk-copy engine (fp32, 16-byte aligned rows)
+  int bulk_store;               // 1: dW row blocks leave through the bulk-copy engine (16-byte sized and aligned)
 };
 size_t sm_pass1_smem(int S, int R, int B, int C);
 int sm_pass1_role_c_ctas(int S, int B);
@@ -187,5 +191,5 @@ struct asi_plan {
 
   // fused small-map path
   bool fast_compress, fast_wgrad, wgrad_bulk;
-  int fast_S, fast_R, n_tiles_b, cpb;
+  int fast_S, fast_R, n_tiles_b, cpb, fold_gs;
 };

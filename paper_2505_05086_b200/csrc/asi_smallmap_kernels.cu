@@ -150,50 +150,26 @@ __device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char
   }
 }
 
-// Small read-only arrays a CTA keeps in shared memory (factors, the core).  fac_issue() starts one
-// 4-byte asynchronous copy (cp.async) per element -- a compact loop, no registers held -- and
+// Small read-only arrays a CTA keeps in shared memory (factors, the core).  fac_issue_*() start one
+// 4-byte asynchronous copy (cp.async) per element -- short loops, no registers held -- and
 // fac_wait() waits for this thread's copies; a __syncthreads() after it publishes them.  Whatever a
 // kernel does in between overlaps the single round trip, and these small loads are ahead of its bulk
-// traffic in the memory system.  Element (k, j) of array i, j < r_dst:
-// dst[k*r_dst + j] = j < r_src ? src[k*r_src + j] : 0.
-struct FacDesc {
-  const float* src;
-  float* dst;
-  int rows, r_src, r_dst;
-};
-template <int NF>
-__device__ __forceinline__ void fac_issue(const FacDesc (&f)[NF]) {
-  int total = 0;
-#pragma unroll
-  for (int i = 0; i < NF; ++i) total += f[i].rows * f[i].r_dst;
+// traffic in the memory system.
+__device__ __forceinline__ void cp_async4(float* dst, const float* src, int bytes /* 4, or 0 to store 0.f */) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(bytes) : "memory");
+}
+// dst[k*RD + j] = j < r ? src[k*r + j] : 0 for k < rows: a factor [rows x r] padded to RD columns
+template <int RD>
+__device__ __forceinline__ void fac_issue_padded(const float* __restrict__ src, float* dst, int rows, int r) {
 #pragma unroll 1
-  for (int idx0 = threadIdx.x; idx0 < total; idx0 += kNT) {
-    int idx = idx0;
-    const float* src = f[0].src;
-    float* dst = f[0].dst;
-    int fill = 0;
-#pragma unroll
-    for (int i = 0; i < NF; ++i) {
-      const int n = f[i].rows * f[i].r_dst;
-      if (idx >= 0 && idx < n) {
-        dst = f[i].dst + idx;
-        if (f[i].r_src == f[i].r_dst) {
-          src = f[i].src + idx;
-          fill = 4;
-        } else {
-          const int row = idx / f[i].r_dst, j = idx - row * f[i].r_dst;
-          if (j < f[i].r_src) {
-            src = f[i].src + row * f[i].r_src + j;
-            fill = 4;
-          }
-        }
-        idx = -1;
-      } else if (idx >= 0) {
-        idx -= n;
-      }
-    }
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(fill) : "memory");
+  for (int idx = threadIdx.x; idx < rows * RD; idx += kNT) {
+    const int k = idx / RD, j = idx % RD;
+    cp_async4(dst + idx, src + (j < r ? k * r + j : 0), j < r ? 4 : 0);
   }
+}
+__device__ __forceinline__ void fac_issue_flat(const float* __restrict__ src, float* dst, int n) {
+#pragma unroll 1
+  for (int idx = threadIdx.x; idx < n; idx += kNT) cp_async4(dst + idx, src + idx, 4);
 }
 __device__ __forceinline__ void fac_wait() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
@@ -394,7 +370,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
   const TX* __restrict__ A = reinterpret_cast<const TX*>(p.act);
   const int B = p.B, C = p.C;
 
-  if (blockIdx.x == 0 && tid < 9) p.status[tid == 0 ? 0 : 15 + tid] = 0;   // status word, counters 16..23
+  if (blockIdx.x == 0 && tid < 241) p.status[tid == 0 ? 0 : 15 + tid] = 0;  // status word, counters 16..255
   pdl_launch_dependents();
 
   constexpr int kNQ = (S == 7) ? 1 : 4;             // role-C CTAs per sample
@@ -408,14 +384,13 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* V1s = U4s + S * R;                        // [J][R]
     float* part = V1s + J * R;                       // [NH1][J][R] (NH1 > 1 only)
     float* red = part + (NH1 > 1 ? NH1 : 0) * J * R; // [8][32]
-    {
-      const FacDesc fd[3] = {{p.U_prev + p.u_off[0], U1s, B, p.r[0], R},
-                             {p.U_prev + p.u_off[2], U3s, S, p.r[2], R},
-                             {p.U_prev + p.u_off[3], U4s, S, p.r[3], R}};
-      fac_issue<3>(fd);
-      stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
-      fac_wait();
+    fac_issue_padded<R>(p.U_prev + p.u_off[0], U1s, B, p.r[0]);
+    if constexpr (!kGram && !kGram14) {
+      fac_issue_padded<R>(p.U_prev + p.u_off[2], U3s, S, p.r[2]);
+      fac_issue_padded<R>(p.U_prev + p.u_off[3], U4s, S, p.r[3]);
     }
+    stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
+    fac_wait();
     if constexpr (kBulk) {
       if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
     } else {
@@ -626,8 +601,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* V2s = U2s + C * R;                        // [HWC][R]
     float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
     const TX* Xb = A + (int64_t)b * C * HW + q * HWC;
-    const FacDesc fdc[1] = {{p.U_prev + p.u_off[1], U2s, C, p.r[1], R}};
-    fac_issue<1>(fdc);
+    fac_issue_padded<R>(p.U_prev + p.u_off[1], U2s, C, p.r[1]);
     if constexpr (kBulkC) {
       stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
     } else if constexpr (NQ == 1) {
@@ -772,7 +746,7 @@ cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cuda
 //     one thread per needed factor row solves u = p R_m^{-1} -- all of U_1, the tile's own rows of
 //     U_2, all of U_3 and U_4 -- and the owners write them to U_new;
 //   W[i][c,h,w] = sum_b U1[b,i] X[b][c,h,w];  Y[i,j][h,w] = sum_c U2[c,j] W[i][c,h,w];
-//   T[i,j,k,l] = Y x_3 U3^T x_4 U4^T  -> per-tile partial core; the last CTA sums the tiles in order.
+//   T[i,j,k,l] = Y x_3 U3^T x_4 U4^T  -> per-tile partial core, summed in two ordered levels.
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
 __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
@@ -791,6 +765,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __shared__ double Dinv[4][R];
   __shared__ double Gfull[2][S * S];    // A_m A_m^T of a Gram mode (m = 3, 4)
   __shared__ double Pm[2][S][R];        // and its P_m = G_m U_m^prev
+  __shared__ float Ups[2][S * R];       // U_m^prev of a Gram mode
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, C = p.C, tile = blockIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
@@ -842,6 +817,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     } else {
       // Gram mode (m = 2, 3; a = S): the four warps fetch G_m = A_m A_m^T
       for (int e = q * 32 + lane; e < S * S; e += 128) Gfull[m - 2][e] = __ldcg(p.Pred[m] + e);
+      for (int e = q * 32 + lane; e < S * r; e += 128) Ups[m - 2][e] = __ldg(p.U_prev + p.u_off[m] + e);
     }
   }
   __syncthreads();
@@ -856,11 +832,10 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
       if (in1) Gs[m][i1][k1] = ((Gq[m][0][e1] + Gq[m][1][e1]) + Gq[m][2][e1]) + Gq[m][3][e1];
     } else {
       // P_m = G_m U_m^prev (Algorithm 1: A_m (A_m^T U)), then its Gram matrix
-      const float* Up = p.U_prev + p.u_off[m];
       for (int e = lane; e < S * r; e += 32) {
         const int k = e / r, j = e - k * r;
         double v = 0.0;
-        for (int k2 = 0; k2 < S; ++k2) v = fma(Gfull[m - 2][k * S + k2], (double)__ldg(Up + k2 * r + j), v);
+        for (int k2 = 0; k2 < S; ++k2) v = fma(Gfull[m - 2][k * S + k2], (double)Ups[m - 2][k2 * r + j], v);
         Pm[m - 2][k][j] = v;
       }
       __syncwarp();
@@ -960,43 +935,49 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     for (int w = 0; w < S; ++w) s = fmaf(T3s[(ij * R + k) * S + w], U4s[w * R + l], s);
     p.Tp[(int64_t)tile * ce + idx] = s;
   }
+  // Two-level sum of the per-tile cores, both levels in index order: the last CTA of every group of
+  // p.gs tiles sums that group, the last group to finish sums the groups.
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(p.counter, 1) == (int)gridDim.x - 1);
+  const int grp = tile / p.gs, gfirst = grp * p.gs;
+  const int gsize = (p.n_tiles - gfirst < p.gs) ? p.n_tiles - gfirst : p.gs;
+  const int ngroups = (p.n_tiles + p.gs - 1) / p.gs;
+  if (tid == 0) s_last = (atomicAdd(p.gcount + grp, 1) == gsize - 1);
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // the last CTA sums the tiles in index order: thread (idx, h) takes the tiles == h (mod nh), 32
-  // loads in flight at a time
-  const int nh = (ce <= kNT / 4) ? 4 : (ce <= kNT / 2) ? 2 : 1;
-  const int per = kNT / nh;
-  float* fold = part;                   // [nh][ce] (nh > 1 only)
-  for (int idx0 = 0; idx0 < ce; idx0 += per) {
-    const int idx = idx0 + (tid & (per - 1)), h = tid >> (31 - __clz(per));
+  for (int idx = tid; idx < ce; idx += kNT) {
+    const float* src = p.Tp + (int64_t)gfirst * ce + idx;
     float s = 0.f;
-    if (idx < ce) {
-      const float* src = p.Tp + idx;
-      for (int t0 = h; t0 < p.n_tiles; t0 += 32 * nh) {
-        float v[32];
+    for (int t0 = 0; t0 < gsize; t0 += 8) {
+      float v[8];
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          const int t = t0 + k * nh;
-          v[k] = (t < p.n_tiles) ? __ldcg(src + (int64_t)t * ce) : 0.f;
-        }
+      for (int k = 0; k < 8; ++k) v[k] = (t0 + k < gsize) ? __ldcg(src + (int64_t)(t0 + k) * ce) : 0.f;
 #pragma unroll
-        for (int k = 0; k < 32; ++k) s += v[k];
-      }
-      if (nh == 1) p.core[idx] = s;
-      else fold[h * ce + idx] = s;
+      for (int k = 0; k < 8; ++k) s += v[k];
     }
+    p.Tg[(int64_t)grp * ce + idx] = s;
   }
-  if (nh > 1) {
-    __syncthreads();
-    for (int idx = tid; idx < ce; idx += kNT) {
-      float s = 0.f;
-      for (int h = 0; h < nh; ++h) s += fold[h * ce + idx];
-      p.core[idx] = s;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    p.gcount[grp] = 0;
+    s_last = (atomicAdd(p.counter, 1) == ngroups - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int idx = tid; idx < ce; idx += kNT) {
+    const float* src = p.Tg + idx;
+    float s = 0.f;
+    for (int g0 = 0; g0 < ngroups; g0 += 16) {
+      float v[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v[k] = (g0 + k < ngroups) ? __ldcg(src + (int64_t)(g0 + k) * ce) : 0.f;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) s += v[k];
     }
+    p.core[idx] = s;
   }
   if (tid == 0) *p.counter = 0;
 }
@@ -1008,40 +989,67 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
 //   Z1 = dY x_1 U1^T on the CTA's channels;
 //   Z4[c',j,kh,kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p];  dW = Z4 x_2 U2.
 // ---------------------------------------------------------------------------------------------
+// Term 5: dW[c0+cl, c, t] = sum_j Z4[cl][t][j] U2[(g cg + c), j].  A thread owns input channel c (its
+// row of U2 stays in registers) and writes the kk taps of every output channel into a staging row
+// block in shared memory; the block [cg x kk] then leaves for global memory in one piece -- by the
+// bulk-copy engine (cp.async.bulk shared -> global) when it is 16-byte sized and aligned, two blocks in
+// flight, else by coalesced stores.
 template <int R>
 __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const float* __restrict__ Z4s,
-                                                  const float* __restrict__ U2s, int c0) {
-  // thread -> fixed kernel tap t = tid mod kk; it walks the input channels c = tid / kk + k * (nthr / kk)
+                                                  const float* __restrict__ U2s, float* stage, int c0) {
   const int kk = p.kh * p.kw;
-  const int r2 = p.r[1];
   const int cg = p.C / p.groups, og = p.Cout / p.groups;
-  const int cstep = kNT / kk, nthr = cstep * kk;
   const int tid = threadIdx.x;
-  if (tid >= nthr) return;
-  const int t = tid % kk, cfirst = tid / kk;
+  const int nblk = cg * kk;
 #pragma unroll 1
   for (int cl = 0; cl < p.cpb; ++cl) {
     const int co = c0 + cl;
     const int g = co / og;
-    float* dw = p.dW + (int64_t)co * cg * kk + t;
+    float* dw = p.dW + (int64_t)co * nblk;
     const float* u2 = U2s + (int64_t)g * cg * R;
-    float z[R];
-#pragma unroll
-    for (int j = 0; j < R; ++j) z[j] = (j < r2) ? Z4s[(cl * r2 + j) * kk + t] : 0.f;
-#pragma unroll 4
-    for (int c = cfirst; c < cg; c += cstep) {
-      float v = 0.f;
+    float* buf = stage + (cl & 1) * nblk;
+    if (p.bulk_store && cl >= 2) {
+      if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      __syncthreads();
+    }
+#pragma unroll 1
+    for (int c = tid; c < cg; c += kNT) {
+      float u[R];
 #pragma unroll
       for (int j = 0; j < R; j += 4) {
-        const float4 u = *reinterpret_cast<const float4*>(u2 + c * R + j);
-        v = fmaf(z[j], u.x, v);
-        v = fmaf(z[j + 1], u.y, v);
-        v = fmaf(z[j + 2], u.z, v);
-        v = fmaf(z[j + 3], u.w, v);
+        const float4 v = *reinterpret_cast<const float4*>(u2 + c * R + j);
+        u[j] = v.x; u[j + 1] = v.y; u[j + 2] = v.z; u[j + 3] = v.w;
       }
-      dw[(int64_t)c * kk] = v;
+      const float* z = Z4s + cl * kk * R;
+#pragma unroll 3
+      for (int t = 0; t < kk; ++t) {
+        float v = 0.f;
+#pragma unroll
+        for (int j = 0; j < R; j += 4) {
+          const float4 zz = *reinterpret_cast<const float4*>(z + t * R + j);
+          v = fmaf(zz.x, u[j], v);
+          v = fmaf(zz.y, u[j + 1], v);
+          v = fmaf(zz.z, u[j + 2], v);
+          v = fmaf(zz.w, u[j + 3], v);
+        }
+        buf[c * kk + t] = v;
+      }
+    }
+    if (p.bulk_store) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncthreads();
+      if (tid == 0) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dw), "r"(smem_u32(buf)),
+                     "r"((uint32_t)nblk * 4u)
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+    } else {
+      __syncthreads();
+      for (int idx = tid; idx < nblk; idx += kNT) dw[idx] = buf[idx];
     }
   }
+  if (p.bulk_store && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
 template <int R, typename TX>
@@ -1057,8 +1065,9 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   const int NH = batch_groups(kNT, J);
   const int c0 = blockIdx.x * p.cpb;
   const int n_out = p.cpb * r2 * kk;
+  const int n_stage = 2 * (p.C / p.groups) * kk;     // two staging blocks of term 5 reuse the tile's space
   float* Ys = smem;                                  // [B][PJ]
-  float* U1s = Ys + p.B * PJ;                        // [B][R]
+  float* U1s = Ys + ((p.B * PJ > n_stage ? p.B * PJ : n_stage) + 3) / 4 * 4;   // [B][R]
   float* U2s = U1s + p.B * R;                        // [C][R]
   float* Z1s = U2s + p.C * R;                        // [J][R]
   float* part = Z1s + J * R;                         // [NH][J][R] (NH > 1 only)
@@ -1068,19 +1077,18 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   float* Tm = U4s + W * r4;                          // [r1 r2][H][r4]
   const int Hp = H + 2 * p.ph, Wp = W + 2 * p.pw;    // Z3 is kept zero-padded: term 4 needs no bounds logic
   float* Z3s = Tm + r1 * r2 * H * r4;                // [r1 r2][Hp][Wp]
-  float* Z4s = Z3s + r1 * r2 * Hp * Wp;              // [cpb][r2][kk]
-  float* red = Z4s + n_out;                          // [r1][cpb r2 kk]
+  float* Z4s = smem + ((Z3s + r1 * r2 * Hp * Wp) - smem + 3) / 4 * 4;   // [cpb][kk][R], 16-byte aligned (rank index fastest, zero-padded)
+  float* red = Z4s + p.cpb * kk * R;                 // [G4][cpb][r2 kk]
 
   const TX* dY = reinterpret_cast<const TX*>(p.dY) + (int64_t)c0 * HoWo;
   const int64_t sstride = (int64_t)p.Cout * HoWo;
   const bool bulk = std::is_same<TX, float>::value && p.bulk;
   {
-    const FacDesc fd[5] = {{p.core, Ss, 1, r1 * r2 * r3 * r4, r1 * r2 * r3 * r4},
-                           {p.U + p.u_off[2], U3s, H, r3, r3},
-                           {p.U + p.u_off[3], U4s, W, r4, r4},
-                           {p.U + p.u_off[0], U1s, p.B, r1, R},
-                           {p.U + p.u_off[1], U2s, p.C, r2, R}};
-    fac_issue<5>(fd);
+    fac_issue_flat(p.core, Ss, r1 * r2 * r3 * r4);
+    fac_issue_flat(p.U + p.u_off[2], U3s, H * r3);
+    fac_issue_flat(p.U + p.u_off[3], U4s, W * r4);
+    fac_issue_padded<R>(p.U + p.u_off[0], U1s, p.B, r1);
+    fac_issue_padded<R>(p.U + p.u_off[1], U2s, p.C, r2);
     if (bulk) {
       stage_rows(&s_bar, reinterpret_cast<char*>(Ys), reinterpret_cast<const char*>(dY), p.B, (uint32_t)J * 4u,
                  sstride * 4, (uint32_t)PJ * 4u);
@@ -1094,7 +1102,7 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   }
   __syncthreads();
   // terms 2-3: Tm[ij][h][l] = sum_k S[ij][k][l] U3[h][k];  Z3[ij][h][w] = sum_l Tm[ij][h][l] U4[w][l]
-  const FDiv d_r4(r4), d_H(H), d_Wp(Wp), d_Hp(Hp), d_nout(n_out), d_kk(kk), d_r2(r2), d_kw(p.kw);
+  const FDiv d_r4(r4), d_H(H), d_Wp(Wp), d_Hp(Hp), d_kk(kk), d_kw(p.kw);
   for (int idx = tid; idx < r1 * r2 * H * r4; idx += kNT) {
     int t0, l, ij, h;
     d_r4.divmod(idx, t0, l);
@@ -1121,35 +1129,49 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   }
   // term 1: Z1[j,:] = sum_b dY[b, c0*HoWo + j] U1[b,:]
   project_batch<R>(Ys, PJ, U1s, p.B, J, part, Z1s, tid, kNT, 0);
-  // term 4: thread (o, i): output o = (cl, j, kh, kw), pseudo-sample i.  Lanes of a warp share (cl, i)
-  // and differ in (j, kh, kw): the Z1 operand is a broadcast, the Z3 operands are a few words apart.
-  // The r1 partial sums meet in order.
-  for (int it = tid; it < n_out * r1; it += kNT) {
-    int i, o, t0, tt, cl, j, ky, kx;
-    d_nout.divmod(it, i, o);
-    d_kk.divmod(o, t0, tt);
-    d_r2.divmod(t0, cl, j);
+  // term 4: thread (n, g): outputs n = (j, kh, kw) of all cpb channels and every G-th pair (i, h') of
+  // the reduction; one Z3 operand feeds cpb FMAs.  The G partial sums meet in order.
+  const int N4 = r2 * kk;
+  int G4 = (N4 <= kNT) ? kNT / N4 : 1;
+  if (G4 > r1 * p.Ho) G4 = r1 * p.Ho;
+  const FDiv d_Ho(p.Ho), d_N4(N4);
+  for (int it = tid; it < N4 * G4; it += kNT) {
+    int g, n, j, tt, ky, kx;
+    d_N4.divmod(it, g, n);
+    d_kk.divmod(n, j, tt);
     d_kw.divmod(tt, ky, kx);
-    const float* z1 = Z1s + cl * HoWo * R + i;
-    const float* z3 = Z3s + ((i * r2 + j) * Hp + ky) * Wp + kx;
-    float acc = 0.f;
-    for (int ho = 0; ho < p.Ho; ++ho) {
-      const float* z1r = z1 + ho * p.Wo * R;
-      const float* z3r = z3 + ho * p.sh * Wp;
+    const float* z3 = Z3s + (j * Hp + ky) * Wp + kx;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int q = g; q < r1 * p.Ho; q += G4) {
+      int i, ho;
+      d_Ho.divmod(q, i, ho);
+      const float* z1r = Z1s + ho * p.Wo * R + i;
+      const float* z3r = z3 + (i * r2 * Hp + ho * p.sh) * Wp;
 #pragma unroll 7
-      for (int wo = 0; wo < p.Wo; ++wo) acc = fmaf(z1r[wo * R], z3r[wo * p.sw], acc);
+      for (int wo = 0; wo < p.Wo; ++wo) {
+        const float b = z3r[wo * p.sw];
+#pragma unroll
+        for (int cl = 0; cl < 4; ++cl)
+          if (cl < p.cpb) acc[cl] = fmaf(z1r[(cl * HoWo + wo) * R], b, acc[cl]);
+      }
     }
-    red[i * n_out + o] = acc;
+#pragma unroll
+    for (int cl = 0; cl < 4; ++cl)
+      if (cl < p.cpb) red[(g * p.cpb + cl) * N4 + n] = acc[cl];
   }
   __syncthreads();
-  for (int o = tid; o < n_out; o += kNT) {
+  for (int o = tid; o < p.cpb * kk * R; o += kNT) {
+    const int j = o % R, ct = o / R;                 // ct = cl*kk + t
+    int cl, tt;
+    d_kk.divmod(ct, cl, tt);
     float v = 0.f;
-    for (int i = 0; i < r1; ++i) v += red[i * n_out + o];
+    if (j < r2)
+      for (int g = 0; g < G4; ++g) v += red[(g * p.cpb + cl) * N4 + j * kk + tt];
     Z4s[o] = v;
   }
   __syncthreads();
   // term 5: dW[c0+cl, c, t] = sum_j Z4[cl][j][t] U2[(g cg + c), j]
-  wgrad_expand_rows<R>(p, Z4s, U2s, c0);
+  wgrad_expand_rows<R>(p, Z4s, U2s, Ys, c0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1183,13 +1205,14 @@ int sm_wgrad_pitch(int J) { return pitch4(J); }
 
 size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
-  const int HW = p.H * p.W, J = p.cpb * p.Ho * p.Wo, kk = p.kh * p.kw;
-  const int n_out = p.cpb * r2 * kk;
+  const int J = p.cpb * p.Ho * p.Wo, kk = p.kh * p.kw;
+  const int N4 = r2 * kk;
   const int NH = batch_groups(kNT, J);
-  size_t n = (size_t)p.B * pitch4(J) + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
+  const size_t tile = (size_t)p.B * pitch4(J), stage = (size_t)2 * (p.C / p.groups) * kk;
+  size_t n = ((tile > stage ? tile : stage) + 3) / 4 * 4 + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
              (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
-             (size_t)r1 * r2 * p.H * r4 + (size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + n_out +
-             (size_t)r1 * n_out;
+             (size_t)r1 * r2 * p.H * r4 + ((size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + 3) / 4 * 4 +
+             (size_t)p.cpb * kk * R + (size_t)p.cpb * (N4 > kNT ? N4 : kNT);
   return 4 * n + 64;
 }
 
