@@ -78,6 +78,21 @@ void choose_kernels(asi_plan* pl) {
 // and the completion counter of the core kernel (byte 64).
 void layout_compress(asi_plan* pl) {
   size_t off = kStatusBytes;
+  int rmax = 0;
+  for (int m = 0; m < pl->nd; ++m) rmax = std::max(rmax, pl->r[m]);
+  pl->small_rank = !pl->fast_compress && rmax <= 8 && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY);
+  for (int m = 0; m < ASI_MAX_MODES; ++m) {
+    pl->fiber[m] = false;
+    pl->fiber_grid[m] = 0;
+  }
+  if (pl->small_rank)
+    for (int m = 0; m < pl->nd; ++m) {
+      const ModeView& v = pl->mv[m];
+      if (v.a <= 128 && fiber_smem((int)v.a) <= kSmemLimit) {
+        pl->fiber[m] = true;
+        pl->fiber_grid[m] = (int)std::min<int64_t>(fiber_tiles(v.O, v.a, v.I), 296);
+      }
+    }
   int64_t vmax = 0;
   if (!pl->fast_compress)
     for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
@@ -94,9 +109,13 @@ void layout_compress(asi_plan* pl) {
     ns = (v.Q + qps - 1) / qps;
     if (pl->fast_compress)                                               // one partial per tile
       ns = (m == 1) ? sm_pass1_role_c_ctas(pl->fast_S, (int)pl->dims[0]) : pl->n_tiles_b;
+    if (pl->fiber[m]) {                                                  // one partial per CTA of k_fiber;
+      ns = pl->fiber_grid[m];                                            // the cold-start expansion uses the
+      qps = ((v.Q + ns - 1) / ns + 63) / 64 * 64;                        // same count (empty splits write 0)
+    }
     pl->nsplit[m] = (int)ns;
     pl->q_per_split[m] = qps;
-    const int qr_rows = pl->fast_compress ? kRedRows : kQRRows;
+    const int qr_rows = (pl->fast_compress || pl->small_rank) ? kRedRows : kQRRows;
     pl->nchunk[m] = (int)((v.a + qr_rows - 1) / qr_rows);
     pl->off_Pp[m] = off;
     size_t pp_elems = (size_t)ns * v.a * v.r;
@@ -136,7 +155,11 @@ void layout_compress(asi_plan* pl) {
     off = align_up(off + (size_t)tmax[t] * 4, 256);
   }
   pl->compress_ws = off;
-  pl->launches_compress = pl->fast_compress ? 3 : 2 * pl->nd + 2 + pl->nd;
+  pl->launches_compress = 3;
+  if (!pl->fast_compress) {
+    pl->launches_compress = 2 + pl->nd;                                    // reduction/QR pair, core chain
+    for (int m = 0; m < pl->nd; ++m) pl->launches_compress += pl->fiber[m] ? 1 : 2;
+  }
 }
 
 void layout_wgrad(asi_plan* pl) {
@@ -207,6 +230,20 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
     ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
     return ASI_OK;      // the core kernel finishes the factorisation
   }
+  if (pl->small_rank) {
+    SmReduceArgs ra;
+    std::memset(&ra, 0, sizeof(ra));
+    for (int m = 0; m < pl->nd; ++m) {
+      ra.m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
+      ra.m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
+      ra.m[m].Gp = reinterpret_cast<double*>(w + pl->off_Gp[m]);
+      ra.m[m].a = (int)pl->dims[m];
+      ra.m[m].r = pl->r[m];
+      ra.m[m].nsplit = pl->nsplit[m];
+      ra.m[m].nchunk = pl->nchunk[m];
+    }
+    ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
+  }
   QRArgs qa;
   std::memset(&qa, 0, sizeof(qa));
   for (int m = 0; m < pl->nd; ++m) {
@@ -220,7 +257,8 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
     qa.m[m].nchunk = pl->nchunk[m];
   }
   qa.status = reinterpret_cast<int*>(w);
-  ASI_CUDA(launch_qr(qa, pl->nd, max_chunks, st));
+  if (pl->small_rank) ASI_CUDA(launch_qr_solve(qa, pl->nd, max_chunks, st));
+  else ASI_CUDA(launch_qr(qa, pl->nd, max_chunks, st));
   return ASI_OK;
 }
 
@@ -467,6 +505,19 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   float* V = reinterpret_cast<float*>(w + pl->off_V);
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
+    if (pl->fiber[m]) {
+      // both products of the mode in one pass; V stays on chip
+      FiberArgs f;
+      f.X = act;
+      f.U = U_prev + pl->u_off[m];
+      f.Pp = reinterpret_cast<float*>(w + pl->off_Pp[m]);
+      f.O = v.O; f.a = v.a; f.I = v.I;
+      f.n_tiles = fiber_tiles(v.O, v.a, v.I);
+      f.r = v.r;
+      f.vec4 = (!pl->bf16 && v.I % 4 == 0 && (reinterpret_cast<uintptr_t>(act) & 15u) == 0) ? 1 : 0;
+      ASI_CUDA(launch_fiber(f, pl->fiber_grid[m], pl->bf16, st));
+      continue;
+    }
     // V = A_m^T U_m^{prev}, stored [b_m x r_m]
     ModeProdArgs a;
     a.X = act;

@@ -9,6 +9,8 @@
 //   k_conv_tail: terms 4 and 5 of C_ASI (appendix "Speedup")
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "asi_internal.h"
 
 namespace asi {
@@ -196,6 +198,203 @@ cudaError_t launch_expand(const ExpandArgs& p, bool x_bf16, cudaStream_t st) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// k_fiber: P_m = A_m (A_m^T U_m) for one mode in ONE pass over the activation (Algorithm 1, both
+// products of a mode).  A tile is TQ whole fibers of the mode: a rows of TQ contiguous values when the
+// mode is not the last one, TQ contiguous fibers when it is.  Per tile, V[q,:] = sum_k X(k,q) U[k,:]
+// stays in shared memory and P[k,:] += sum_q X(k,q) V[q,:] accumulates in registers across all tiles
+// of the CTA, so V never reaches global memory and each CTA writes one partial of P.  fp32 tiles are
+// double-buffered with cp.async.  Requires a <= 128, r <= R.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFiberTQ = 64;
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) {
+  return static_cast<unsigned>(__cvta_generic_to_shared(p));
+}
+
+template <int R, typename TX>
+__global__ void __launch_bounds__(256) k_fiber(FiberArgs p) {
+  constexpr int TQ = kFiberTQ, NT = 256, KS = NT / TQ;
+  extern __shared__ __align__(16) float fsm[];
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int a = (int)p.a, r = p.r;
+  const bool last = p.I == 1;                       // fibers are contiguous
+  // logical X(k, q) of a staged tile sits at k*SK + q*SQ
+  const int PQ = TQ + 4;                            // row pitch, 16-byte aligned rows
+  const int PA = a | 1;                             // fiber pitch (odd: conflict-free fiber-per-thread reads)
+  const int SK = last ? 1 : PQ, SQ = last ? PA : 1;
+  const int tile_floats = last ? TQ * PA : a * PQ;
+  float* Xs0 = fsm;
+  float* Xs1 = fsm + ((tile_floats + 3) & ~3);
+  float* Us = Xs1 + ((tile_floats + 3) & ~3);      // [a][R]
+  float* Vp = Us + a * R;                           // [KS][TQ][R]
+  float* Vs = Vp + KS * TQ * R;                     // [TQ][R]
+  for (int idx = tid; idx < a * R; idx += NT) {
+    const int k = idx / R, j = idx % R;
+    Us[idx] = (j < r) ? p.U[k * r + j] : 0.f;
+  }
+  const TX* __restrict__ X = reinterpret_cast<const TX*>(p.X);
+  const int64_t tiles_per_o = last ? 0 : (p.I + TQ - 1) / TQ;
+
+  auto stage = [&](float* dst, int64_t t, int& n_q) {
+    if (last) {
+      const int64_t q0 = t * TQ;
+      n_q = (int)((p.O - q0 < TQ) ? (p.O - q0) : TQ);
+      const TX* src = X + q0 * a;
+      for (int idx = tid; idx < n_q * a; idx += NT) {
+        const int q = idx / a, k = idx - q * a;
+        if constexpr (sizeof(TX) == 4) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(dst + q * PA + k)), "l"(src + idx) : "memory");
+        } else {
+          dst[q * PA + k] = ld_as_float(src + idx);
+        }
+      }
+    } else {
+      const int64_t o = t / tiles_per_o, i0 = (t - o * tiles_per_o) * TQ;
+      n_q = (int)((p.I - i0 < TQ) ? (p.I - i0) : TQ);
+      const TX* src = X + o * a * p.I + i0;
+      if (sizeof(TX) == 4 && p.vec4) {
+        const int n4 = n_q >> 2;                    // I and TQ are multiples of 4 here
+        for (int idx = tid; idx < a * n4; idx += NT) {
+          const int k = idx / n4, v = idx - k * n4;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst + k * PQ + 4 * v)),
+                       "l"(src + (int64_t)k * p.I + 4 * v)
+                       : "memory");
+        }
+      } else {
+        for (int idx = tid; idx < a * n_q; idx += NT) {
+          const int k = idx / n_q, q = idx - k * n_q;
+          if constexpr (sizeof(TX) == 4) {
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(dst + k * PQ + q)),
+                         "l"(src + (int64_t)k * p.I + q)
+                         : "memory");
+          } else {
+            dst[k * PQ + q] = ld_as_float(src + (int64_t)k * p.I + q);
+          }
+        }
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  // thread roles: projection (q, ks), expansion (k, qs)
+  const int pq = tid % TQ, pks = tid / TQ;
+  int QS = 32;
+  while (QS * a > NT && QS > 1) QS >>= 1;           // largest power of two with QS * a <= 256
+  const int ek = tid / QS, eqs = tid % QS;
+  float acc2[R];
+#pragma unroll
+  for (int j = 0; j < R; ++j) acc2[j] = 0.f;
+
+  int n_cur = 0, n_next = 0;
+  int64_t t = blockIdx.x;
+  if (t < p.n_tiles) stage(Xs0, t, n_cur);
+  int buf = 0;
+  for (; t < p.n_tiles; t += gridDim.x) {
+    float* Xc = buf ? Xs1 : Xs0;
+    float* Xn = buf ? Xs0 : Xs1;
+    const int64_t tn = t + gridDim.x;
+    if (tn < p.n_tiles) {
+      stage(Xn, tn, n_next);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    // projection: V[q,:] = sum_k X(k,q) U[k,:]
+    {
+      float acc[R];
+#pragma unroll
+      for (int j = 0; j < R; ++j) acc[j] = 0.f;
+      if (pq < n_cur) {
+#pragma unroll 4
+        for (int k = pks; k < a; k += KS) {
+          const float x = Xc[k * SK + pq * SQ];
+#pragma unroll
+          for (int j = 0; j < R; j += 4) {
+            const float4 u = *reinterpret_cast<const float4*>(Us + k * R + j);
+            acc[j] = fmaf(x, u.x, acc[j]);
+            acc[j + 1] = fmaf(x, u.y, acc[j + 1]);
+            acc[j + 2] = fmaf(x, u.z, acc[j + 2]);
+            acc[j + 3] = fmaf(x, u.w, acc[j + 3]);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < R; j += 4)
+        *reinterpret_cast<float4*>(Vp + (pks * TQ + pq) * R + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+    }
+    __syncthreads();
+    for (int idx = tid; idx < TQ * R; idx += NT) {
+      float v = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) v += Vp[ks * TQ * R + idx];
+      Vs[idx] = v;
+    }
+    __syncthreads();
+    // expansion: P[k,:] += sum_q X(k,q) V[q,:]
+    if (ek < a) {
+#pragma unroll 4
+      for (int q = eqs; q < n_cur; q += QS) {
+        const float x = Xc[ek * SK + q * SQ];
+#pragma unroll
+        for (int j = 0; j < R; j += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(Vs + q * R + j);
+          acc2[j] = fmaf(x, v.x, acc2[j]);
+          acc2[j + 1] = fmaf(x, v.y, acc2[j + 1]);
+          acc2[j + 2] = fmaf(x, v.z, acc2[j + 2]);
+          acc2[j + 3] = fmaf(x, v.w, acc2[j + 3]);
+        }
+      }
+    }
+    __syncthreads();
+    n_cur = n_next;
+    buf ^= 1;
+  }
+  // the QS threads of a row meet by shuffles (fixed order), one partial of P per CTA
+#pragma unroll
+  for (int j = 0; j < R; ++j)
+    for (int off = 1; off < QS; off <<= 1) acc2[j] += __shfl_xor_sync(0xffffffffu, acc2[j], off);
+  (void)lane;
+  if (ek < a && eqs == 0) {
+    float* dst = p.Pp + ((int64_t)blockIdx.x * a + ek) * r;
+#pragma unroll
+    for (int j = 0; j < R; ++j)
+      if (j < r) dst[j] = acc2[j];
+  }
+}
+
+size_t fiber_smem(int a) {
+  const int TQ = kFiberTQ, PQ = TQ + 4, PA = a | 1;
+  const size_t tile = (size_t)std::max(TQ * PA, a * PQ);
+  return 4 * (2 * ((tile + 3) & ~(size_t)3) + (size_t)a * 8 + 5 * TQ * 8) + 64;
+}
+
+int64_t fiber_tiles(int64_t O, int64_t a, int64_t I) {
+  (void)a;
+  return I == 1 ? (O + kFiberTQ - 1) / kFiberTQ : O * ((I + kFiberTQ - 1) / kFiberTQ);
+}
+
+template <int R, typename TX>
+static cudaError_t launch_fiber_t(const FiberArgs& p, int grid, cudaStream_t st) {
+  static size_t granted = 48 * 1024;
+  const size_t smem = fiber_smem((int)p.a);
+  if (smem > granted) {
+    cudaError_t e = cudaFuncSetAttribute(k_fiber<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    granted = smem;
+  }
+  k_fiber<R, TX><<<grid, 256, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fiber(const FiberArgs& p, int grid, bool x_bf16, cudaStream_t st) {
+  ProfScope prof(ASI_K_EXPAND, st,
+                 (double)p.O * p.a * p.I * (x_bf16 ? 2 : 4) + 4.0 * ((double)p.a * p.r * (grid + 1)));
+  if (p.r <= 4) return x_bf16 ? launch_fiber_t<4, __nv_bfloat16>(p, grid, st) : launch_fiber_t<4, float>(p, grid, st);
+  return x_bf16 ? launch_fiber_t<8, __nv_bfloat16>(p, grid, st) : launch_fiber_t<8, float>(p, grid, st);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Orthogonalize.  Stage 1 (k_qr_gram): sum the column-split partials of P in fp64 in a fixed
 // order, keep P in fp64, and form this row chunk's share of G = P^T P.  Stage 2 (k_qr_solve):
 // G = R^T R by Cholesky (R upper, positive diagonal), U = P R^{-1} row by row.  That U is the
@@ -286,6 +485,12 @@ __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
       }
     }
   }
+}
+
+cudaError_t launch_qr_solve(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) {
+  dim3 grid((unsigned)max_chunks, (unsigned)nd);
+  k_qr_solve<<<grid, 256, 0, st>>>(p);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) {

@@ -44,6 +44,15 @@ struct ExpandArgs {
   int64_t q_per_split;
 };
 
+// One mode's P = A_m (A_m^T U) in a single pass (k_fiber); Pp: [grid][a][r] partials.
+struct FiberArgs {
+  const void* X;
+  const float* U;
+  float* Pp;
+  int64_t O, a, I, n_tiles;
+  int r, vec4;
+};
+
 struct QRMode {
   const float* Pp;     // [nsplit][a][r]
   double* Pred;        // [a][r]
@@ -161,6 +170,10 @@ struct ProfScope {
 cudaError_t launch_modeprod(const ModeProdArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_expand(const ExpandArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
+cudaError_t launch_qr_solve(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
+cudaError_t launch_fiber(const FiberArgs& p, int grid, bool x_bf16, cudaStream_t st);
+size_t fiber_smem(int a);
+int64_t fiber_tiles(int64_t O, int64_t a, int64_t I);
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
 
 }  // namespace asi
@@ -191,5 +204,8 @@ struct asi_plan {
 
   // fused small-map path
   bool fast_compress, fast_wgrad, wgrad_bulk;
+  bool small_rank;                 // every rank <= 8: partials are reduced by the parallel fp64 kernel
+  bool fiber[ASI_MAX_MODES];       // mode handled by the single-pass fiber kernel
+  int fiber_grid[ASI_MAX_MODES];
   int fast_S, fast_R, n_tiles_b, cpb, fold_gs;
 };
