@@ -250,3 +250,41 @@ def test_step_from_host_buffers_matches_device_path():
     np.testing.assert_array_equal(hUn.numpy(), run.U[run.cur].cpu().numpy())
     np.testing.assert_array_equal(hS.numpy(), run.core.cpu().numpy())
     np.testing.assert_array_equal(hdW.numpy(), run.dW.cpu().numpy())
+
+
+def test_cuda_graph_replay_matches_direct_launches():
+    """bench.py replays the step as a CUDA graph with one branch per layer; the replayed kernels (incl.
+    the programmatically dependent ones) must give the bits the direct launches give."""
+    cfg = get_config(1)
+    li = 1
+    L = cfg.layers[li]
+    st = make_stream(cfg, li)
+    A, dY = st.next()
+    run = make_runner(L)
+    a, d = run.to_device(A), run.to_device(dY)
+    run.set_factors(st.u_prev0())
+    run.compress(a)
+    run.wgrad(d)
+    torch.cuda.synchronize()
+    ref = (run.U[run.cur].clone(), run.core.clone(), run.dW.clone())
+    # same step again from the same previous factors, captured and replayed twice
+    run.cur = 1 - run.cur
+    run.set_factors(st.u_prev0())
+    s = torch.cuda.Stream()
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        cur = torch.cuda.current_stream()
+        side.wait_stream(cur)
+        run.compress(a, side)
+        run.wgrad(d, side)
+        cur.wait_stream(side)
+    for _ in range(2):
+        run.core.zero_()
+        run.dW.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert run.ok()
+        assert torch.equal(run.U[run.cur], ref[0])
+        assert torch.equal(run.core, ref[1])
+        assert torch.equal(run.dW, ref[2])
