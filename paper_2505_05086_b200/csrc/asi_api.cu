@@ -85,8 +85,17 @@ void layout_compress(asi_plan* pl) {
     pl->fiber[m] = false;
     pl->fiber_grid[m] = 0;
   }
+  pl->plane = false;
+  pl->plane_grid = 0;
+  if (pl->small_rank && pl->d.kind == ASI_CONV2D && pl->dims[2] == pl->dims[3] && pl->dims[2] % 4 == 0 &&
+      pl->dims[2] >= 8 && pl->dims[2] <= 64 && plane_smem((int)pl->dims[2]) <= kSmemLimit) {
+    pl->plane = true;
+    const int64_t np = 256 / pl->dims[2], planes = pl->dims[0] * pl->dims[1];
+    pl->plane_grid = (int)std::min<int64_t>((planes + np - 1) / np, 296);
+  }
   if (pl->small_rank)
     for (int m = 0; m < pl->nd; ++m) {
+      if (pl->plane && m >= 2) continue;
       const ModeView& v = pl->mv[m];
       if (v.a <= 128 && fiber_smem((int)v.a) <= kSmemLimit) {
         pl->fiber[m] = true;
@@ -109,10 +118,10 @@ void layout_compress(asi_plan* pl) {
     ns = (v.Q + qps - 1) / qps;
     if (pl->fast_compress)                                               // one partial per tile
       ns = (m == 1) ? sm_pass1_role_c_ctas(pl->fast_S, (int)pl->dims[0]) : pl->n_tiles_b;
-    if (pl->fiber[m]) {                                                  // one partial per CTA of k_fiber;
-      ns = pl->fiber_grid[m];                                            // the cold-start expansion uses the
-      qps = ((v.Q + ns - 1) / ns + 63) / 64 * 64;                        // same count (empty splits write 0)
-    }
+    if (pl->fiber[m] || (pl->plane && m >= 2)) {                         // one partial per CTA of k_fiber /
+      ns = pl->fiber[m] ? pl->fiber_grid[m] : pl->plane_grid;            // k_plane; the cold-start expansion
+      qps = ((v.Q + ns - 1) / ns + 63) / 64 * 64;                        // uses the same count (empty splits
+    }                                                                    // write 0)
     pl->nsplit[m] = (int)ns;
     pl->q_per_split[m] = qps;
     const int qr_rows = (pl->fast_compress || pl->small_rank) ? kRedRows : kQRRows;
@@ -158,7 +167,8 @@ void layout_compress(asi_plan* pl) {
   pl->launches_compress = 3;
   if (!pl->fast_compress) {
     pl->launches_compress = 2 + pl->nd;                                    // reduction/QR pair, core chain
-    for (int m = 0; m < pl->nd; ++m) pl->launches_compress += pl->fiber[m] ? 1 : 2;
+    for (int m = 0; m < pl->nd; ++m)
+      pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
   }
 }
 
@@ -503,8 +513,23 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   }
   ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
   float* V = reinterpret_cast<float*>(w + pl->off_V);
+  if (pl->plane) {
+    PlaneArgs g;
+    g.X = act;
+    g.U3 = U_prev + pl->u_off[2];
+    g.U4 = U_prev + pl->u_off[3];
+    g.Pp3 = reinterpret_cast<float*>(w + pl->off_Pp[2]);
+    g.Pp4 = reinterpret_cast<float*>(w + pl->off_Pp[3]);
+    g.n_planes = pl->dims[0] * pl->dims[1];
+    g.S = (int)pl->dims[2];
+    g.r3 = pl->r[2];
+    g.r4 = pl->r[3];
+    g.vec4 = (!pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u) == 0) ? 1 : 0;
+    ASI_CUDA(launch_plane(g, pl->plane_grid, pl->bf16, st));
+  }
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
+    if (pl->plane && m >= 2) continue;
     if (pl->fiber[m]) {
       // both products of the mode in one pass; V stays on chip
       FiberArgs f;

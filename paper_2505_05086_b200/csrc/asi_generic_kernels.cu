@@ -363,6 +363,179 @@ __global__ void __launch_bounds__(256) k_fiber(FiberArgs p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// k_plane: the two spatial modes of a conv activation in one pass.  A tile is NP = 256 / S whole
+// planes X[h][w] (S x S, S a multiple of 4); thread (plane, i) owns column w = i and row h = i:
+//   V3[w,:] = sum_h X[h][w] U3[h,:]   (column read)      V4[h,:] = sum_w X[h][w] U4[w,:]   (row read)
+//   P3[h,:] += sum_w X[h][w] V3[w,:]  (row read)         P4[w,:] += sum_h X[h][w] V4[h,:]  (column read)
+// i.e. P_m = A_m (A_m^T U_m) for m = 3, 4 (Algorithm 1).  Rows are read as float4 (conflict-free for the
+// unpadded pitch S), columns as scalars.  P3 / P4 accumulate in registers across the CTA's tiles.
+// ---------------------------------------------------------------------------------------------
+template <int R, typename TX>
+__global__ void __launch_bounds__(256) k_plane(PlaneArgs p) {
+  constexpr int NT = 256;
+  extern __shared__ __align__(16) float fsm[];
+  const int tid = threadIdx.x;
+  const int S = p.S, SS = S * S, NP = NT / S;
+  float* Xs0 = fsm;
+  float* Xs1 = Xs0 + NP * SS;
+  float* U3s = Xs1 + NP * SS;                       // [S][R]
+  float* U4s = U3s + S * R;                         // [S][R]
+  float* V3s = U4s + S * R;                         // [NP][S][R]
+  float* V4s = V3s + NP * S * R;                    // [NP][S][R]
+  for (int idx = tid; idx < S * R; idx += NT) {
+    const int k = idx / R, j = idx % R;
+    U3s[idx] = (j < p.r3) ? p.U3[k * p.r3 + j] : 0.f;
+    U4s[idx] = (j < p.r4) ? p.U4[k * p.r4 + j] : 0.f;
+  }
+  const TX* __restrict__ X = reinterpret_cast<const TX*>(p.X);
+  const int pl = tid / S, i = tid - pl * S;
+  const int64_t n_tiles = (p.n_planes + NP - 1) / NP;
+
+  auto stage = [&](float* dst, int64_t t, int& np) {
+    const int64_t p0 = t * NP;
+    np = (int)((p.n_planes - p0 < NP) ? (p.n_planes - p0) : NP);
+    const TX* src = X + p0 * SS;
+    if (sizeof(TX) == 4 && p.vec4) {
+      for (int idx = tid; idx < np * SS / 4; idx += NT)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst + 4 * idx)), "l"(src + 4 * idx) : "memory");
+    } else {
+      for (int idx = tid; idx < np * SS; idx += NT) dst[idx] = ld_as_float(src + idx);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  float acc3[R], acc4[R];
+#pragma unroll
+  for (int j = 0; j < R; ++j) acc3[j] = acc4[j] = 0.f;
+  int n_cur = 0, n_next = 0, buf = 0;
+  int64_t t = blockIdx.x;
+  if (t < n_tiles) stage(Xs0, t, n_cur);
+  for (; t < n_tiles; t += gridDim.x) {
+    float* Xc = buf ? Xs1 : Xs0;
+    float* Xn = buf ? Xs0 : Xs1;
+    const int64_t tn = t + gridDim.x;
+    if (tn < n_tiles) {
+      stage(Xn, tn, n_next);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const bool on = pl < n_cur;                     // pl < NP follows
+    const float* Xp = Xc + pl * SS;
+    if (on) {
+      float v3[R], v4[R];
+#pragma unroll
+      for (int j = 0; j < R; ++j) v3[j] = v4[j] = 0.f;
+#pragma unroll 4
+      for (int h = 0; h < S; ++h) {                 // column i
+        const float x = Xp[h * S + i];
+#pragma unroll
+        for (int j = 0; j < R; j += 4) {
+          const float4 u = *reinterpret_cast<const float4*>(U3s + h * R + j);
+          v3[j] = fmaf(x, u.x, v3[j]); v3[j + 1] = fmaf(x, u.y, v3[j + 1]);
+          v3[j + 2] = fmaf(x, u.z, v3[j + 2]); v3[j + 3] = fmaf(x, u.w, v3[j + 3]);
+        }
+      }
+#pragma unroll 2
+      for (int w = 0; w < S; w += 4) {              // row i
+        const float4 x = *reinterpret_cast<const float4*>(Xp + i * S + w);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+          for (int j = 0; j < R; j += 4) {
+            const float4 u = *reinterpret_cast<const float4*>(U4s + (w + e) * R + j);
+            v4[j] = fmaf(xs[e], u.x, v4[j]); v4[j + 1] = fmaf(xs[e], u.y, v4[j + 1]);
+            v4[j + 2] = fmaf(xs[e], u.z, v4[j + 2]); v4[j + 3] = fmaf(xs[e], u.w, v4[j + 3]);
+          }
+      }
+#pragma unroll
+      for (int j = 0; j < R; j += 4) {
+        *reinterpret_cast<float4*>(V3s + (pl * S + i) * R + j) = make_float4(v3[j], v3[j + 1], v3[j + 2], v3[j + 3]);
+        *reinterpret_cast<float4*>(V4s + (pl * S + i) * R + j) = make_float4(v4[j], v4[j + 1], v4[j + 2], v4[j + 3]);
+      }
+    }
+    __syncthreads();
+    if (on) {
+      const float* V3p = V3s + pl * S * R;
+      const float* V4p = V4s + pl * S * R;
+#pragma unroll 2
+      for (int w = 0; w < S; w += 4) {              // row i: P3[i,:]
+        const float4 x = *reinterpret_cast<const float4*>(Xp + i * S + w);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+          for (int j = 0; j < R; j += 4) {
+            const float4 v = *reinterpret_cast<const float4*>(V3p + (w + e) * R + j);
+            acc3[j] = fmaf(xs[e], v.x, acc3[j]); acc3[j + 1] = fmaf(xs[e], v.y, acc3[j + 1]);
+            acc3[j + 2] = fmaf(xs[e], v.z, acc3[j + 2]); acc3[j + 3] = fmaf(xs[e], v.w, acc3[j + 3]);
+          }
+      }
+#pragma unroll 4
+      for (int h = 0; h < S; ++h) {                 // column i: P4[i,:]
+        const float x = Xp[h * S + i];
+#pragma unroll
+        for (int j = 0; j < R; j += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(V4p + h * R + j);
+          acc4[j] = fmaf(x, v.x, acc4[j]); acc4[j + 1] = fmaf(x, v.y, acc4[j + 1]);
+          acc4[j + 2] = fmaf(x, v.z, acc4[j + 2]); acc4[j + 3] = fmaf(x, v.w, acc4[j + 3]);
+        }
+      }
+    }
+    __syncthreads();
+    n_cur = n_next;
+    buf ^= 1;
+  }
+  // the NP planes of the CTA meet in shared memory in plane order: one partial of P3 and P4 per CTA
+  if (pl < NP) {
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+      V3s[(pl * S + i) * R + j] = acc3[j];
+      V4s[(pl * S + i) * R + j] = acc4[j];
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < S * R; idx += NT) {
+    const int k = idx / R, j = idx % R;
+    float s3 = 0.f, s4 = 0.f;
+    for (int q = 0; q < NP; ++q) {
+      s3 += V3s[q * S * R + idx];
+      s4 += V4s[q * S * R + idx];
+    }
+    if (j < p.r3) p.Pp3[((int64_t)blockIdx.x * S + k) * p.r3 + j] = s3;
+    if (j < p.r4) p.Pp4[((int64_t)blockIdx.x * S + k) * p.r4 + j] = s4;
+  }
+}
+
+size_t plane_smem(int S) {
+  const int NP = 256 / S;
+  return 4 * ((size_t)2 * NP * S * S + 2 * S * 8 + 2 * NP * S * 8) + 64;
+}
+
+template <int R, typename TX>
+static cudaError_t launch_plane_t(const PlaneArgs& p, int grid, cudaStream_t st) {
+  static size_t granted = 48 * 1024;
+  const size_t smem = plane_smem(p.S);
+  if (smem > granted) {
+    cudaError_t e = cudaFuncSetAttribute(k_plane<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    granted = smem;
+  }
+  k_plane<R, TX><<<grid, 256, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t st) {
+  ProfScope prof(ASI_K_EXPAND, st,
+                 (double)p.n_planes * p.S * p.S * (x_bf16 ? 2 : 4) + 4.0 * p.S * (p.r3 + p.r4) * (grid + 1));
+  const int r = p.r3 > p.r4 ? p.r3 : p.r4;
+  if (r <= 4) return x_bf16 ? launch_plane_t<4, __nv_bfloat16>(p, grid, st) : launch_plane_t<4, float>(p, grid, st);
+  return x_bf16 ? launch_plane_t<8, __nv_bfloat16>(p, grid, st) : launch_plane_t<8, float>(p, grid, st);
+}
+
 size_t fiber_smem(int a) {
   const int TQ = kFiberTQ, PQ = TQ + 4, PA = a | 1;
   const size_t tile = (size_t)std::max(TQ * PA, a * PQ);

@@ -53,6 +53,17 @@ struct FiberArgs {
   int r, vec4;
 };
 
+// Modes 3 and 4 of a conv activation in one pass over whole planes (k_plane).
+struct PlaneArgs {
+  const void* X;
+  const float* U3;
+  const float* U4;
+  float* Pp3;          // [grid][S][r3]
+  float* Pp4;          // [grid][S][r4]
+  int64_t n_planes;
+  int S, r3, r4, vec4;
+};
+
 struct QRMode {
   const float* Pp;     // [nsplit][a][r]
   double* Pred;        // [a][r]
@@ -173,6 +184,8 @@ cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_qr_solve(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_fiber(const FiberArgs& p, int grid, bool x_bf16, cudaStream_t st);
 size_t fiber_smem(int a);
+cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t st);
+size_t plane_smem(int S);
 int64_t fiber_tiles(int64_t O, int64_t a, int64_t I);
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
 
@@ -207,5 +220,7 @@ struct asi_plan {
   bool small_rank;                 // every rank <= 8: partials are reduced by the parallel fp64 kernel
   bool fiber[ASI_MAX_MODES];       // mode handled by the single-pass fiber kernel
   int fiber_grid[ASI_MAX_MODES];
+  bool plane;                      // modes 3 and 4 together by the whole-plane kernel
+  int plane_grid;
   int fast_S, fast_R, n_tiles_b, cpb, fold_gs;
 };
