@@ -193,6 +193,15 @@ void layout_wgrad(asi_plan* pl) {
     pl->off_Z[t] = off;
     off = align_up(off + (size_t)z[t] * 4, 256);
   }
+  pl->conv_nsp = 1;
+  pl->off_Z4p = off;
+  if (pl->d.kind == ASI_CONV2D && !pl->fast_wgrad && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) &&
+      (int64_t)pl->r[0] * pl->Ho * pl->Wo >= 1024 && pl->d.cout < 296) {
+    pl->conv_nsp = (int)std::min<int64_t>(16, std::max<int64_t>(2, 592 / pl->d.cout));
+    pl->conv_nsp = (int)std::min<int64_t>(pl->conv_nsp, (int64_t)pl->r[0] * pl->Ho);
+    off = align_up(off + (size_t)pl->conv_nsp * pl->d.cout * pl->r[1] * pl->d.kh * pl->d.kw * 4, 256);
+    pl->launches_wgrad = 5;
+  }
   pl->wgrad_ws = off;
 }
 
@@ -684,7 +693,10 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
   t.H = (int)H; t.W = (int)W; t.Ho = (int)pl->Ho; t.Wo = (int)pl->Wo;
   t.kh = pl->d.kh; t.kw = pl->d.kw; t.sh = pl->d.stride_h; t.sw = pl->d.stride_w;
   t.ph = pl->d.pad_h; t.pw = pl->d.pad_w; t.groups = pl->d.groups;
-  ASI_CUDA(launch_conv_tail(t, st));
+  if (pl->conv_nsp > 1)
+    ASI_CUDA(launch_conv_tail_split(t, reinterpret_cast<float*>(w + pl->off_Z4p), pl->conv_nsp, st));
+  else
+    ASI_CUDA(launch_conv_tail(t, st));
   return ASI_OK;
 }
 

@@ -753,6 +753,90 @@ __global__ void __launch_bounds__(256) k_conv_tail(ConvTailArgs p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Terms 4 and 5 for large output maps, in two launches so the long reduction over (i, h', w') is
+// spread over Cout x nsp CTAs: k_conv_z4 writes nsp partial Z4 per output channel (CTA (c', sp)
+// takes the pairs (i, h') == sp (mod nsp); thread (o, g) every G-th of those), k_conv_dw sums them in
+// order and expands with U2.  Loop bounds are computed per tap, so the inner loops carry no branch.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_conv_z4(ConvTailArgs p, float* __restrict__ Z4p, int nsp) {
+  extern __shared__ float sm[];
+  const int tid = threadIdx.x;
+  const int co = blockIdx.x, sp = blockIdx.y;
+  const int kk = p.kh * p.kw;
+  const int n_out = p.r2 * kk;
+  const int G = (n_out <= 256) ? 256 / n_out : 1;
+  float* red = sm;                                  // [G][n_out]
+  const int n_items = p.r1 * p.Ho;
+  for (int t = tid; t < n_out * G; t += 256) {
+    const int o = t % n_out, g = t / n_out;
+    const int j = o / kk, tt = o % kk, ky = tt / p.kw, kx = tt % p.kw;
+    int wo_lo = (p.pw - kx > 0) ? (p.pw - kx + p.sw - 1) / p.sw : 0;
+    int wo_hi = (p.W - 1 + p.pw - kx >= 0) ? (p.W - 1 + p.pw - kx) / p.sw + 1 : 0;
+    if (wo_hi > p.Wo) wo_hi = p.Wo;
+    float acc0 = 0.f, acc1 = 0.f;
+    for (int it = sp + nsp * g; it < n_items; it += nsp * G) {
+      const int i = it / p.Ho, ho = it - i * p.Ho;
+      const int h = ho * p.sh + ky - p.ph;
+      if (h < 0 || h >= p.H) continue;
+      const float* z1 = p.Z1 + (((int64_t)i * p.Cout + co) * p.Ho + ho) * p.Wo;
+      const float* z3 = p.Z3 + (((int64_t)i * p.r2 + j) * p.H + h) * p.W + kx - p.pw;
+      int wo = wo_lo;
+#pragma unroll 4
+      for (; wo + 1 < wo_hi; wo += 2) {
+        acc0 = fmaf(__ldg(z1 + wo), __ldg(z3 + wo * p.sw), acc0);
+        acc1 = fmaf(__ldg(z1 + wo + 1), __ldg(z3 + (wo + 1) * p.sw), acc1);
+      }
+      if (wo < wo_hi) acc0 = fmaf(__ldg(z1 + wo), __ldg(z3 + wo * p.sw), acc0);
+    }
+    red[g * n_out + o] = acc0 + acc1;
+  }
+  __syncthreads();
+  for (int o = tid; o < n_out; o += 256) {
+    float v = 0.f;
+    for (int g = 0; g < G; ++g) v += red[g * n_out + o];
+    Z4p[((int64_t)sp * p.Cout + co) * n_out + o] = v;
+  }
+}
+
+__global__ void __launch_bounds__(256) k_conv_dw(ConvTailArgs p, const float* __restrict__ Z4p, int nsp) {
+  extern __shared__ float sm[];
+  const int tid = threadIdx.x;
+  const int co = blockIdx.x;
+  const int kk = p.kh * p.kw;
+  const int n_out = p.r2 * kk;
+  float* Z4s = sm;
+  for (int o = tid; o < n_out; o += 256) {
+    float v = 0.f;
+    for (int s = 0; s < nsp; ++s) v += Z4p[((int64_t)s * p.Cout + co) * n_out + o];
+    Z4s[o] = v;
+  }
+  __syncthreads();
+  const int cg = p.C / p.groups, og = p.Cout / p.groups;
+  const int g = co / og;
+  float* dw = p.dW + (int64_t)co * cg * kk;
+  for (int idx = tid; idx < cg * kk; idx += 256) {
+    const int cl = idx / kk, t = idx % kk;
+    const float* u = p.U2 + (int64_t)(g * cg + cl) * p.r2;
+    float v = 0.f;
+    for (int j = 0; j < p.r2; ++j) v = fmaf(Z4s[j * kk + t], u[j], v);
+    dw[idx] = v;
+  }
+}
+
+cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, cudaStream_t st) {
+  ProfScope prof(ASI_K_CONV_TAIL, st,
+                 4.0 * ((double)p.r1 * p.Cout * p.Ho * p.Wo + (double)p.r1 * p.r2 * p.H * p.W +
+                        (double)p.C * p.r2 + (double)p.Cout * (p.C / p.groups) * p.kh * p.kw));
+  const int n_out = p.r2 * p.kh * p.kw;
+  const int G = (n_out <= 256) ? 256 / n_out : 1;
+  k_conv_z4<<<dim3(p.Cout, nsp), 256, (size_t)G * n_out * sizeof(float), st>>>(p, Z4p, nsp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_conv_dw<<<p.Cout, 256, (size_t)n_out * sizeof(float), st>>>(p, Z4p, nsp);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_CONV_TAIL, st,
                  4.0 * ((double)p.r1 * p.Cout * p.Ho * p.Wo + (double)p.r1 * p.r2 * p.H * p.W +

@@ -188,6 +188,7 @@ cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t
 size_t plane_smem(int S);
 int64_t fiber_tiles(int64_t O, int64_t a, int64_t I);
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
+cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, cudaStream_t st);
 
 }  // namespace asi
 
@@ -210,7 +211,8 @@ struct asi_plan {
   size_t compress_ws;
 
   // wgrad workspace (byte offsets)
-  size_t off_Z[3];
+  size_t off_Z[3], off_Z4p;
+  int conv_nsp;                    // > 1: terms 4-5 in two launches with conv_nsp partial Z4 per channel
   size_t wgrad_ws;
 
   int launches_compress, launches_wgrad;
