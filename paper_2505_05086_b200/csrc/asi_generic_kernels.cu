@@ -106,11 +106,107 @@ __global__ void __launch_bounds__(128) k_modeprod(ModeProdArgs p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// k_gemm: register-tiled fp32 GEMM C = op(A) B for the last mode of a tensor (contiguous fibers) at
+// ranks >= 16, where the thread-per-column kernels above run out of parallelism:
+//   AKMAJOR  : C[M x N] = A[M x K] B[K x N], A stored [M][lda]      (V = A_m^T U, core product)
+//   !AKMAJOR : C[M x N] = A^T B,            A stored [K][lda]      (P = A_m V), K split over grid.y
+// CTA tile 64 x BN, K chunks of 32, thread tile 4 x BN/16; B and C are row-major with N columns.
+// ---------------------------------------------------------------------------------------------
+struct GemmArgs {
+  const void* A;
+  const float* B;
+  float* C;            // [nsplit][M][N]
+  int M, N, K;
+  int64_t lda;
+  int k_per_split;
+};
+
+template <bool AKMAJOR, int BN, typename TX>
+__global__ void __launch_bounds__(256) k_gemm(GemmArgs p) {
+  constexpr int BM = 64, BK = 32, TN = BN / 16;
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.x * BM;
+  const int kb = blockIdx.y * p.k_per_split;
+  const int ke = (kb + p.k_per_split < p.K) ? kb + p.k_per_split : p.K;
+  const TX* __restrict__ A = reinterpret_cast<const TX*>(p.A);
+  float acc[4][TN];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+  for (int k0 = kb; k0 < ke; k0 += BK) {
+    if (AKMAJOR) {
+      for (int idx = tid; idx < BM * BK; idx += 256) {
+        const int r = idx / BK, kk = idx % BK;
+        const int m = m0 + r, k = k0 + kk;
+        As[kk][r] = (m < p.M && k < ke) ? ld_as_float(A + (int64_t)m * p.lda + k) : 0.f;
+      }
+    } else {
+      for (int idx = tid; idx < BM * BK; idx += 256) {
+        const int kk = idx / BM, r = idx % BM;
+        const int m = m0 + r, k = k0 + kk;
+        As[kk][r] = (m < p.M && k < ke) ? ld_as_float(A + (int64_t)k * p.lda + m) : 0.f;
+      }
+    }
+    for (int idx = tid; idx < BK * BN; idx += 256) {
+      const int kk = idx / BN, n = idx % BN;
+      const int k = k0 + kk;
+      Bs[kk][n] = (k < ke && n < p.N) ? p.B[(int64_t)k * p.N + n] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w};
+      float bv[TN];
+      if constexpr (TN == 4) {
+        const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+        bv[0] = b.x; bv[1] = b.y; bv[2] = b.z; bv[3] = b.w;
+      } else {
+        const float2 b = *reinterpret_cast<const float2*>(&Bs[kk][tx * 2]);
+        bv[0] = b.x; bv[1] = b.y;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* C = p.C + (int64_t)blockIdx.y * p.M * p.N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= p.M) continue;
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      const int n = tx * TN + j;
+      if (n < p.N) C[(int64_t)m * p.N + n] = acc[i][j];
+    }
+  }
+}
+
+template <bool AKMAJOR, typename TX>
+static cudaError_t launch_gemm_t(const GemmArgs& g, int nsplit, cudaStream_t st) {
+  dim3 grid((unsigned)((g.M + 63) / 64), (unsigned)nsplit);
+  if (g.N <= 32) k_gemm<AKMAJOR, 32, TX><<<grid, 256, 0, st>>>(g);
+  else k_gemm<AKMAJOR, 64, TX><<<grid, 256, 0, st>>>(g);
+  return cudaGetLastError();
+}
+
 template <typename TX>
 static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
   if (p.Q <= 0 || p.n_out <= 0) return cudaSuccess;
   ProfScope prof(ASI_K_MODEPROD, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
+  if (p.I == 1 && p.n_out >= 16 && p.n_out <= 64 && p.a >= 64 && p.Q >= 64 && p.sj == 1 && p.so == p.n_out &&
+      p.ldb_k == p.n_out && p.ldb_j == 1 && p.Q < (1 << 30) && p.a < (1 << 30)) {
+    GemmArgs g = {p.X, p.B, p.Y, (int)p.Q, p.n_out, (int)p.a, p.a, (int)p.a};
+    return launch_gemm_t<true, TX>(g, 1, st);
+  }
   int R = 4;
   while (R < p.n_out && R < 64) R *= 2;
   dim3 grid((unsigned)((p.Q + 127) / 128), (unsigned)((p.n_out + R - 1) / R));
@@ -181,6 +277,10 @@ template <typename TX>
 static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_EXPAND, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.Q * p.r + (double)p.nsplit * p.a * p.r));
+  if (p.I == 1 && p.r >= 16 && p.a >= 64 && p.Q < (1 << 30) && p.a < (1 << 30)) {
+    GemmArgs g = {p.X, p.V, p.Pp, (int)p.a, p.r, (int)p.Q, p.a, (int)p.q_per_split};
+    return launch_gemm_t<false, TX>(g, p.nsplit, st);
+  }
   int R = 8;
   while (R < p.r) R *= 2;
   dim3 grid((unsigned)((p.a + kExpandKC - 1) / kExpandKC), (unsigned)p.nsplit);
