@@ -120,11 +120,12 @@ struct GemmArgs {
   int M, N, K;
   int64_t lda;
   int k_per_split;
+  int vec8;            // bf16 A rows may be read 16 bytes at a time (aligned base, lda % 8 == 0)
 };
 
-template <bool AKMAJOR, int BN, typename TX>
-__global__ void __launch_bounds__(256) k_gemm(GemmArgs p) {
-  constexpr int BM = 64, BK = 32, TN = BN / 16;
+template <bool AKMAJOR, int BM, int BN, typename TX>
+__global__ void __launch_bounds__(BM * 4) k_gemm(GemmArgs p) {
+  constexpr int BK = 32, TN = BN / 16, NT = BM * 4;
   __shared__ __align__(16) float As[BK][BM + 4];
   __shared__ __align__(16) float Bs[BK][BN];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -139,19 +140,35 @@ __global__ void __launch_bounds__(256) k_gemm(GemmArgs p) {
     for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
   for (int k0 = kb; k0 < ke; k0 += BK) {
     if (AKMAJOR) {
-      for (int idx = tid; idx < BM * BK; idx += 256) {
-        const int r = idx / BK, kk = idx % BK;
-        const int m = m0 + r, k = k0 + kk;
-        As[kk][r] = (m < p.M && k < ke) ? ld_as_float(A + (int64_t)m * p.lda + k) : 0.f;
+      if (sizeof(TX) == 2 && p.vec8 && k0 + BK <= ke) {
+        // 8 bf16 (16 bytes) per load: thread -> row r, k-octet o
+        for (int idx = tid; idx < BM * (BK / 8); idx += NT) {
+          const int r = idx / (BK / 8), o = idx % (BK / 8);
+          const int m = m0 + r;
+          uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+          if (m < p.M) raw = *reinterpret_cast<const uint4*>(A + (int64_t)m * p.lda + k0 + 8 * o);
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            As[8 * o + 2 * e][r] = __uint_as_float(w[e] << 16);
+            As[8 * o + 2 * e + 1][r] = __uint_as_float(w[e] & 0xffff0000u);
+          }
+        }
+      } else {
+        for (int idx = tid; idx < BM * BK; idx += NT) {
+          const int r = idx / BK, kk = idx % BK;
+          const int m = m0 + r, k = k0 + kk;
+          As[kk][r] = (m < p.M && k < ke) ? ld_as_float(A + (int64_t)m * p.lda + k) : 0.f;
+        }
       }
     } else {
-      for (int idx = tid; idx < BM * BK; idx += 256) {
+      for (int idx = tid; idx < BM * BK; idx += NT) {
         const int kk = idx / BM, r = idx % BM;
         const int m = m0 + r, k = k0 + kk;
         As[kk][r] = (m < p.M && k < ke) ? ld_as_float(A + (int64_t)k * p.lda + m) : 0.f;
       }
     }
-    for (int idx = tid; idx < BK * BN; idx += 256) {
+    for (int idx = tid; idx < BK * BN; idx += NT) {
       const int kk = idx / BN, n = idx % BN;
       const int k = k0 + kk;
       Bs[kk][n] = (k < ke && n < p.N) ? p.B[(int64_t)k * p.N + n] : 0.f;
@@ -191,9 +208,18 @@ __global__ void __launch_bounds__(256) k_gemm(GemmArgs p) {
 
 template <bool AKMAJOR, typename TX>
 static cudaError_t launch_gemm_t(const GemmArgs& g, int nsplit, cudaStream_t st) {
-  dim3 grid((unsigned)((g.M + 63) / 64), (unsigned)nsplit);
-  if (g.N <= 32) k_gemm<AKMAJOR, 32, TX><<<grid, 256, 0, st>>>(g);
-  else k_gemm<AKMAJOR, 64, TX><<<grid, 256, 0, st>>>(g);
+  GemmArgs a = g;
+  a.vec8 = (sizeof(TX) == 2 && g.lda % 8 == 0 && (reinterpret_cast<uintptr_t>(g.A) & 15u) == 0 &&
+            g.k_per_split % 8 == 0) ? 1 : 0;
+  if ((int64_t)((g.M + 63) / 64) * nsplit >= 148) {     // enough 64-row tiles to fill the machine
+    dim3 grid((unsigned)((g.M + 63) / 64), (unsigned)nsplit);
+    if (g.N <= 32) k_gemm<AKMAJOR, 64, 32, TX><<<grid, 256, 0, st>>>(a);
+    else k_gemm<AKMAJOR, 64, 64, TX><<<grid, 256, 0, st>>>(a);
+  } else {
+    dim3 grid((unsigned)((g.M + 31) / 32), (unsigned)nsplit);
+    if (g.N <= 32) k_gemm<AKMAJOR, 32, 32, TX><<<grid, 128, 0, st>>>(a);
+    else k_gemm<AKMAJOR, 32, 64, TX><<<grid, 128, 0, st>>>(a);
+  }
   return cudaGetLastError();
 }
 
@@ -204,7 +230,7 @@ static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
   if (p.I == 1 && p.n_out >= 16 && p.n_out <= 64 && p.a >= 64 && p.Q >= 64 && p.sj == 1 && p.so == p.n_out &&
       p.ldb_k == p.n_out && p.ldb_j == 1 && p.Q < (1 << 30) && p.a < (1 << 30)) {
-    GemmArgs g = {p.X, p.B, p.Y, (int)p.Q, p.n_out, (int)p.a, p.a, (int)p.a};
+    GemmArgs g = {p.X, p.B, p.Y, (int)p.Q, p.n_out, (int)p.a, p.a, (int)p.a, 0};
     return launch_gemm_t<true, TX>(g, 1, st);
   }
   int R = 4;
@@ -278,7 +304,7 @@ static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_EXPAND, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.Q * p.r + (double)p.nsplit * p.a * p.r));
   if (p.I == 1 && p.r >= 16 && p.a >= 64 && p.Q < (1 << 30) && p.a < (1 << 30)) {
-    GemmArgs g = {p.X, p.V, p.Pp, (int)p.a, p.r, (int)p.Q, p.a, (int)p.q_per_split};
+    GemmArgs g = {p.X, p.V, p.Pp, (int)p.a, p.r, (int)p.Q, p.a, (int)p.q_per_split, 0};
     return launch_gemm_t<false, TX>(g, p.nsplit, st);
   }
   int R = 8;
