@@ -66,9 +66,13 @@ void choose_kernels(asi_plan* pl) {
     a.B = (int)B; a.C = (int)C; a.Cout = Cout; a.H = (int)H; a.W = (int)W;
     a.Ho = (int)pl->Ho; a.Wo = (int)pl->Wo; a.kh = pl->d.kh; a.kw = pl->d.kw; a.cpb = cpb;
     a.ph = pl->d.pad_h; a.pw = pl->d.pad_w; a.groups = pl->d.groups;
+    // term 5 expands the channels in two rounds when the staging blocks fit, else one at a time
+    a.ncl = cpb >= 2 ? cpb / 2 : 1;
+    if (sm_wgrad_smem(a, R) > kSmemLimit) a.ncl = 1;
     if (sm_wgrad_smem(a, R) <= kSmemLimit) {
       pl->fast_wgrad = true;
       pl->cpb = cpb;
+      pl->wgrad_ncl = a.ncl;
       pl->wgrad_bulk = rows_ok && !pl->bf16;
     }
   }
@@ -651,6 +655,7 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
     g.H = (int)pl->dims[2]; g.W = (int)pl->dims[3]; g.Ho = (int)pl->Ho; g.Wo = (int)pl->Wo;
     g.kh = pl->d.kh; g.kw = pl->d.kw; g.sh = pl->d.stride_h; g.sw = pl->d.stride_w;
     g.ph = pl->d.pad_h; g.pw = pl->d.pad_w; g.groups = pl->d.groups; g.cpb = pl->cpb;
+    g.ncl = pl->wgrad_ncl;
     g.pj = sm_wgrad_pitch(pl->cpb * (int)(pl->Ho * pl->Wo));
     g.bulk = pl->wgrad_bulk ? 1 : 0;
     if (g.bulk && (reinterpret_cast<uintptr_t>(dY) & 15u)) return ASI_ERR_INVALID_ARG;

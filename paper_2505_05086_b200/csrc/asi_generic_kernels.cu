@@ -643,7 +643,7 @@ size_t plane_smem(int S) {
 
 template <int R, typename TX>
 static cudaError_t launch_plane_t(const PlaneArgs& p, int grid, cudaStream_t st) {
-  static size_t granted = 48 * 1024;
+  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = plane_smem(p.S);
   if (smem > granted) {
     cudaError_t e = cudaFuncSetAttribute(k_plane<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -675,7 +675,7 @@ int64_t fiber_tiles(int64_t O, int64_t a, int64_t I) {
 
 template <int R, typename TX>
 static cudaError_t launch_fiber_t(const FiberArgs& p, int grid, cudaStream_t st) {
-  static size_t granted = 48 * 1024;
+  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = fiber_smem((int)p.a);
   if (smem > granted) {
     cudaError_t e = cudaFuncSetAttribute(k_fiber<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

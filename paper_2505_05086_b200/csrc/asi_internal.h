@@ -139,6 +139,7 @@ struct SmWgradArgs {
   int B, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups, cpb;
   int pj;                       // row pitch (floats) of the staged dY tile
   int bulk;                     // 1: rows staged by the bulk-copy engine (fp32, 16-byte aligned rows)
+  int ncl;                      // output channels expanded per round of term 5 (divides cpb)
   int bulk_store;               // 1: dW row blocks leave through the bulk-copy engine (16-byte sized and aligned)
 };
 size_t sm_pass1_smem(int S, int R, int B, int C);
@@ -224,5 +225,5 @@ struct asi_plan {
   int fiber_grid[ASI_MAX_MODES];
   bool plane;                      // modes 3 and 4 together by the whole-plane kernel
   int plane_grid;
-  int fast_S, fast_R, n_tiles_b, cpb, fold_gs;
+  int fast_S, fast_R, n_tiles_b, cpb, wgrad_ncl, fold_gs;
 };

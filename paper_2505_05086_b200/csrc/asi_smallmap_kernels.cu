@@ -117,21 +117,6 @@ __device__ __forceinline__ bool cta_wait_tile(uint64_t* bar, int* s_flag, int* s
   return ok;
 }
 
-// Warp 0 stages `rows` rows of `row_bytes` each: row i from src + i*src_stride_bytes to
-// dst + i*dst_stride_bytes.
-__device__ __forceinline__ void stage_rows(uint64_t* bar, char* dst, const char* src, int rows,
-                                           uint32_t row_bytes, int64_t src_stride_bytes,
-                                           uint32_t dst_stride_bytes) {
-  const int lane = threadIdx.x & 31;
-  if ((threadIdx.x >> 5) != 0) return;
-  if (lane == 0) {
-    mbar_init(bar, 1);
-    mbar_expect_tx(bar, (uint32_t)rows * row_bytes);
-  }
-  __syncwarp();
-  for (int i = lane; i < rows; i += 32)
-    bulk_g2s(dst + (size_t)i * dst_stride_bytes, src + (int64_t)i * src_stride_bytes, row_bytes, bar);
-}
 // Warp 0 stages one contiguous block in chunks of 16 KB.
 __device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char* src, uint32_t bytes) {
   constexpr uint32_t kChunk = 16384;
@@ -173,6 +158,24 @@ __device__ __forceinline__ void fac_issue_flat(const float* __restrict__ src, fl
 }
 __device__ __forceinline__ void fac_wait() {
   asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's committed groups are still in flight
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// Starts the copy of `rows` fp32 rows of J values (J a multiple of 4, both sides 16-byte aligned): row i
+// from src + i*src_stride to dst + i*PJ, 16 bytes per cp.async, one row per warp at a time.  (One bulk
+// copy per row would leave the issuing warp busy for ~60 cycles per row: the tile of a 64-sample
+// batch would arrive ~2 us later.)
+__device__ __forceinline__ void stage_rows_async(float* dst, const float* __restrict__ src, int rows, int J,
+                                                 int64_t src_stride, int PJ) {
+  const int lane = threadIdx.x & 31, nv = J >> 2;
+  for (int i = threadIdx.x >> 5; i < rows; i += kNT / 32) {
+    const float* s = src + i * src_stride;
+    float* d = dst + i * PJ;
+    for (int v = lane; v < nv; v += 32)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(d + 4 * v)), "l"(s + 4 * v) : "memory");
+  }
 }
 
 template <int R>
@@ -331,10 +334,9 @@ __device__ __forceinline__ void project_channels(const float* __restrict__ Xs, c
 // Stages one tile [B x J] (row b at src + b*sample_stride) as fp32 rows of pitch PJ.
 template <typename TX>
 __device__ __forceinline__ void stage_tile_begin(const TX* __restrict__ src, int64_t sample_stride, float* Xs,
-                                                 int B, int J, int PJ, uint64_t* bar) {
+                                                 int B, int J, int PJ) {
   if constexpr (std::is_same<TX, float>::value) {
-    stage_rows(bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(src), B, (uint32_t)J * 4u,
-               sample_stride * 4, (uint32_t)PJ * 4u);
+    stage_rows_async(Xs, src, B, J, sample_stride, PJ);
   } else {
     const int J4 = J / 4;
     for (int idx = threadIdx.x; idx < B * J4; idx += kNT) {
@@ -389,13 +391,9 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
       fac_issue_padded<R>(p.U_prev + p.u_off[2], U3s, S, p.r[2]);
       fac_issue_padded<R>(p.U_prev + p.u_off[3], U4s, S, p.r[3]);
     }
-    stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ, &s_bar);
+    stage_tile_begin<TX>(A + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ);
     fac_wait();
-    if constexpr (kBulk) {
-      if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
-    } else {
-      __syncthreads();
-    }
+    __syncthreads();
     const int t = tid & (kNG - 1), wg = t >> 5;
     if (tid < kNG) {
       // ---- half 0: mode 1.  V[j,:] = sum_b X[b,j] U1[b,:], then P1[b,:] = sum_j X[b,j] V[j,:]
@@ -601,9 +599,10 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* V2s = U2s + C * R;                        // [HWC][R]
     float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
     const TX* Xb = A + (int64_t)b * C * HW + q * HWC;
+    if constexpr (kBulkC)
+      stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
     fac_issue_padded<R>(p.U_prev + p.u_off[1], U2s, C, p.r[1]);
     if constexpr (kBulkC) {
-      stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
     } else if constexpr (NQ == 1) {
       const int n4 = C * HW / 4;
       for (int idx = tid; idx < n4; idx += kNT) *reinterpret_cast<float4*>(Xs + 4 * idx) = ld4<TX>(Xb + 4 * idx);
@@ -750,15 +749,12 @@ cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cuda
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
 __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
-  constexpr bool kBulk = std::is_same<TX, float>::value;
   constexpr int HW = S * S;
   constexpr int CC = (S == 7) ? 4 : 1;
   constexpr int J = CC * HW;
   constexpr int PJ = pitch4(J);
   constexpr int NH = batch_groups(kNT, J);
   extern __shared__ __align__(128) float smem[];
-  __shared__ __align__(8) uint64_t s_bar;
-  __shared__ int s_flag;
   __shared__ int s_last;
   __shared__ double Gq[4][4][R * R];
   __shared__ double Gs[4][R][R + 1];
@@ -778,8 +774,8 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   float* part = Ws + J * R;             // [NH][J][R]
   float* Ysm = part + NH * J * R;       // [R R][HW]
   float* T3s = Ysm + R * R * HW;        // [R R][R][S]
-  stage_tile_begin<TX>(reinterpret_cast<const TX*>(p.act) + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ,
-                       &s_bar);
+  stage_tile_begin<TX>(reinterpret_cast<const TX*>(p.act) + (int64_t)tile * J, (int64_t)C * HW, Xs, B, J, PJ);
+  cp_async_commit();
   pdl_wait();                           // P_m and the Gram shares come from the reduction kernel
   // ---- the factor row this thread will solve for: [U1: B rows][U2: CC rows][U3: S][U4: S]
   const int nrows = B + CC + 2 * S;     // <= kNT (checked when the plan picks this kernel)
@@ -894,11 +890,8 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
       rdst[j] = out;
     }
   }
-  if constexpr (kBulk) {
-    if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
-  } else {
-    __syncthreads();
-  }
+  cp_async_wait<0>();
+  __syncthreads();
   project_batch<R>(Xs, PJ, U1s, B, J, part, Ws, tid, kNT, 0);
   // Y[(i,j)][hw] = sum_cl U2[cl][j] W[cl*HW + hw][i]
   const int r12 = r1 * r2;
@@ -989,11 +982,15 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
 //   Z1 = dY x_1 U1^T on the CTA's channels;
 //   Z4[c',j,kh,kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p];  dW = Z4 x_2 U2.
 // ---------------------------------------------------------------------------------------------
-// Term 5: dW[c0+cl, c, t] = sum_j Z4[cl][t][j] U2[(g cg + c), j].  A thread owns input channel c (its
-// row of U2 stays in registers) and writes the kk taps of every output channel into a staging row
-// block in shared memory; the block [cg x kk] then leaves for global memory in one piece -- by the
-// bulk-copy engine (cp.async.bulk shared -> global) when it is 16-byte sized and aligned, two blocks in
-// flight, else by coalesced stores.
+// Term 5: dW[c0+cl, c, t] = sum_j Z4[cl][t][j] U2[(g cg + c), j].  The rows of Z4 are the same for every
+// thread, so each 16-byte shared-memory read of one costs a full warp-wide transfer; a thread therefore
+// owns up to four input channels (their rows of U2 stay in registers) and every row of Z4 it reads feeds
+// four dot products (fewer, busier threads: the shared-memory pipe is the limit).  p.ncl output channels
+// are expanded per round, one thread group each, into a staging block [ncl][cg x kk] in shared memory
+// that then leaves for global memory in one piece per channel -- by the bulk-copy engine
+// (cp.async.bulk shared -> global) when a channel's block is 16-byte sized and aligned, else by
+// coalesced stores.  With more than one round there are two staging blocks, so that a round's stores
+// run under the next round's arithmetic: the write of dW by all CTAs at once is DRAM-bound.
 template <int R>
 __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const float* __restrict__ Z4s,
                                                   const float* __restrict__ U2s, float* stage, int c0) {
@@ -1001,52 +998,73 @@ __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const fl
   const int cg = p.C / p.groups, og = p.Cout / p.groups;
   const int tid = threadIdx.x;
   const int nblk = cg * kk;
+  const int lg = (p.ncl == 4) ? 2 : (p.ncl == 2 ? 1 : 0);
+  const int TG = kNT >> lg;                          // threads per output channel
+  const int grp = tid / TG, tg = tid - grp * TG;
+  int ta = (((cg + 3) >> 2) + 31) & ~31;             // active threads of a group: four channels each
+  if (ta > TG) ta = TG;
+  const int rounds = p.cpb / p.ncl;
 #pragma unroll 1
-  for (int cl = 0; cl < p.cpb; ++cl) {
+  for (int rd = 0; rd < rounds; ++rd) {
+    const int cl = rd * p.ncl + grp;
     const int co = c0 + cl;
     const int g = co / og;
-    float* dw = p.dW + (int64_t)co * nblk;
+    float* dw = p.dW + (int64_t)(c0 + rd * p.ncl) * nblk;
     const float* u2 = U2s + (int64_t)g * cg * R;
-    float* buf = stage + (cl & 1) * nblk;
-    if (p.bulk_store && cl >= 2) {
+    float* buf = stage + (rd & 1) * p.ncl * nblk;
+    if (p.bulk_store && rd >= 2) {
       if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
       __syncthreads();
     }
+    float* out = buf + grp * nblk;
+    const float* z = Z4s + cl * kk * R;
 #pragma unroll 1
-    for (int c = tid; c < cg; c += kNT) {
-      float u[R];
+    for (int cb = tg; cb < cg && tg < ta; cb += 4 * ta) {
+      float u[4][R];
 #pragma unroll
-      for (int j = 0; j < R; j += 4) {
-        const float4 v = *reinterpret_cast<const float4*>(u2 + c * R + j);
-        u[j] = v.x; u[j + 1] = v.y; u[j + 2] = v.z; u[j + 3] = v.w;
+      for (int m = 0; m < 4; ++m) {
+        const int c = cb + m * ta;
+#pragma unroll
+        for (int j = 0; j < R; j += 4) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (c < cg) v = *reinterpret_cast<const float4*>(u2 + c * R + j);
+          u[m][j] = v.x; u[m][j + 1] = v.y; u[m][j + 2] = v.z; u[m][j + 3] = v.w;
+        }
       }
-      const float* z = Z4s + cl * kk * R;
 #pragma unroll 3
       for (int t = 0; t < kk; ++t) {
-        float v = 0.f;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < R; j += 4) {
           const float4 zz = *reinterpret_cast<const float4*>(z + t * R + j);
-          v = fmaf(zz.x, u[j], v);
-          v = fmaf(zz.y, u[j + 1], v);
-          v = fmaf(zz.z, u[j + 2], v);
-          v = fmaf(zz.w, u[j + 3], v);
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            v[m] = fmaf(zz.x, u[m][j], v[m]);
+            v[m] = fmaf(zz.y, u[m][j + 1], v[m]);
+            v[m] = fmaf(zz.z, u[m][j + 2], v[m]);
+            v[m] = fmaf(zz.w, u[m][j + 3], v[m]);
+          }
         }
-        buf[c * kk + t] = v;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int c = cb + m * ta;
+          if (c < cg) out[c * kk + t] = v[m];
+        }
       }
     }
     if (p.bulk_store) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncthreads();
       if (tid == 0) {
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dw), "r"(smem_u32(buf)),
-                     "r"((uint32_t)nblk * 4u)
-                     : "memory");
+        for (int q = 0; q < p.ncl; ++q)
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dw + (int64_t)q * nblk),
+                       "r"(smem_u32(buf + q * nblk)), "r"((uint32_t)nblk * 4u)
+                       : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     } else {
       __syncthreads();
-      for (int idx = tid; idx < nblk; idx += kNT) dw[idx] = buf[idx];
+      for (int idx = tid; idx < p.ncl * nblk; idx += kNT) dw[idx] = buf[idx];
     }
   }
   if (p.bulk_store && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -1055,8 +1073,6 @@ __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const fl
 template <int R, typename TX>
 __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   extern __shared__ __align__(128) float smem[];
-  __shared__ __align__(8) uint64_t s_bar;
-  __shared__ int s_flag;
   const int tid = threadIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
   const int H = p.H, W = p.W, HW = H * W, HoWo = p.Ho * p.Wo, kk = p.kh * p.kw;
@@ -1065,7 +1081,8 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   const int NH = batch_groups(kNT, J);
   const int c0 = blockIdx.x * p.cpb;
   const int n_out = p.cpb * r2 * kk;
-  const int n_stage = 2 * (p.C / p.groups) * kk;     // two staging blocks of term 5 reuse the tile's space
+  // staging blocks of term 5 reuse the tile's space: ncl channels per round, doubled when rounds follow
+  const int n_stage = (p.cpb > p.ncl ? 2 : 1) * p.ncl * (p.C / p.groups) * kk;
   float* Ys = smem;                                  // [B][PJ]
   float* U1s = Ys + ((p.B * PJ > n_stage ? p.B * PJ : n_stage) + 3) / 4 * 4;   // [B][R]
   float* U2s = U1s + p.B * R;                        // [C][R]
@@ -1089,16 +1106,18 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
     fac_issue_flat(p.U + p.u_off[3], U4s, W * r4);
     fac_issue_padded<R>(p.U + p.u_off[0], U1s, p.B, r1);
     fac_issue_padded<R>(p.U + p.u_off[1], U2s, p.C, r2);
-    if (bulk) {
-      stage_rows(&s_bar, reinterpret_cast<char*>(Ys), reinterpret_cast<const char*>(dY), p.B, (uint32_t)J * 4u,
-                 sstride * 4, (uint32_t)PJ * 4u);
-    } else {
+    cp_async_commit();                               // group 1: factors and core; group 0 (younger): the tile
+    if constexpr (std::is_same<TX, float>::value) {
+      if (bulk) stage_rows_async(Ys, reinterpret_cast<const float*>(dY), p.B, J, sstride, PJ);
+    }
+    if (!bulk) {
       for (int idx = tid; idx < p.B * J; idx += kNT) {
         const int b = idx / J, j = idx - b * J;
         Ys[b * PJ + j] = to_f(dY[b * sstride + j]);
       }
     }
-    fac_wait();
+    cp_async_commit();
+    cp_async_wait<1>();
   }
   __syncthreads();
   // terms 2-3: Tm[ij][h][l] = sum_k S[ij][k][l] U3[h][k];  Z3[ij][h][w] = sum_l Tm[ij][h][l] U4[w][l]
@@ -1122,11 +1141,8 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
       for (int l = 0; l < r4; ++l) s = fmaf(Tm[(ij * H + h) * r4 + l], U4s[w * r4 + l], s);
     Z3s[idx] = s;
   }
-  if (bulk) {
-    if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
-  } else {
-    __syncthreads();
-  }
+  cp_async_wait<0>();
+  __syncthreads();
   // term 1: Z1[j,:] = sum_b dY[b, c0*HoWo + j] U1[b,:]
   project_batch<R>(Ys, PJ, U1s, p.B, J, part, Z1s, tid, kNT, 0);
   // term 4: thread (n, g): outputs n = (j, kh, kw) of all cpb channels and every G-th pair (i, h') of
@@ -1208,7 +1224,8 @@ size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   const int J = p.cpb * p.Ho * p.Wo, kk = p.kh * p.kw;
   const int N4 = r2 * kk;
   const int NH = batch_groups(kNT, J);
-  const size_t tile = (size_t)p.B * pitch4(J), stage = (size_t)2 * (p.C / p.groups) * kk;
+  const size_t tile = (size_t)p.B * pitch4(J),
+               stage = (size_t)(p.cpb > p.ncl ? 2 : 1) * p.ncl * (p.C / p.groups) * kk;
   size_t n = ((tile > stage ? tile : stage) + 3) / 4 * 4 + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
              (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
              (size_t)r1 * r2 * p.H * r4 + ((size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + 3) / 4 * 4 +
@@ -1227,7 +1244,7 @@ static cudaError_t opt_in_smem(K kernel, size_t* granted, size_t need) {
 
 template <int S, int R, typename TX>
 static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
-  static size_t granted = 48 * 1024;
+  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = sm_pass1_smem(S, R, p.B, p.C);
   cudaError_t e = opt_in_smem(k_sm_pass1<S, R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
@@ -1237,7 +1254,7 @@ static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
 
 template <int S, int R, typename TX>
 static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
-  static size_t granted = 48 * 1024;
+  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = sm_core_smem(S, R, p.B);
   cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
@@ -1246,7 +1263,7 @@ static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
 
 template <int R, typename TX>
 static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
-  static size_t granted = 48 * 1024;
+  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = sm_wgrad_smem(p, R);
   cudaError_t e = opt_in_smem(k_sm_wgrad<R, TX>, &granted, smem);
   if (e != cudaSuccess) return e;
