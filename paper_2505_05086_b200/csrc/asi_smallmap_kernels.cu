@@ -346,8 +346,73 @@ __device__ __forceinline__ void stage_tile_begin(const TX* __restrict__ src, int
   }
 }
 
+// Role C of the first pass takes the positions of a sample in NQ parts.  S = 7: the whole map.  Larger
+// maps: four parts that start on 16-byte boundaries -- 14 x 14 splits its 49 float4 per channel as
+// 13 + 12 + 12 + 12 (parts 1..3 carry four zero columns), 16 x 16 as 4 x 16.
+__host__ __device__ constexpr int role_c_hwc(int S) { return S == 7 ? 49 : (S == 14 ? 52 : S * S / 4); }
+__host__ __device__ constexpr int role_c_pitch(int S) { return S == 7 ? 49 : pitch4(role_c_hwc(S)); }
+
 __host__ __device__ constexpr int tri_index(int S, int k, int k2) {   // k <= k2 < S, row-major upper triangle
   return k * S - k * (k - 1) / 2 + (k2 - k);
+}
+
+// 14 x 14 Gram matrix G = A_m A_m^T of a tile [planes x 196] in 7 x 7 blocks.  With a = rows 0..6 and
+// b = rows 7..13 of a fiber, warp role 0 accumulates the upper triangle of a a^T, role 1 that of
+// b b^T, role 2 the block a b[0..3]^T and role 3 the block a b[4..6]^T (<= 28 accumulators each).
+// A unit is a quarter of a plane (fibers == part mod 4), so the lanes of a warp hit 32 banks; this
+// thread takes units u0, u0 + ustride, ...  es = step between the elements of a fiber, cs = step
+// between neighbouring fibers (mode 3: 14, 1; mode 4: 1, 14).
+template <int PJ>
+__device__ __forceinline__ void gram14_accumulate(const float* __restrict__ Xs, int nunits, int u0, int ustride,
+                                                  int role, int es, int cs, float (&acc)[32]) {
+#pragma unroll
+  for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+  for (int un = u0; un < nunits; un += ustride) {
+    const float* base = Xs + (un >> 2) * PJ;
+#pragma unroll 1
+    for (int col = un & 3; col < 14; col += 4) {
+      const float* colp = base + col * cs;
+      if (role < 2) {
+        const float* q = colp + role * 7 * es;
+        float x[7];
+#pragma unroll
+        for (int k = 0; k < 7; ++k) x[k] = q[k * es];
+#pragma unroll
+        for (int k = 0; k < 7; ++k)
+#pragma unroll
+          for (int k2 = k; k2 < 7; ++k2) acc[tri_index(7, k, k2)] = fmaf(x[k], x[k2], acc[tri_index(7, k, k2)]);
+      } else if (role == 2) {
+        float xa[7], xb[4];
+#pragma unroll
+        for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) xb[k] = colp[(7 + k) * es];
+#pragma unroll
+        for (int k = 0; k < 7; ++k)
+#pragma unroll
+          for (int k2 = 0; k2 < 4; ++k2) acc[k * 4 + k2] = fmaf(xa[k], xb[k2], acc[k * 4 + k2]);
+      } else {
+        float xa[7], xb[3];
+#pragma unroll
+        for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) xb[k] = colp[(11 + k) * es];
+#pragma unroll
+        for (int k = 0; k < 7; ++k)
+#pragma unroll
+          for (int k2 = 0; k2 < 3; ++k2) acc[k * 3 + k2] = fmaf(xa[k], xb[k2], acc[k * 3 + k2]);
+      }
+    }
+  }
+}
+// which role (rl) and accumulator (e) hold element o = k*14 + k2 of the symmetric 14 x 14 matrix
+__device__ __forceinline__ void gram14_slot(int o, int& rl, int& e) {
+  const int k = o / 14, k2 = o % 14;
+  const int lo = k < k2 ? k : k2, hi = k < k2 ? k2 : k;
+  if (hi < 7) { rl = 0; e = tri_index(7, lo, hi); }
+  else if (lo >= 7) { rl = 1; e = tri_index(7, lo - 7, hi - 7); }
+  else if (hi < 11) { rl = 2; e = lo * 4 + (hi - 7); }
+  else { rl = 3; e = lo * 3 + (hi - 11); }
 }
 
 }  // namespace
@@ -385,7 +450,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* U4s = U3s + S * R;                        // [S][R]
     float* V1s = U4s + S * R;                        // [J][R]
     float* part = V1s + J * R;                       // [NH1][J][R] (NH1 > 1 only)
-    float* red = part + (NH1 > 1 ? NH1 : 0) * J * R; // [8][32]
+    float* red = part + (NH1 > 1 ? NH1 : 0) * J * R; // [8][32], S = 14: [8 + 16][32]
     fac_issue_padded<R>(p.U_prev + p.u_off[0], U1s, B, p.r[0]);
     if constexpr (!kGram && !kGram14) {
       fac_issue_padded<R>(p.U_prev + p.u_off[2], U3s, S, p.r[2]);
@@ -461,74 +526,18 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
         bar_sync(2, kNG);
       }
     } else if constexpr (kGram14) {
-      // ---- half 1, S = 14: G_m = A_m A_m^T for m = 3, 4 in 7 x 7 blocks.  With a = rows 0..6 and
-      // b = rows 7..13 of a fiber, warp role 0 accumulates the upper triangle of a a^T, role 1 that of
-      // b b^T, role 2 the block a b[0..3]^T and role 3 the block a b[4..6]^T (<= 28 accumulators each).
-      // A unit is a quarter of a plane (fibers == part mod 4), so the lanes of a warp hit 32 banks.
-      constexpr int NACC = 32;
+      // ---- half 1, S = 14: G_3 = A_3 A_3^T (see gram14_accumulate); G_4 follows on all sixteen warps
       const int role = wg & 3;
-      const int u0 = (wg >> 2) * 32 + lane;
-      const int nunits = B * CC * 4;
-#pragma unroll 1
-      for (int mode = 2; mode <= 3; ++mode) {
-        const int es = (mode == 2) ? S : 1;
-        const int cs = (mode == 2) ? 1 : S;
-        float* Gm = p.Pp[mode] + (int64_t)tile * HW;
-        float acc[NACC];
-#pragma unroll
-        for (int i = 0; i < NACC; ++i) acc[i] = 0.f;
-        for (int un = u0; un < nunits; un += 64) {
-          const int pl = un >> 2, part_ = un & 3;
-          const float* base = Xs + (pl / CC) * PJ + (pl % CC) * HW;
-#pragma unroll 1
-          for (int col = part_; col < S; col += 4) {
-            const float* colp = base + col * cs;
-            if (role < 2) {
-              const float* q = colp + role * 7 * es;
-              float x[7];
-#pragma unroll
-              for (int k = 0; k < 7; ++k) x[k] = q[k * es];
-#pragma unroll
-              for (int k = 0; k < 7; ++k)
-#pragma unroll
-                for (int k2 = k; k2 < 7; ++k2) acc[tri_index(7, k, k2)] = fmaf(x[k], x[k2], acc[tri_index(7, k, k2)]);
-            } else if (role == 2) {
-              float xa[7], xb[4];
-#pragma unroll
-              for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) xb[k] = colp[(7 + k) * es];
-#pragma unroll
-              for (int k = 0; k < 7; ++k)
-#pragma unroll
-                for (int k2 = 0; k2 < 4; ++k2) acc[k * 4 + k2] = fmaf(xa[k], xb[k2], acc[k * 4 + k2]);
-            } else {
-              float xa[7], xb[3];
-#pragma unroll
-              for (int k = 0; k < 7; ++k) xa[k] = colp[k * es];
-#pragma unroll
-              for (int k = 0; k < 3; ++k) xb[k] = colp[(11 + k) * es];
-#pragma unroll
-              for (int k = 0; k < 7; ++k)
-#pragma unroll
-                for (int k2 = 0; k2 < 3; ++k2) acc[k * 3 + k2] = fmaf(xa[k], xb[k2], acc[k * 3 + k2]);
-            }
-          }
-        }
-        warp_reduce_scatter<NACC>(acc, lane);
-        red[wg * 32 + scatter_base<NACC>(lane)] = acc[0];
-        bar_sync(2, kNG);
-        for (int o = t; o < HW; o += kNG) {
-          const int k = o / S, k2 = o % S;
-          const int lo = k < k2 ? k : k2, hi = k < k2 ? k2 : k;
-          int rl, e;
-          if (hi < 7) { rl = 0; e = tri_index(7, lo, hi); }
-          else if (lo >= 7) { rl = 1; e = tri_index(7, lo - 7, hi - 7); }
-          else if (hi < 11) { rl = 2; e = lo * 4 + (hi - 7); }
-          else { rl = 3; e = lo * 3 + (hi - 11); }
-          Gm[o] = red[rl * 32 + e] + red[(rl + 4) * 32 + e];
-        }
-        bar_sync(2, kNG);
+      float* Gm = p.Pp[2] + (int64_t)tile * HW;
+      float acc[32];
+      gram14_accumulate<PJ>(Xs, B * 4, (wg >> 2) * 32 + lane, 64, role, S, 1, acc);
+      warp_reduce_scatter<32>(acc, lane);
+      red[wg * 32 + scatter_base<32>(lane)] = acc[0];
+      bar_sync(2, kNG);
+      for (int o = t; o < HW; o += kNG) {
+        int rl, e;
+        gram14_slot(o, rl, e);
+        Gm[o] = red[rl * 32 + e] + red[(rl + 4) * 32 + e];
       }
     } else {
       // ---- half 1, other sizes: P_m = A_m (A_m^T U_m^prev) for m = 3, 4.  A unit is a quarter of a plane
@@ -584,21 +593,40 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
         bar_sync(2, kNG);
       }
     }
+    if constexpr (kGram14) {
+      // ---- S = 14, G_4 = A_4 A_4^T: each half joins as it finishes its first job (mode 1 or G_3)
+      const int gw = tid >> 5, role = gw & 3;
+      float* red4 = red + 8 * 32;                    // [16][32]
+      float acc[32];
+      gram14_accumulate<PJ>(Xs, B * 4, (gw >> 2) * 32 + lane, 128, role, 1, S, acc);
+      warp_reduce_scatter<32>(acc, lane);
+      red4[gw * 32 + scatter_base<32>(lane)] = acc[0];
+      __syncthreads();
+      float* Gm = p.Pp[3] + (int64_t)tile * HW;
+      for (int o = tid; o < HW; o += kNT) {
+        int rl, e;
+        gram14_slot(o, rl, e);
+        Gm[o] = ((red4[rl * 32 + e] + red4[(rl + 4) * 32 + e]) + red4[(rl + 8) * 32 + e]) + red4[(rl + 12) * 32 + e];
+      }
+    }
   } else {
     // ---------------- role C: mode 2 on block [C x HWC] of one sample ----------------
-    // S = 7: the whole sample (contiguous, staged by the bulk-copy engine); larger maps: one quarter
-    // of the positions, rows gathered with plain loads (they are only 4-byte aligned).
+    // S = 7: the whole sample (contiguous, staged by the bulk-copy engine, odd row pitch for the
+    // row-per-thread reads below); larger maps: one part of the positions, rows staged by 16-byte
+    // cp.async at a pitch == 4 (mod 32), read back as float4.
     constexpr int NQ = (S == 7) ? 1 : 4;
-    constexpr int HWC = HW / NQ;
-    constexpr int PC = (HWC % 2 == 0) ? HWC + 1 : HWC;     // odd pitch: conflict-free row-per-thread reads
+    constexpr int HWC = role_c_hwc(S);
+    constexpr int PC = role_c_pitch(S);
     constexpr int G = kNT / HWC;
     constexpr bool kBulkC = kBulk && NQ == 1;
     const int b = blockIdx.x / NQ, q = blockIdx.x % NQ;
+    const int hw0 = (S == 14) ? (q == 0 ? 0 : 4 + 48 * q) : q * HWC;     // first position of this part
+    const int nval = (S == 14 && q > 0) ? 48 : HWC;                      // positions it holds
     float* Xs = smem;                                // [C][PC]
     float* U2s = Xs + ((C * PC + 3) & ~3);           // [C][R]
     float* V2s = U2s + C * R;                        // [HWC][R]
     float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
-    const TX* Xb = A + (int64_t)b * C * HW + q * HWC;
+    const TX* Xb = A + (int64_t)b * C * HW + hw0;
     if constexpr (kBulkC)
       stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
     fac_issue_padded<R>(p.U_prev + p.u_off[1], U2s, C, p.r[1]);
@@ -607,18 +635,19 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
       const int n4 = C * HW / 4;
       for (int idx = tid; idx < n4; idx += kNT) *reinterpret_cast<float4*>(Xs + 4 * idx) = ld4<TX>(Xb + 4 * idx);
     } else {
-      // rows of a quarter are only 4-byte aligned: one 4-byte asynchronous copy per element (fp32),
-      // all of a thread's copies in flight at once
-      const int n = C * HWC;
+      constexpr int NV = HWC / 4;
+      const int n = C * NV;
 #pragma unroll 1
       for (int idx = tid; idx < n; idx += kNT) {
-        const int c = idx / HWC, hw = idx - c * HWC;
-        if constexpr (kBulk) {
-          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(Xs + c * PC + hw)),
-                       "l"(Xb + (int64_t)c * HW + hw)
-                       : "memory");
+        const int c = idx / NV, v = idx - c * NV;
+        float* dst = Xs + c * PC + 4 * v;
+        const TX* src = Xb + (int64_t)c * HW + 4 * v;
+        if (4 * v >= nval) {
+          *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else if constexpr (kBulk) {
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
         } else {
-          Xs[c * PC + hw] = to_f(Xb[(int64_t)c * HW + hw]);
+          *reinterpret_cast<float4*>(dst) = ld4<TX>(src);
         }
       }
     }
@@ -636,8 +665,19 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
       float acc[R];
 #pragma unroll
       for (int j = 0; j < R; ++j) acc[j] = 0.f;
+      if constexpr (NQ == 1) {
 #pragma unroll 7
-      for (int hw = 0; hw < HWC; ++hw) fma_row<R>(acc, row[hw], V2s + hw * R);
+        for (int hw = 0; hw < HWC; ++hw) fma_row<R>(acc, row[hw], V2s + hw * R);
+      } else {
+#pragma unroll 2
+        for (int hw = 0; hw < HWC; hw += 4) {
+          const float4 x = *reinterpret_cast<const float4*>(row + hw);
+          fma_row<R>(acc, x.x, V2s + hw * R);
+          fma_row<R>(acc, x.y, V2s + (hw + 1) * R);
+          fma_row<R>(acc, x.z, V2s + (hw + 2) * R);
+          fma_row<R>(acc, x.w, V2s + (hw + 3) * R);
+        }
+      }
 #pragma unroll
       for (int j = 0; j < R; ++j)
         if (j < p.r[1]) P2[c * p.r[1] + j] = acc[j];
@@ -1199,9 +1239,8 @@ size_t sm_pass1_smem(int S, int R, int B, int C) {
   const int HW = S * S, CC = (S == 7) ? 4 : 1, J = CC * HW, PJ = pitch4(J);
   const int NH1 = batch_groups(kNG, J);
   const size_t role_b = (size_t)B * PJ + (size_t)B * R + 2 * S * R + (size_t)J * R +
-                        (NH1 > 1 ? (size_t)NH1 * J * R : 0) + 8 * 32;
-  const int HWC = (S == 7) ? HW : HW / 4;
-  const int PC = (HWC % 2 == 0) ? HWC + 1 : HWC;
+                        (NH1 > 1 ? (size_t)NH1 * J * R : 0) + 24 * 32;
+  const int HWC = role_c_hwc(S), PC = role_c_pitch(S);
   const int G = kNT / HWC;
   const size_t vp = (C >= (G - 1) * HWC) ? 0 : (size_t)(G - 1) * HWC * R;
   const size_t role_c = (size_t)((C * PC + 3) & ~3) + (size_t)C * R + (size_t)HWC * R + vp;
