@@ -139,6 +139,14 @@ void layout_compress(asi_plan* pl) {
     pl->off_Gp[m] = off;
     off = align_up(off + (size_t)pl->nchunk[m] * v.r * v.r * 8, 256);
   }
+  pl->off_Rf = off;                                   // Cholesky factors of the fused path
+  off = align_up(off + (size_t)ASI_MAX_MODES * kRfStride * 8, 256);
+  for (int m = 0; m < ASI_MAX_MODES; ++m) pl->off_Pg[m] = 0;
+  if (pl->fast_compress)
+    for (int m = 2; m < 4; ++m) {                     // P_m of a Gram mode
+      pl->off_Pg[m] = off;
+      off = align_up(off + (size_t)pl->dims[m] * pl->r[m] * 8, 256);
+    }
   // core chain: contract the mode with the largest a_m / r_m first, then the rest in order
   int order[ASI_MAX_MODES];
   for (int m = 0; m < pl->nd; ++m) order[m] = m;
@@ -247,11 +255,17 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
       if (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) {
         ra.m[m].gram = 1;
         ra.m[m].nchunk = (int)((pl->dims[m] * pl->dims[m] + 24) / 25);   // ~25 Gram elements per CTA
+        ra.m[m].Pg = reinterpret_cast<double*>(w + pl->off_Pg[m]);
+        ra.m[m].U_prev = gram_U_prev + pl->u_off[m];
         max_chunks = std::max(max_chunks, ra.m[m].nchunk);
       }
     }
+    ra.factor = 1;
+    ra.Rf = reinterpret_cast<double*>(w + pl->off_Rf);
+    ra.counter = reinterpret_cast<int*>(w) + 20;
+    ra.status = reinterpret_cast<int*>(w);
     ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
-    return ASI_OK;      // the core kernel finishes the factorisation
+    return ASI_OK;      // the core kernel solves for the rows of U_m
   }
   if (pl->small_rank) {
     SmReduceArgs ra;
@@ -294,7 +308,7 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     SmCoreArgs c;
     c.act = act;
     c.U_new = U_new;
-    c.U_prev = gram_U_prev;
+    c.Rf = reinterpret_cast<const double*>(w + pl->off_Rf);
     c.Tp = reinterpret_cast<float*>(w + pl->off_T[0]);
     c.core = core;
     c.status = reinterpret_cast<int*>(w);
@@ -303,10 +317,8 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     c.gs = pl->fold_gs;
     c.Tg = reinterpret_cast<float*>(w + pl->off_T[1]);
     for (int m = 0; m < 4; ++m) {
-      c.Pred[m] = reinterpret_cast<const double*>(w + pl->off_Pred[m]);
-      c.Gp[m] = reinterpret_cast<const double*>(w + pl->off_Gp[m]);
-      c.nchunk[m] = pl->nchunk[m];
-      c.gram[m] = (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) ? 1 : 0;
+      const bool gram = gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2;
+      c.Pred[m] = reinterpret_cast<const double*>(w + (gram ? pl->off_Pg[m] : pl->off_Pred[m]));
       c.u_off[m] = pl->u_off[m];
       c.r[m] = pl->r[m];
     }

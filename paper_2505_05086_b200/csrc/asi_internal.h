@@ -103,19 +103,23 @@ struct SmReduceMode {
   const float* Pp;     // [nsplit][a][r], or [nsplit][a][a] Gram matrices A_m A_m^T when gram != 0
   double* Pred;        // [a][r], or [a][a] (the summed Gram matrix) when gram != 0
   double* Gp;          // [nchunk][r][r]
+  double* Pg;          // gram != 0 and factor != 0: [a][r], P_m = G_m U_m^prev
+  const float* U_prev; // gram != 0 and factor != 0: U_m^prev [a][r]
   int a, r, nsplit, nchunk, gram;
 };
+constexpr int kRfStride = 80;   // doubles per mode in Rf: rows of R_m at pitch 8, then 1 / diag(R_m) at [64..72)
 struct SmReduceArgs {
   SmReduceMode m[ASI_MAX_MODES];
+  int factor;          // != 0: the last CTA of each mode factors G_m = R_m^T R_m into Rf (ranks <= 8)
+  double* Rf;          // [modes][kRfStride]
+  int* counter;        // one per mode, zero on entry, zero again on exit
+  int* status;
 };
-// Finishes Orthogonalize (Cholesky of G_m, U_m = P_m R_m^{-1}) in its prologue, then the core.
+// Finishes Orthogonalize (U_m = P_m R_m^{-1}, rows it needs) in its prologue, then the core.
 struct SmCoreArgs {
   const void* act;
-  const double* Pred[ASI_MAX_MODES];
-  const double* Gp[ASI_MAX_MODES];
-  int nchunk[ASI_MAX_MODES];
-  int gram[ASI_MAX_MODES];      // != 0: Pred[m] holds G_m = A_m A_m^T (a x a), P_m = G_m U_prev is formed here
-  const float* U_prev;
+  const double* Pred[ASI_MAX_MODES];   // P_m [a][r] in fp64
+  const double* Rf;                    // [4][kRfStride]: the Cholesky factors written by the reduction kernel
   float* U_new;
   float* Tp;                    // [n_tiles][core_elems] per-tile partial cores
   float* Tg;                    // [ceil(n_tiles / gs)][core_elems] per-group partial cores
@@ -206,6 +210,7 @@ struct asi_plan {
 
   // compress workspace (byte offsets)
   size_t off_V, off_Pp[ASI_MAX_MODES], off_Pred[ASI_MAX_MODES], off_Gp[ASI_MAX_MODES], off_T[2];
+  size_t off_Rf, off_Pg[ASI_MAX_MODES];
   int nsplit[ASI_MAX_MODES], nchunk[ASI_MAX_MODES];
   int64_t q_per_split[ASI_MAX_MODES];
   int core_order[ASI_MAX_MODES];

@@ -689,8 +689,10 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
 // k_sm_reduce: CTA (c, m) sums rows [16 c, 16 c + 16) of the per-tile partials of P_m in fp64 in a
 // fixed order (thread (e, sg) takes the partials s == sg (mod SG); the SG sums meet in shared memory
 // in index order), stores them in fp64 and adds its share of P_m^T P_m.  A mode whose partials are
-// Gram matrices A_m A_m^T (a <= 16) is summed the same way, a slice of the a x a elements per CTA,
-// and left in fp64 for the core kernel.
+// Gram matrices A_m A_m^T (a <= 16) is summed the same way, a slice of the a x a elements per CTA.
+// With args.factor the last CTA of a mode to finish then factors the mode once for all CTAs of the
+// core kernel: it sums the shares of P_m^T P_m (a Gram mode: forms P_m = G_m U_m^prev first), and
+// leaves the Cholesky factor R_m and 1 / diag(R_m) in args.Rf.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   constexpr int RM = 8, RPC = kRedRows;
@@ -737,18 +739,108 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
       Ps[k][j] = v;
     }
   }
-  if (M.gram) return;                              // the core kernel forms P_m = G_m U_m^prev itself
-  __syncthreads();
-  if (tid < r * r) {
-    const FDiv dr(r);
-    int i, j;
-    dr.divmod(tid, i, j);
-    double g = 0.0;
-    if (j >= i) {
+  if (!M.gram) {
+    __syncthreads();
+    if (tid < r * r) {
+      const FDiv dr(r);
+      int i, j;
+      dr.divmod(tid, i, j);
+      double g = 0.0;
+      if (j >= i) {
 #pragma unroll 4
-      for (int rl = 0; rl < RPC; ++rl) g = fma(Ps[rl][i], Ps[rl][j], g);
+        for (int rl = 0; rl < RPC; ++rl) g = fma(Ps[rl][i], Ps[rl][j], g);
+      }
+      M.Gp[((int64_t)c * r + i) * r + j] = g;
     }
-    M.Gp[((int64_t)c * r + i) * r + j] = g;
+  }
+  if (!args.factor) return;
+  // ---- the last CTA of a mode to get here factors the mode once for every CTA of the core kernel:
+  // G_m = P_m^T P_m = R_m^T R_m (Cholesky), stored as the rows of R_m and 1 / diag(R_m)
+  __shared__ int s_last;
+  __shared__ double Gq[8][RM * RM];
+  __shared__ double Gs[RM][RM + 1];
+  __shared__ double Dinv[RM];
+  __shared__ double Gfull[16 * 16];
+  __shared__ double Pm[16][RM];
+  __shared__ float Ups[16 * RM];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(args.counter + blockIdx.y, 1) == M.nchunk - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const int lane = tid & 31, warp = tid >> 5;
+  if (!M.gram) {
+    // warp q sums the shares of the chunks == q (mod 8); the eight sums meet in index order
+    for (int e = lane; e < r * r; e += 32) {
+      double g = 0.0;
+#pragma unroll 8
+      for (int cc = warp; cc < M.nchunk; cc += 8) g += __ldcg(M.Gp + (int64_t)cc * r * r + e);
+      Gq[warp][e] = g;
+    }
+    __syncthreads();
+    if (tid < r * r) {
+      double g = Gq[0][tid];
+#pragma unroll
+      for (int q = 1; q < 8; ++q) g += Gq[q][tid];
+      const int i = tid / r, k = tid - i * r;
+      Gs[i][k] = g;
+    }
+  } else {
+    // Gram mode (a <= 16): P_m = G_m U_m^prev (Algorithm 1: A_m (A_m^T U)), kept in fp64 for the row
+    // solves of the core kernel, then its Gram matrix
+    for (int e = tid; e < a * a; e += kRedNT) Gfull[e] = __ldcg(M.Pred + e);
+    for (int e = tid; e < a * r; e += kRedNT) Ups[e] = __ldg(M.U_prev + e);
+    __syncthreads();
+    if (tid < a * r) {
+      const int k = tid / r, j = tid - k * r;
+      double v = 0.0;
+      for (int k2 = 0; k2 < a; ++k2) v = fma(Gfull[k * a + k2], (double)Ups[k2 * r + j], v);
+      Pm[k][j] = v;
+      M.Pg[tid] = v;
+    }
+    __syncthreads();
+    if (tid < r * r) {
+      const int i = tid / r, k = tid - i * r;
+      double g = 0.0;
+      if (k >= i)
+        for (int kk = 0; kk < a; ++kk) g = fma(Pm[kk][i], Pm[kk][k], g);
+      Gs[i][k] = g;
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    // right-looking Cholesky G = R^T R on one warp; lane owns entries e0 = lane and e1 = lane + 32
+    const int e0 = lane, e1 = lane + 32;
+    const int i0 = e0 / r, k0 = e0 - i0 * r, i1 = e1 / r, k1 = e1 - i1 * r;
+    const bool in0 = e0 < r * r, in1 = e1 < r * r;
+    double trace = 0.0;
+    for (int i = 0; i < r; ++i) trace += Gs[i][i];
+    const double floor_d = 1e-12 * trace;
+    for (int j = 0; j < r; ++j) {
+      double d = Gs[j][j];
+      if (!(d > floor_d)) {
+        if (lane == 0) atomicMax(args.status, (int)ASI_ERR_RANK_DEFICIENT);
+        d = (floor_d > 0.0) ? floor_d : 1.0;
+      }
+      const double inv = rsqrt(d);
+      __syncwarp();
+      if (lane == j) {
+        Gs[j][j] = d * inv;
+        Dinv[j] = inv;
+      } else if (lane > j && lane < r) {
+        Gs[j][lane] *= inv;
+      }
+      __syncwarp();
+      if (in0 && i0 > j && k0 >= i0) Gs[i0][k0] -= Gs[j][i0] * Gs[j][k0];
+      if (in1 && i1 > j && k1 >= i1) Gs[i1][k1] -= Gs[j][i1] * Gs[j][k1];
+      __syncwarp();
+    }
+    double* Rf = args.Rf + blockIdx.y * kRfStride;
+    if (in0) Rf[i0 * RM + k0] = Gs[i0][k0];
+    if (in1) Rf[i1 * RM + k1] = Gs[i1][k1];
+    if (lane < r) Rf[RM * RM + lane] = Dinv[lane];
+    if (lane == 0) args.counter[blockIdx.y] = 0;
   }
 }
 
@@ -780,10 +872,9 @@ cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cuda
 
 // ---------------------------------------------------------------------------------------------
 // k_sm_core.  Tile t = [all B x J] as in role B of the first pass.
-//   prologue (while the tile is in flight): each thread fetches the fp64 row of P_m it will solve
-//     for; warps 4m..4m+3 sum the Gram shares of mode m and warp 4m factors G_m = R_m^T R_m; then
-//     one thread per needed factor row solves u = p R_m^{-1} -- all of U_1, the tile's own rows of
-//     U_2, all of U_3 and U_4 -- and the owners write them to U_new;
+//   prologue (while the tile is in flight): one thread per needed factor row fetches the fp64 row of
+//     P_m and solves u = p R_m^{-1} with the Cholesky factor the reduction kernel left -- all of U_1,
+//     the tile's own rows of U_2, all of U_3 and U_4 -- and the owners write them to U_new;
 //   W[i][c,h,w] = sum_b U1[b,i] X[b][c,h,w];  Y[i,j][h,w] = sum_c U2[c,j] W[i][c,h,w];
 //   T[i,j,k,l] = Y x_3 U3^T x_4 U4^T  -> per-tile partial core, summed in two ordered levels.
 // ---------------------------------------------------------------------------------------------
@@ -796,12 +887,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   constexpr int NH = batch_groups(kNT, J);
   extern __shared__ __align__(128) float smem[];
   __shared__ int s_last;
-  __shared__ double Gq[4][4][R * R];
-  __shared__ double Gs[4][R][R + 1];
-  __shared__ double Dinv[4][R];
-  __shared__ double Gfull[2][S * S];    // A_m A_m^T of a Gram mode (m = 3, 4)
-  __shared__ double Pm[2][S][R];        // and its P_m = G_m U_m^prev
-  __shared__ float Ups[2][S * R];       // U_m^prev of a Gram mode
+  __shared__ double Rs[4][kRfStride];   // per mode: rows of R_m (pitch 8), then 1 / diag(R_m) at [64..]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, C = p.C, tile = blockIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
@@ -831,85 +917,13 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     else if (tid < B + CC + S) { rm = 2; rk = tid - B - CC; rdst = U3s + rk * R; rowner = tile == 0; }
     else { rm = 3; rk = tid - B - CC - S; rdst = U4s + rk * R; rowner = tile == 0; }
     rr = p.r[rm];
-    if (!p.gram[rm]) {
-      const double* src = p.Pred[rm] + (int64_t)rk * rr;
+    const double* src = p.Pred[rm] + (int64_t)rk * rr;
 #pragma unroll
-      for (int j = 0; j < R; ++j)
-        if (j < rr) prow[j] = __ldcg(src + j);
-    }
+    for (int j = 0; j < R; ++j)
+      if (j < rr) prow[j] = __ldcg(src + j);
   }
-  // ---- Gram shares: warp 4m + q sums the chunks == q (mod 4) of mode m
-  {
-    const int m = warp >> 2, q = warp & 3, r = p.r[m];
-    if (!p.gram[m]) {
-      const double* Gp = p.Gp[m];
-      const int nch = p.nchunk[m];
-      for (int e = lane; e < r * r; e += 32) {
-        double g = 0.0;
-#pragma unroll 8
-        for (int cc = q; cc < nch; cc += 4) g += __ldcg(Gp + (int64_t)cc * r * r + e);
-        Gq[m][q][e] = g;
-      }
-    } else {
-      // Gram mode (m = 2, 3; a = S): the four warps fetch G_m = A_m A_m^T
-      for (int e = q * 32 + lane; e < S * S; e += 128) Gfull[m - 2][e] = __ldcg(p.Pred[m] + e);
-      for (int e = q * 32 + lane; e < S * r; e += 128) Ups[m - 2][e] = __ldg(p.U_prev + p.u_off[m] + e);
-    }
-  }
-  __syncthreads();
-  if ((warp & 3) == 0) {
-    // right-looking Cholesky G = R^T R on one warp; lane owns entries e0 = lane and e1 = lane + 32
-    const int m = warp >> 2, r = p.r[m];
-    const int e0 = lane, e1 = lane + 32;
-    const int i0 = e0 / r, k0 = e0 - i0 * r, i1 = e1 / r, k1 = e1 - i1 * r;
-    const bool in0 = e0 < r * r, in1 = e1 < r * r;
-    if (!p.gram[m]) {
-      if (in0) Gs[m][i0][k0] = ((Gq[m][0][e0] + Gq[m][1][e0]) + Gq[m][2][e0]) + Gq[m][3][e0];
-      if (in1) Gs[m][i1][k1] = ((Gq[m][0][e1] + Gq[m][1][e1]) + Gq[m][2][e1]) + Gq[m][3][e1];
-    } else {
-      // P_m = G_m U_m^prev (Algorithm 1: A_m (A_m^T U)), then its Gram matrix
-      for (int e = lane; e < S * r; e += 32) {
-        const int k = e / r, j = e - k * r;
-        double v = 0.0;
-        for (int k2 = 0; k2 < S; ++k2) v = fma(Gfull[m - 2][k * S + k2], (double)Ups[m - 2][k2 * r + j], v);
-        Pm[m - 2][k][j] = v;
-      }
-      __syncwarp();
-      if (in0 && k0 >= i0) {
-        double g = 0.0;
-        for (int k = 0; k < S; ++k) g = fma(Pm[m - 2][k][i0], Pm[m - 2][k][k0], g);
-        Gs[m][i0][k0] = g;
-      }
-      if (in1 && k1 >= i1) {
-        double g = 0.0;
-        for (int k = 0; k < S; ++k) g = fma(Pm[m - 2][k][i1], Pm[m - 2][k][k1], g);
-        Gs[m][i1][k1] = g;
-      }
-    }
-    __syncwarp();
-    double trace = 0.0;
-    for (int i = 0; i < r; ++i) trace += Gs[m][i][i];
-    const double floor_d = 1e-12 * trace;
-    for (int j = 0; j < r; ++j) {
-      double d = Gs[m][j][j];
-      if (!(d > floor_d)) {
-        if (blockIdx.x == 0 && lane == 0) atomicMax(p.status, (int)ASI_ERR_RANK_DEFICIENT);
-        d = (floor_d > 0.0) ? floor_d : 1.0;
-      }
-      const double inv = rsqrt(d);
-      __syncwarp();
-      if (lane == j) {
-        Gs[m][j][j] = d * inv;
-        Dinv[m][j] = inv;
-      } else if (lane > j && lane < r) {
-        Gs[m][j][lane] *= inv;
-      }
-      __syncwarp();
-      if (in0 && i0 > j && k0 >= i0) Gs[m][i0][k0] -= Gs[m][j][i0] * Gs[m][j][k0];
-      if (in1 && i1 > j && k1 >= i1) Gs[m][i1][k1] -= Gs[m][j][i1] * Gs[m][j][k1];
-      __syncwarp();
-    }
-  }
+  // ---- the Cholesky factors of the four modes (computed once, by the reduction kernel)
+  for (int e = tid; e < 4 * kRfStride; e += kNT) (&Rs[0][0])[e] = __ldcg(p.Rf + e);
   __syncthreads();
   if (tid < nrows) {
     float* gdst = p.U_new + p.u_off[rm] + (int64_t)rk * rr;
@@ -918,11 +932,11 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
     for (int j = 0; j < R; ++j) {
       float out = 0.f;
       if (j < rr) {
-        double v = p.gram[rm] ? Pm[rm - 2][rk][j] : prow[j];
+        double v = prow[j];
 #pragma unroll
         for (int i = 0; i < R; ++i)
-          if (i < j) v -= q[i] * Gs[rm][i][j];
-        v *= Dinv[rm][j];
+          if (i < j) v -= q[i] * Rs[rm][i * 8 + j];
+        v *= Rs[rm][64 + j];
         q[j] = v;
         out = (float)v;
         if (rowner) gdst[j] = out;
