@@ -1014,17 +1014,44 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  for (int idx = tid; idx < ce; idx += kNT) {
-    const float* src = p.Tg + idx;
-    float s = 0.f;
-    for (int g0 = 0; g0 < ngroups; g0 += 16) {
-      float v[16];
+  if (ce * 2 <= kNT) {
+    // few core elements: thread (e, q) sums the groups == q (mod nq) of element e, the nq sums meet
+    // in index order (shared memory: the tile is no longer needed)
+    int nq = kNT / ce;
+    nq = nq > 8 ? 8 : nq;
+    float* fold = smem;                              // [nq][ce]
+    if (tid < nq * ce) {
+      const int q = tid / ce, e = tid - q * ce;
+      const float* src = p.Tg + e;
+      float s = 0.f;
+      for (int g0 = q; g0 < ngroups; g0 += 8 * nq) {
+        float v[8];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) v[k] = (g0 + k < ngroups) ? __ldcg(src + (int64_t)(g0 + k) * ce) : 0.f;
+        for (int k = 0; k < 8; ++k) v[k] = (g0 + k * nq < ngroups) ? __ldcg(src + (int64_t)(g0 + k * nq) * ce) : 0.f;
 #pragma unroll
-      for (int k = 0; k < 16; ++k) s += v[k];
+        for (int k = 0; k < 8; ++k) s += v[k];
+      }
+      fold[tid] = s;
     }
-    p.core[idx] = s;
+    __syncthreads();
+    if (tid < ce) {
+      float s = fold[tid];
+      for (int q = 1; q < nq; ++q) s += fold[q * ce + tid];
+      p.core[tid] = s;
+    }
+  } else {
+    for (int idx = tid; idx < ce; idx += kNT) {
+      const float* src = p.Tg + idx;
+      float s = 0.f;
+      for (int g0 = 0; g0 < ngroups; g0 += 16) {
+        float v[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = (g0 + k < ngroups) ? __ldcg(src + (int64_t)(g0 + k) * ce) : 0.f;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) s += v[k];
+      }
+      p.core[idx] = s;
+    }
   }
   if (tid == 0) *p.counter = 0;
 }
