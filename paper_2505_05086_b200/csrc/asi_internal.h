@@ -87,7 +87,7 @@ struct ConvTailArgs {
 };
 
 // Fused small-map conv kernels (asi_smallmap_kernels.cu)
-constexpr int kRedRows = 16;         // rows of P per CTA in the partial-reduction kernel
+constexpr int kRedRows = 8;          // rows of P per CTA in the partial-reduction kernel
 struct SmPass1Args {
   const void* act;
   const float* U_prev;

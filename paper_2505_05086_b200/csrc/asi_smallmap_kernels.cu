@@ -772,7 +772,7 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   const int lane = tid & 31, warp = tid >> 5;
   if (!M.gram) {
     // warp q sums the shares of the chunks == q (mod 8); the eight sums meet in index order
-    for (int e = lane; e < r * r; e += 32) {
+    for (int e = lane; e < r * r && warp < 8; e += 32) {
       double g = 0.0;
 #pragma unroll 8
       for (int cc = warp; cc < M.nchunk; cc += 8) g += __ldcg(M.Gp + (int64_t)cc * r * r + e);
