@@ -52,7 +52,7 @@ void choose_kernels(asi_plan* pl) {
     const int Cout = pl->d.cout;
     const int64_t HoWo = pl->Ho * pl->Wo;
     // channels per CTA: the smallest count that makes a staged row a multiple of 16 bytes (rows can
-    // then be staged by the bulk-copy engine); failing that, the smallest that makes it even
+    // then be staged by 16-byte asynchronous copies); failing that, the smallest that makes it even
     int cpb = 0;
     bool rows_ok = false;
     for (int c = 1; c <= 4 && !cpb; c *= 2)
@@ -519,7 +519,7 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
   if (pl->fast_compress) {
-    // fp32 tiles are staged by the bulk-copy engine, which needs 16-byte aligned sources
+    // fp32 tiles are staged by 16-byte asynchronous copies, which need 16-byte aligned sources
     if (!pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
     SmPass1Args a;
     a.act = act;

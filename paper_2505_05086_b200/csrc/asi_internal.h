@@ -142,7 +142,7 @@ struct SmWgradArgs {
   int r[ASI_MAX_MODES];
   int B, C, Cout, H, W, Ho, Wo, kh, kw, sh, sw, ph, pw, groups, cpb;
   int pj;                       // row pitch (floats) of the staged dY tile
-  int bulk;                     // 1: rows staged by the bulk-copy engine (fp32, 16-byte aligned rows)
+  int bulk;                     // 1: rows staged by 16-byte asynchronous copies (fp32, 16-byte aligned rows)
   int ncl;                      // output channels expanded per round of term 5 (divides cpb)
   int bulk_store;               // 1: dW row blocks leave through the bulk-copy engine (16-byte sized and aligned)
 };

@@ -1058,7 +1058,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
 
 // ---------------------------------------------------------------------------------------------
 // k_sm_wgrad: CTA owns cpb consecutive output channels, i.e. the dY tile [B x J], J = cpb*Ho*Wo
-// contiguous values per sample (staged by the bulk-copy engine when fp32).
+// contiguous values per sample (staged by 16-byte cp.async when fp32 and 16-byte aligned).
 //   Z3 = core x_3 U3 x_4 U4 (recomputed per CTA while the tile is in flight);
 //   Z1 = dY x_1 U1^T on the CTA's channels;
 //   Z4[c',j,kh,kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p];  dW = Z4 x_2 U2.
