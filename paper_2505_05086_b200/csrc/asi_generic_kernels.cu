@@ -19,6 +19,20 @@ ProfState g_prof = {0, nullptr, 0, 0, 0.0};
 
 __device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+// four neighbouring values read once (streaming hint), as fp32
+template <typename TX>
+__device__ __forceinline__ float4 ld4_stream(const TX* p);
+template <>
+__device__ __forceinline__ float4 ld4_stream<float>(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+template <>
+__device__ __forceinline__ float4 ld4_stream<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(p));
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
 
 // ---------------------------------------------------------------------------------------------
 // Tile loader: Xs[kl][ql] = X(k0 + kl, q0 + ql), zero outside [0,a) x [q0, q_end).
@@ -223,11 +237,81 @@ static cudaError_t launch_gemm_t(const GemmArgs& g, int nsplit, cudaStream_t st)
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// k_rowstream: the first-mode product Y[j][q] = sum_k B(k, j) X[k][q] (O = 1: row k of X is one
+// contiguous slab of Q values) with n_out <= R <= 8.  Pure streaming: a thread owns four neighbouring
+// columns and walks down the a rows with UNR 16-byte loads in flight; the factor sits in shared
+// memory.  X is read exactly once, coalesced; nothing else of size moves.
+// ---------------------------------------------------------------------------------------------
+template <int R, typename TX>
+__global__ void __launch_bounds__(128) k_rowstream(ModeProdArgs p) {
+  constexpr int NT = 128, UNR = 8;
+  extern __shared__ __align__(16) float Bsm[];       // [a][R], zero-padded
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < (int)p.a * R; idx += NT) {
+    const int k = idx / R, j = idx % R;
+    Bsm[idx] = (j < p.n_out) ? p.B[k * p.ldb_k + j * p.ldb_j] : 0.f;
+  }
+  __syncthreads();
+  const int64_t q = ((int64_t)blockIdx.x * NT + tid) * 4;
+  if (q >= p.Q) return;
+  const TX* X = reinterpret_cast<const TX*>(p.X) + q;
+  float acc[4][R];
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+#pragma unroll
+    for (int j = 0; j < R; ++j) acc[c][j] = 0.f;
+  const int a = (int)p.a;
+  int k0 = 0;
+  for (; k0 + UNR <= a; k0 += UNR) {
+    float4 x[UNR];
+#pragma unroll
+    for (int u = 0; u < UNR; ++u) x[u] = ld4_stream<TX>(X + (int64_t)(k0 + u) * p.Q);
+#pragma unroll
+    for (int u = 0; u < UNR; ++u) {
+#pragma unroll
+      for (int j = 0; j < R; j += 4) {
+        const float4 b = *reinterpret_cast<const float4*>(Bsm + (k0 + u) * R + j);
+        const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          acc[c][j] = fmaf(xs[c], b.x, acc[c][j]);
+          acc[c][j + 1] = fmaf(xs[c], b.y, acc[c][j + 1]);
+          acc[c][j + 2] = fmaf(xs[c], b.z, acc[c][j + 2]);
+          acc[c][j + 3] = fmaf(xs[c], b.w, acc[c][j + 3]);
+        }
+      }
+    }
+  }
+  for (; k0 < a; ++k0) {
+    const float4 xv = ld4_stream<TX>(X + (int64_t)k0 * p.Q);
+    const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+      const float b = Bsm[k0 * R + j];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[c][j] = fmaf(xs[c], b, acc[c][j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < R; ++j)
+    if (j < p.n_out)
+      *reinterpret_cast<float4*>(p.Y + (int64_t)j * p.sj + q) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+}
+
 template <typename TX>
 static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
   if (p.Q <= 0 || p.n_out <= 0) return cudaSuccess;
   ProfScope prof(ASI_K_MODEPROD, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
+  if (p.O == 1 && p.n_out <= 8 && p.si == 1 && p.Q % 4 == 0 && p.sj % 4 == 0 && p.Q >= (1 << 16) &&
+      p.a <= 1024 && p.a >= 8 && (reinterpret_cast<uintptr_t>(p.X) & 15u) == 0 &&
+      (reinterpret_cast<uintptr_t>(p.Y) & 15u) == 0) {
+    const unsigned grid = (unsigned)((p.Q / 4 + 127) / 128);
+    if (p.n_out <= 4) k_rowstream<4, TX><<<grid, 128, (size_t)p.a * 4 * 4, st>>>(p);
+    else k_rowstream<8, TX><<<grid, 128, (size_t)p.a * 8 * 4, st>>>(p);
+    return cudaGetLastError();
+  }
   if (p.I == 1 && p.n_out >= 16 && p.n_out <= 64 && p.a >= 64 && p.Q >= 64 && p.sj == 1 && p.so == p.n_out &&
       p.ldb_k == p.n_out && p.ldb_j == 1 && p.Q < (1 << 30) && p.a < (1 << 30)) {
     GemmArgs g = {p.X, p.B, p.Y, (int)p.Q, p.n_out, (int)p.a, p.a, (int)p.a, 0};
