@@ -240,63 +240,91 @@ static cudaError_t launch_gemm_t(const GemmArgs& g, int nsplit, cudaStream_t st)
 // ---------------------------------------------------------------------------------------------
 // k_rowstream: the first-mode product Y[j][q] = sum_k B(k, j) X[k][q] (O = 1: row k of X is one
 // contiguous slab of Q values) with n_out <= R <= 8.  Pure streaming: a thread owns four neighbouring
-// columns and walks down the a rows with UNR 16-byte loads in flight; the factor sits in shared
-// memory.  X is read exactly once, coalesced; nothing else of size moves.
+// columns and one of KS slices of the rows, and walks down its rows with UNR 16-byte loads in flight
+// (a single thread walking all rows is bound by the latency of its own loads); the KS partial sums
+// meet in shared memory in slice order.  The factor sits in shared memory.  X is read exactly once,
+// coalesced; nothing else of size moves.
 // ---------------------------------------------------------------------------------------------
 template <int R, typename TX>
-__global__ void __launch_bounds__(128) k_rowstream(ModeProdArgs p) {
-  constexpr int NT = 128, UNR = 8;
-  extern __shared__ __align__(16) float Bsm[];       // [a][R], zero-padded
+__global__ void __launch_bounds__(256) k_rowstream(ModeProdArgs p) {
+  constexpr int NT = 256, CG = 64, KS = NT / CG, UNR = 8;
+  extern __shared__ __align__(16) float rs_smem[];
+  float* Bsm = rs_smem;                              // [a][R], zero-padded
+  float* part = rs_smem + (((int)p.a * R + 3) & ~3); // [KS - 1][CG][4 R]
   const int tid = threadIdx.x;
   for (int idx = tid; idx < (int)p.a * R; idx += NT) {
     const int k = idx / R, j = idx % R;
     Bsm[idx] = (j < p.n_out) ? p.B[k * p.ldb_k + j * p.ldb_j] : 0.f;
   }
   __syncthreads();
-  const int64_t q = ((int64_t)blockIdx.x * NT + tid) * 4;
-  if (q >= p.Q) return;
-  const TX* X = reinterpret_cast<const TX*>(p.X) + q;
+  const int cg = tid & (CG - 1), ks = tid / CG;
+  const int64_t q = ((int64_t)blockIdx.x * CG + cg) * 4;
+  const bool live = q < p.Q;
   float acc[4][R];
 #pragma unroll
   for (int c = 0; c < 4; ++c)
 #pragma unroll
     for (int j = 0; j < R; ++j) acc[c][j] = 0.f;
   const int a = (int)p.a;
-  int k0 = 0;
-  for (; k0 + UNR <= a; k0 += UNR) {
-    float4 x[UNR];
+  const int kper = (a + KS - 1) / KS;
+  int k0 = ks * kper;
+  const int k1 = (k0 + kper < a) ? k0 + kper : a;
+  if (live) {
+    const TX* X = reinterpret_cast<const TX*>(p.X) + q;
+    for (; k0 + UNR <= k1; k0 += UNR) {
+      float4 x[UNR];
 #pragma unroll
-    for (int u = 0; u < UNR; ++u) x[u] = ld4_stream<TX>(X + (int64_t)(k0 + u) * p.Q);
+      for (int u = 0; u < UNR; ++u) x[u] = ld4_stream<TX>(X + (int64_t)(k0 + u) * p.Q);
 #pragma unroll
-    for (int u = 0; u < UNR; ++u) {
-#pragma unroll
-      for (int j = 0; j < R; j += 4) {
-        const float4 b = *reinterpret_cast<const float4*>(Bsm + (k0 + u) * R + j);
+      for (int u = 0; u < UNR; ++u) {
         const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          acc[c][j] = fmaf(xs[c], b.x, acc[c][j]);
-          acc[c][j + 1] = fmaf(xs[c], b.y, acc[c][j + 1]);
-          acc[c][j + 2] = fmaf(xs[c], b.z, acc[c][j + 2]);
-          acc[c][j + 3] = fmaf(xs[c], b.w, acc[c][j + 3]);
+        for (int j = 0; j < R; j += 4) {
+          const float4 b = *reinterpret_cast<const float4*>(Bsm + (k0 + u) * R + j);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            acc[c][j] = fmaf(xs[c], b.x, acc[c][j]);
+            acc[c][j + 1] = fmaf(xs[c], b.y, acc[c][j + 1]);
+            acc[c][j + 2] = fmaf(xs[c], b.z, acc[c][j + 2]);
+            acc[c][j + 3] = fmaf(xs[c], b.w, acc[c][j + 3]);
+          }
         }
       }
     }
-  }
-  for (; k0 < a; ++k0) {
-    const float4 xv = ld4_stream<TX>(X + (int64_t)k0 * p.Q);
-    const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
+    for (; k0 < k1; ++k0) {
+      const float4 xv = ld4_stream<TX>(X + (int64_t)k0 * p.Q);
+      const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
-    for (int j = 0; j < R; ++j) {
-      const float b = Bsm[k0 * R + j];
+      for (int j = 0; j < R; ++j) {
+        const float b = Bsm[k0 * R + j];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) acc[c][j] = fmaf(xs[c], b, acc[c][j]);
+        for (int c = 0; c < 4; ++c) acc[c][j] = fmaf(xs[c], b, acc[c][j]);
+      }
     }
   }
+  if (ks > 0) {
+    float* dst = part + ((ks - 1) * CG + cg) * 4 * R;
 #pragma unroll
-  for (int j = 0; j < R; ++j)
-    if (j < p.n_out)
-      *reinterpret_cast<float4*>(p.Y + (int64_t)j * p.sj + q) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int j = 0; j < R; j += 4)
+        *reinterpret_cast<float4*>(dst + c * R + j) = make_float4(acc[c][j], acc[c][j + 1], acc[c][j + 2], acc[c][j + 3]);
+  }
+  __syncthreads();
+  if (ks == 0 && live) {
+#pragma unroll 1
+    for (int s = 1; s < KS; ++s) {
+      const float* src = part + ((s - 1) * CG + cg) * 4 * R;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int j = 0; j < R; ++j) acc[c][j] += src[c * R + j];
+    }
+#pragma unroll
+    for (int j = 0; j < R; ++j)
+      if (j < p.n_out)
+        *reinterpret_cast<float4*>(p.Y + (int64_t)j * p.sj + q) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+  }
 }
 
 template <typename TX>
@@ -305,11 +333,12 @@ static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_MODEPROD, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
   if (p.O == 1 && p.n_out <= 8 && p.si == 1 && p.Q % 4 == 0 && p.sj % 4 == 0 && p.Q >= (1 << 16) &&
-      p.a <= 1024 && p.a >= 8 && (reinterpret_cast<uintptr_t>(p.X) & 15u) == 0 &&
+      p.a <= 512 && p.a >= 8 && (reinterpret_cast<uintptr_t>(p.X) & 15u) == 0 &&
       (reinterpret_cast<uintptr_t>(p.Y) & 15u) == 0) {
-    const unsigned grid = (unsigned)((p.Q / 4 + 127) / 128);
-    if (p.n_out <= 4) k_rowstream<4, TX><<<grid, 128, (size_t)p.a * 4 * 4, st>>>(p);
-    else k_rowstream<8, TX><<<grid, 128, (size_t)p.a * 8 * 4, st>>>(p);
+    const unsigned grid = (unsigned)((p.Q / 4 + 63) / 64);
+    const auto smem = [&](int R) { return (size_t)((((int)p.a * R + 3) & ~3) + 3 * 64 * 4 * R) * 4; };
+    if (p.n_out <= 4) k_rowstream<4, TX><<<grid, 256, smem(4), st>>>(p);
+    else k_rowstream<8, TX><<<grid, 256, smem(8), st>>>(p);
     return cudaGetLastError();
   }
   if (p.I == 1 && p.n_out >= 16 && p.n_out <= 64 && p.a >= 64 && p.Q >= 64 && p.sj == 1 && p.so == p.n_out &&
