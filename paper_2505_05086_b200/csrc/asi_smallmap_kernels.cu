@@ -1169,12 +1169,12 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   float* U2s = U1s + p.B * R;                        // [C][R]
   float* Z1s = U2s + p.C * R;                        // [J][R]
   float* part = Z1s + J * R;                         // [NH][J][R] (NH > 1 only)
-  float* Ss = part + (NH > 1 ? NH : 0) * J * R;      // [r1 r2 r3 r4]
-  float* U3s = Ss + r1 * r2 * r3 * r4;               // [H][r3]
-  float* U4s = U3s + H * r3;                         // [W][r4]
-  float* Tm = U4s + W * r4;                          // [r1 r2][H][r4]
+  float* Ss = part + (NH > 1 ? NH : 0) * J * R;      // [r1 r2][R (l)][R (k)]: core, modes 3 and 4 swapped, zero-padded
+  float* U3s = Ss + r1 * r2 * R * R;                 // [H][R]
+  float* U4s = U3s + H * R;                          // [W][R]
+  float* Tm = U4s + W * R;                           // [r1 r2][H][R]
   const int Hp = H + 2 * p.ph, Wp = W + 2 * p.pw;    // Z3 is kept zero-padded: term 4 needs no bounds logic
-  float* Z3s = Tm + r1 * r2 * H * r4;                // [r1 r2][Hp][Wp]
+  float* Z3s = Tm + r1 * r2 * H * R;                 // [r1 r2][Hp][Wp]
   float* Z4s = smem + ((Z3s + r1 * r2 * Hp * Wp) - smem + 3) / 4 * 4;   // [cpb][kk][R], 16-byte aligned (rank index fastest, zero-padded)
   float* red = Z4s + p.cpb * kk * R;                 // [G4][cpb][r2 kk]
 
@@ -1182,9 +1182,14 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   const int64_t sstride = (int64_t)p.Cout * HoWo;
   const bool bulk = std::is_same<TX, float>::value && p.bulk;
   {
-    fac_issue_flat(p.core, Ss, r1 * r2 * r3 * r4);
-    fac_issue_flat(p.U + p.u_off[2], U3s, H * r3);
-    fac_issue_flat(p.U + p.u_off[3], U4s, W * r4);
+#pragma unroll 1
+    for (int idx = tid; idx < r1 * r2 * R * R; idx += kNT) {      // Ss[ij][l][k] = core[ij][k][l]
+      const int k = idx % R, l = (idx / R) % R, ij = idx / (R * R);
+      const bool in = k < r3 && l < r4;
+      cp_async4(Ss + idx, p.core + (in ? (ij * r3 + k) * r4 + l : 0), in ? 4 : 0);
+    }
+    fac_issue_padded<R>(p.U + p.u_off[2], U3s, H, r3);
+    fac_issue_padded<R>(p.U + p.u_off[3], U4s, W, r4);
     fac_issue_padded<R>(p.U + p.u_off[0], U1s, p.B, r1);
     fac_issue_padded<R>(p.U + p.u_off[1], U2s, p.C, r2);
     cp_async_commit();                               // group 1: factors and core; group 0 (younger): the tile
@@ -1202,13 +1207,20 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   }
   __syncthreads();
   // terms 2-3: Tm[ij][h][l] = sum_k S[ij][k][l] U3[h][k];  Z3[ij][h][w] = sum_l Tm[ij][h][l] U4[w][l]
-  const FDiv d_r4(r4), d_H(H), d_Wp(Wp), d_Hp(Hp), d_kk(kk), d_kw(p.kw);
-  for (int idx = tid; idx < r1 * r2 * H * r4; idx += kNT) {
-    int t0, l, ij, h;
-    d_r4.divmod(idx, t0, l);
+  // (rank indices padded to R with zeros: every sum is a fixed-length dot product of 16-byte reads)
+  const FDiv d_H(H), d_Wp(Wp), d_Hp(Hp), d_kk(kk), d_kw(p.kw);
+  for (int idx = tid; idx < r1 * r2 * H * R; idx += kNT) {
+    const int l = idx % R, t0 = idx / R;
+    int ij, h;
     d_H.divmod(t0, ij, h);
+    const float* sp = Ss + (ij * R + l) * R;
+    const float* up = U3s + h * R;
     float s = 0.f;
-    for (int k = 0; k < r3; ++k) s = fmaf(Ss[(ij * r3 + k) * r4 + l], U3s[h * r3 + k], s);
+#pragma unroll
+    for (int k = 0; k < R; k += 4) {
+      const float4 a = *reinterpret_cast<const float4*>(sp + k), b = *reinterpret_cast<const float4*>(up + k);
+      s = fmaf(a.x, b.x, s); s = fmaf(a.y, b.y, s); s = fmaf(a.z, b.z, s); s = fmaf(a.w, b.w, s);
+    }
     Tm[idx] = s;
   }
   __syncthreads();
@@ -1218,8 +1230,15 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
     d_Hp.divmod(t0, ij, hp);
     const int h = hp - p.ph, w = wp - p.pw;
     float s = 0.f;
-    if (h >= 0 && h < H && w >= 0 && w < W)
-      for (int l = 0; l < r4; ++l) s = fmaf(Tm[(ij * H + h) * r4 + l], U4s[w * r4 + l], s);
+    if (h >= 0 && h < H && w >= 0 && w < W) {
+      const float* tp = Tm + (ij * H + h) * R;
+      const float* up = U4s + w * R;
+#pragma unroll
+      for (int l = 0; l < R; l += 4) {
+        const float4 a = *reinterpret_cast<const float4*>(tp + l), b = *reinterpret_cast<const float4*>(up + l);
+        s = fmaf(a.x, b.x, s); s = fmaf(a.y, b.y, s); s = fmaf(a.z, b.z, s); s = fmaf(a.w, b.w, s);
+      }
+    }
     Z3s[idx] = s;
   }
   cp_async_wait<0>();
@@ -1300,15 +1319,15 @@ int sm_core_max_rows() { return kNT; }
 int sm_wgrad_pitch(int J) { return pitch4(J); }
 
 size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
-  const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
+  const int r1 = p.r[0], r2 = p.r[1];
   const int J = p.cpb * p.Ho * p.Wo, kk = p.kh * p.kw;
   const int N4 = r2 * kk;
   const int NH = batch_groups(kNT, J);
   const size_t tile = (size_t)p.B * pitch4(J),
                stage = (size_t)(p.cpb > p.ncl ? 2 : 1) * p.ncl * (p.C / p.groups) * kk;
   size_t n = ((tile > stage ? tile : stage) + 3) / 4 * 4 + (size_t)p.B * R + (size_t)p.C * R + (size_t)J * R +
-             (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * r3 * r4 + (size_t)p.H * r3 + (size_t)p.W * r4 +
-             (size_t)r1 * r2 * p.H * r4 + ((size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + 3) / 4 * 4 +
+             (NH > 1 ? (size_t)NH * J * R : 0) + (size_t)r1 * r2 * R * R + (size_t)p.H * R + (size_t)p.W * R +
+             (size_t)r1 * r2 * p.H * R + ((size_t)r1 * r2 * (p.H + 2 * p.ph) * (p.W + 2 * p.pw) + 3) / 4 * 4 +
              (size_t)p.cpb * kk * R + (size_t)p.cpb * (N4 > kNT ? N4 : kNT);
   return 4 * n + 64;
 }
