@@ -842,6 +842,7 @@ asi_status_t asi_poll_status(const asi_plan_t* pl, const void* ws, void* stream,
   int v = 0;
   ASI_CUDA(cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, st));
   ASI_CUDA(cudaStreamSynchronize(st));
+  if (v == 0 && pl->bf16 && tc_error_flag()) v = (int)ASI_ERR_TIMEOUT;   // a wait of the tensor-core kernel expired
   *device_status = static_cast<asi_status_t>(v);
   return ASI_OK;
 }

@@ -11,6 +11,8 @@
 
 #include <algorithm>
 
+#include <type_traits>
+
 #include "asi_internal.h"
 
 namespace asi {
@@ -332,6 +334,11 @@ static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
   if (p.Q <= 0 || p.n_out <= 0) return cudaSuccess;
   ProfScope prof(ASI_K_MODEPROD, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
+  if constexpr (std::is_same<TX, __nv_bfloat16>::value) {
+    // a dense contraction with a wide factor: tensor cores (tcgen05), when the shape fits
+    const cudaError_t e = launch_tc_lastmode(p, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
   if (p.O == 1 && p.n_out <= 8 && p.si == 1 && p.Q % 4 == 0 && p.sj % 4 == 0 && p.Q >= (1 << 16) &&
       p.a <= 512 && p.a >= 8 && (reinterpret_cast<uintptr_t>(p.X) & 15u) == 0 &&
       (reinterpret_cast<uintptr_t>(p.Y) & 15u) == 0) {

@@ -153,6 +153,9 @@ int sm_core_max_rows();
 size_t sm_wgrad_smem(const SmWgradArgs& p, int R);
 int sm_wgrad_pitch(int J);
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st);
+// Tensor-core last-mode product of a bf16 tensor (tcgen05); cudaErrorNotSupported when the shape does not fit.
+cudaError_t launch_tc_lastmode(const ModeProdArgs& p, cudaStream_t st);
+int tc_error_flag();   // != 0: a bounded wait of the tensor-core kernel expired
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
 cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t st);

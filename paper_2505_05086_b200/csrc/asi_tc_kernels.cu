@@ -1,0 +1,312 @@
+// Tensor-core kernel (sm_100a: tcgen05.mma, TMEM accumulator, TMA operand staging) for the one step of
+// the path that is a plain dense contraction: the last-mode product of a bf16 tensor with a wide factor,
+//   Y[q][j] = sum_k X[q][k] U[k][j],   X bf16 [Q x a] (k contiguous), U fp32 [a x n], n = 16..64,
+// i.e. V_3 = A_(3)^T U_3 and the first core product of token layers (Algorithm 1 on a B x N x D
+// activation).  X is exact in bf16; the fp32 factor is split into three bf16 terms (24 mantissa bits),
+// so three MMAs per k-step reproduce the fp32 product to fp32 rounding with fp32 accumulation in TMEM.
+//
+// One CTA (256 threads) owns a 128-row tile of Y and walks K in chunks of 64:
+//   * the X tile [128 x 64] arrives by TMA (cp.async.bulk.tensor, 128-byte swizzle, 4 stages);
+//   * all threads split the factor chunk [64 x n] into the three bf16 operands, written K-major in the
+//     same 128-byte-swizzled layout (two buffers);
+//   * one thread issues 4 k-steps x 3 terms of tcgen05.mma (M = 128, N = n, K = 16) and commits them to
+//     the mbarriers that free the X stage and the factor buffer;
+//   * the epilogue reads the accumulator with tcgen05.ld (lane = row) and stores fp32 rows.
+// Every wait has a time limit; on expiry the kernel raises g_tc_error, frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <mutex>
+
+#include "asi_internal.h"
+
+namespace asi {
+
+namespace {
+
+constexpr int kTcThreads = 256;
+constexpr int kTcM = 128;          // rows of Y per CTA (= TMEM lanes)
+constexpr int kTcKC = 64;          // k per chunk: 64 bf16 = one 128-byte swizzle row
+constexpr int kTcStages = 4;       // X stages in flight
+constexpr int kTcNMax = 64;
+constexpr uint32_t kTileA = kTcM * kTcKC * 2;       // 16 KB
+constexpr uint32_t kTileB = kTcNMax * kTcKC * 2;    // 8 KB per term
+
+__device__ int g_tc_error = 0;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// waits for the phase with the given parity; gives up after ~1 s
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint64_t t0 = globaltimer_ns();
+  for (uint32_t it = 0; it < (1u << 28); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && globaltimer_ns() - t0 > 1000000000ull) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of 8 rows
+// 1024 bytes apart (start address, leading and stride offsets in 16-byte units; descriptor version 1)
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused by swizzled K-major layouts)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+  d |= (uint64_t)1 << 46;                 // version
+  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+  return d;
+}
+// instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major
+__device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(acc), "r"(0u)    // no output lane disabled
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// byte offset of element (row, k) of a K-major bf16 tile with 64 k per row in the 128-byte-swizzled layout
+__device__ __forceinline__ uint32_t sw128_offset(int row, int k) {
+  return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((((k >> 3) ^ (row & 7)) & 7) << 4) + (k & 7) * 2);
+}
+
+struct TcArgs {
+  const float* U;      // [K][ldu]
+  float* Y;            // [M][ldy]
+  int M, N, K, ldu, ldy;
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX, TcArgs p) {
+  extern __shared__ __align__(1024) uint8_t tc_smem[];
+  // carve-up: X stages, factor buffers (3 terms each), then barriers
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem) + 1023) & ~(uintptr_t)1023);
+  uint8_t* As = base;                                   // [stages][16 KB]
+  uint8_t* Bs = As + kTcStages * kTileA;                // [2][3][8 KB]
+  uint64_t* full = reinterpret_cast<uint64_t*>(Bs + 2 * 3 * kTileB);   // [stages] X landed
+  uint64_t* a_free = full + kTcStages;                  // [stages] MMAs that read the stage are done
+  uint64_t* b_free = a_free + kTcStages;                // [2]      MMAs that read the factor buffer are done
+  uint64_t* done = b_free + 2;                          // all MMAs of the tile are done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row0 = blockIdx.x * kTcM;
+  const int nchunk = p.K / kTcKC;
+  const int N = p.N;
+
+  if (tid == 0) {
+    for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(a_free + s, 1); }
+    mbar_init(b_free, 1); mbar_init(b_free + 1, 1); mbar_init(done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {                                      // TMEM: 64 fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(64)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (tid == 0) {                                       // first X stages
+    for (int c = 0; c < kTcStages && c < nchunk; ++c) {
+      mbar_expect_tx(full + c, kTileA);
+      tma_load_2d(As + c * kTileA, &mapX, c * kTcKC, row0, full + c);
+    }
+  }
+  const uint32_t idesc = instr_desc_bf16(kTcM, N);
+  bool ok = true;      // this thread's waits so far; failures are shared at the barriers (__syncthreads_or)
+  bool fail = false;   // uniform across the CTA
+#pragma unroll 1
+  for (int c = 0; c < nchunk; ++c) {
+    const int s = c % kTcStages, b = c & 1;
+    // ---- the factor chunk U[c*64 .. c*64+64)[0..N) as three bf16 operands, K-major, swizzled.
+    // A warp covers 8 factor columns (operand rows) x one 16-byte chunk of k: conflict-free 4-byte stores.
+    if (c >= 2) ok = mbar_wait(b_free + b, ((c >> 1) - 1) & 1) && ok;
+    if (ok) {
+      uint8_t* B0 = Bs + b * 3 * kTileB;
+      const int kq = lane & 3, jr = lane >> 2;
+      const float* Uc = p.U + (int64_t)c * kTcKC * p.ldu;
+      for (int it = warp; it < (N >> 3) * 8; it += kTcThreads / 32) {
+        const int jb = it >> 3, kc8 = it & 7;           // 8-column block, 16-byte chunk of k
+        const int j = jb * 8 + jr, k = kc8 * 8 + kq * 2;
+        const float u0 = __ldg(Uc + (int64_t)k * p.ldu + j), u1 = __ldg(Uc + (int64_t)(k + 1) * p.ldu + j);
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(u0), h1 = __float2bfloat16_rn(u1);
+        const float r0 = u0 - __bfloat162float(h0), r1 = u1 - __bfloat162float(h1);
+        const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(r0 - __bfloat162float(m0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(r1 - __bfloat162float(m1));
+        const uint32_t off = sw128_offset(j, k);
+        *reinterpret_cast<__nv_bfloat162*>(B0 + off) = __halves2bfloat162(h0, h1);
+        *reinterpret_cast<__nv_bfloat162*>(B0 + kTileB + off) = __halves2bfloat162(m0, m1);
+        *reinterpret_cast<__nv_bfloat162*>(B0 + 2 * kTileB + off) = __halves2bfloat162(l0, l1);
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    fail = __syncthreads_or(ok ? 0 : 1) != 0;
+    if (fail) break;
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // refill the stage of the previous chunk once its MMAs have finished reading it
+      if (c >= 1 && c - 1 + kTcStages < nchunk) {
+        const int sp = (c - 1) % kTcStages;
+        ok = mbar_wait(a_free + sp, ((c - 1) / kTcStages) & 1) && ok;
+        if (ok) {
+          mbar_expect_tx(full + sp, kTileA);
+          tma_load_2d(As + sp * kTileA, &mapX, (c - 1 + kTcStages) * kTcKC, row0, full + sp);
+        }
+      }
+      ok = mbar_wait(full + s, (c / kTcStages) & 1) && ok;
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(As + s * kTileA);
+        const uint32_t b_addr = smem_u32(Bs + b * 3 * kTileB);
+#pragma unroll
+        for (int ks = 0; ks < kTcKC / 16; ++ks) {       // 16 bf16 = 32 bytes along k inside the swizzle row
+          const uint64_t da = smem_desc_sw128(a_addr + ks * 32);
+#pragma unroll
+          for (int t = 0; t < 3; ++t) {
+            const uint64_t db = smem_desc_sw128(b_addr + t * kTileB + ks * 32);
+            umma_bf16(tmem_d, da, db, idesc, (c | ks | t) ? 1u : 0u);
+          }
+        }
+      }
+      umma_commit(a_free + s);
+      umma_commit(b_free + b);
+      if (c == nchunk - 1) umma_commit(done);
+    }
+  }
+  if (!fail) {
+    ok = mbar_wait(done, 0) && ok;                      // every thread observes the completed phase
+    fail = __syncthreads_or(ok ? 0 : 1) != 0;
+  }
+  if (!fail) {
+    // thread = row: warp w reads lanes 32 (w % 4) ..., warps 0-3 the columns [0, N/2), warps 4-7 the rest
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int half = N >> 1;                            // 8, 16, 24 or 32 columns per warp
+    const int col0 = (warp >> 2) * half;
+    const int row = row0 + (warp & 3) * 32 + lane;
+    const uint32_t taddr = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
+    for (int cc = 0; cc < half; cc += 8) {
+      uint32_t v[8];
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                   : "r"(taddr + (uint32_t)cc)
+                   : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (row < p.M) {
+        float* y = p.Y + (int64_t)row * p.ldy + col0 + cc;
+        *reinterpret_cast<float4*>(y) = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+        *reinterpret_cast<float4*>(y + 4) = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
+      }
+    }
+  } else if (tid == 0) {
+    atomicExch(&g_tc_error, 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(64) : "memory");
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(p);
+  });
+  return fn;
+}
+
+}  // namespace
+
+// Y[q][j] = sum_k X[q][k] U[k][j] on the tensor cores.  Returns cudaErrorNotSupported when the shape or the
+// alignment does not fit (the caller then takes the SIMT kernel).
+cudaError_t launch_tc_lastmode(const ModeProdArgs& p, cudaStream_t st) {
+  const int64_t M = p.Q, K = p.a;
+  const int N = p.n_out;
+  if (p.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || K % kTcKC != 0 || K < kTcKC || M < kTcM ||
+      M >= (1ll << 31) || K >= (1ll << 31) || p.sj != 1 || p.so % 4 != 0 || p.ldb_j != 1 ||
+      (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u) || (K * 2) % 16 != 0)
+    return cudaErrorNotSupported;
+  EncodeFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)kTcM};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p.X), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorNotSupported;
+  static const size_t smem = 1024 + kTcStages * kTileA + 2 * 3 * kTileB + 16 * 8 + 16;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(k_tc_lastmode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  });
+  if (attr_err != cudaSuccess) return attr_err;
+  TcArgs a = {p.B, p.Y, (int)M, N, (int)K, (int)p.ldb_k, (int)p.so};
+  const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
+  k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(map, a);
+  return cudaGetLastError();
+}
+
+int tc_error_flag() {
+  int v = 0;
+  cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int));
+  return v;
+}
+
+}  // namespace asi
