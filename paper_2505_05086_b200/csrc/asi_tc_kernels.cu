@@ -3,15 +3,19 @@
 //   Y[q][j] = sum_k X[q][k] U[k][j],   X bf16 [Q x a] (k contiguous), U fp32 [a x n], n = 16..64,
 // i.e. V_3 = A_(3)^T U_3 and the first core product of token layers (Algorithm 1 on a B x N x D
 // activation).  X is exact in bf16; the fp32 factor is split into three bf16 terms (24 mantissa bits),
-// so three MMAs per k-step reproduce the fp32 product to fp32 rounding with fp32 accumulation in TMEM.
+// so one MMA of width 3 n per k-step (the three terms stacked as operand rows) yields three partial products
+// in TMEM whose sum reproduces the fp32 product to fp32 rounding.
 //
-// One CTA (256 threads) owns a 128-row tile of Y and walks K in chunks of 64:
-//   * the X tile [128 x 64] arrives by TMA (cp.async.bulk.tensor, 128-byte swizzle, 4 stages);
-//   * all threads split the factor chunk [64 x n] into the three bf16 operands, written K-major in the
-//     same 128-byte-swizzled layout (two buffers);
-//   * one thread issues 4 k-steps x 3 terms of tcgen05.mma (M = 128, N = n, K = 16) and commits them to
-//     the mbarriers that free the X stage and the factor buffer;
-//   * the epilogue reads the accumulator with tcgen05.ld (lane = row) and stores fp32 rows.
+// One CTA owns a 128-row tile of Y and walks K in chunks of 64, its warps in three roles that meet only
+// through mbarriers:
+//   * a producer thread keeps four X tiles [128 x 64] in flight by TMA (cp.async.bulk.tensor, 128-byte
+//     swizzle);
+//   * sixteen converter warps split the factor chunk [64 x n] into the three bf16 operands, written
+//     K-major in the same 128-byte-swizzled layout (four buffers);
+//   * an issuer thread launches 4 k-steps of tcgen05.mma (M = 128, N = 3 n, K = 16) per chunk and
+//     commits them to the mbarriers that free the X stage and the factor buffer;
+//   * eight warps then read the three accumulator groups with tcgen05.ld (lane = row), add them and store
+//     fp32 rows.
 // Every wait has a time limit; on expiry the kernel raises g_tc_error, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -26,10 +30,13 @@ namespace asi {
 
 namespace {
 
-constexpr int kTcThreads = 256;
+constexpr int kTcWorkers = 16;      // converter warps (the first eight also run the epilogue)
+constexpr int kTcThreads = (kTcWorkers + 2) * 32;   // + the MMA issuer warp and the TMA producer warp
 constexpr int kTcM = 128;          // rows of Y per CTA (= TMEM lanes)
 constexpr int kTcKC = 64;          // k per chunk: 64 bf16 = one 128-byte swizzle row
 constexpr int kTcStages = 4;       // X stages in flight
+constexpr int kTcBufs = 4;         // factor-operand buffers: the chain MMA -> convert -> MMA of one buffer is
+                                   // ~3 K cycles long, four buffers keep the tensor pipe fed
 constexpr int kTcNMax = 64;
 constexpr uint32_t kTileA = kTcM * kTcKC * 2;       // 16 KB
 constexpr uint32_t kTileB = kTcNMax * kTcKC * 2;    // 8 KB per term
@@ -41,6 +48,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
@@ -64,10 +74,11 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 }
 // waits for the phase with the given parity; gives up after ~1 s
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;       // the common case costs no timer read
   const uint64_t t0 = globaltimer_ns();
   for (uint32_t it = 0; it < (1u << 28); ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && globaltimer_ns() - t0 > 1000000000ull) return false;
+    if ((it & 1023u) == 1023u && globaltimer_ns() - t0 > 1000000000ull) return false;
   }
   return false;
 }
@@ -105,6 +116,12 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {   // 8 columns of this thread's lane
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
 // byte offset of element (row, k) of a K-major bf16 tile with 64 k per row in the 128-byte-swizzled layout
 __device__ __forceinline__ uint32_t sw128_offset(int row, int k) {
   return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((((k >> 3) ^ (row & 7)) & 7) << 4) + (k & 7) * 2);
@@ -121,11 +138,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   // carve-up: X stages, factor buffers (3 terms each), then barriers
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem) + 1023) & ~(uintptr_t)1023);
   uint8_t* As = base;                                   // [stages][16 KB]
-  uint8_t* Bs = As + kTcStages * kTileA;                // [2][3][8 KB]
-  uint64_t* full = reinterpret_cast<uint64_t*>(Bs + 2 * 3 * kTileB);   // [stages] X landed
+  uint8_t* Bs = As + kTcStages * kTileA;                // [kTcBufs][3][8 KB]
+  uint64_t* full = reinterpret_cast<uint64_t*>(Bs + kTcBufs * 3 * kTileB);   // [stages] X landed
   uint64_t* a_free = full + kTcStages;                  // [stages] MMAs that read the stage are done
-  uint64_t* b_free = a_free + kTcStages;                // [2]      MMAs that read the factor buffer are done
-  uint64_t* done = b_free + 2;                          // all MMAs of the tile are done
+  uint64_t* b_free = a_free + kTcStages;                // [bufs]   MMAs that read the factor buffer are done
+  uint64_t* b_ready = b_free + kTcBufs;                 // [bufs]   the converter warps have filled it
+  uint64_t* done = b_ready + kTcBufs;                         // all MMAs of the tile are done
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -135,12 +153,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(a_free + s, 1); }
-    mbar_init(b_free, 1); mbar_init(b_free + 1, 1); mbar_init(done, 1);
+    for (int i = 0; i < kTcBufs; ++i) { mbar_init(b_free + i, 1); mbar_init(b_ready + i, kTcWorkers); }
+    mbar_init(done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {                                      // TMEM: 64 fp32 columns x 128 lanes
+  if (warp == 0) {                                      // TMEM: 256 fp32 columns x 128 lanes (3 N are used)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(64)
+                 "r"(256)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -149,97 +168,118 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = *tmem_slot;
 
-  if (tid == 0) {                                       // first X stages
-    for (int c = 0; c < kTcStages && c < nchunk; ++c) {
-      mbar_expect_tx(full + c, kTileA);
-      tma_load_2d(As + c * kTileA, &mapX, c * kTcKC, row0, full + c);
-    }
-  }
-  const uint32_t idesc = instr_desc_bf16(kTcM, N);
-  bool ok = true;      // this thread's waits so far; failures are shared at the barriers (__syncthreads_or)
-  bool fail = false;   // uniform across the CTA
-#pragma unroll 1
-  for (int c = 0; c < nchunk; ++c) {
-    const int s = c % kTcStages, b = c & 1;
-    // ---- the factor chunk U[c*64 .. c*64+64)[0..N) as three bf16 operands, K-major, swizzled.
-    // A warp covers 8 factor columns (operand rows) x one 16-byte chunk of k: conflict-free 4-byte stores.
-    if (c >= 2) ok = mbar_wait(b_free + b, ((c >> 1) - 1) & 1) && ok;
-    if (ok) {
-      uint8_t* B0 = Bs + b * 3 * kTileB;
-      const int kq = lane & 3, jr = lane >> 2;
+  // The three bf16 terms of the factor are stacked along the operand's rows: one MMA of width 3 N per
+  // k-step reads the X tile once and leaves the three partial products in three column groups of TMEM.
+  const uint32_t idesc = instr_desc_bf16(kTcM, 3 * N);
+  const uint32_t term_bytes = (uint32_t)N * 128u;      // rows of one term in the swizzled operand tile
+  bool ok = true;                                      // this thread's waits so far
+  if (warp < kTcWorkers) {
+    // ---- converter warps: the factor chunk U[c*64 .. c*64+64)[0..N) as three bf16 operands, K-major,
+    // swizzled.  A warp covers 8 factor columns (operand rows) x one 16-byte chunk of k per item:
+    // conflict-free 4-byte shared-memory stores.  The values are fetched one chunk ahead.
+    constexpr int kItems = (kTcNMax / 8) * 8 / kTcWorkers;         // items per warp at N = 64
+    const int nitems = (N >> 3) * 8;
+    const int kq = lane & 3, jr = lane >> 2;
+    float2 ureg[kItems];
+    auto load_chunk = [&](int c) {
       const float* Uc = p.U + (int64_t)c * kTcKC * p.ldu;
-      for (int it = warp; it < (N >> 3) * 8; it += kTcThreads / 32) {
-        const int jb = it >> 3, kc8 = it & 7;           // 8-column block, 16-byte chunk of k
-        const int j = jb * 8 + jr, k = kc8 * 8 + kq * 2;
-        const float u0 = __ldg(Uc + (int64_t)k * p.ldu + j), u1 = __ldg(Uc + (int64_t)(k + 1) * p.ldu + j);
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(u0), h1 = __float2bfloat16_rn(u1);
-        const float r0 = u0 - __bfloat162float(h0), r1 = u1 - __bfloat162float(h1);
-        const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
-        const __nv_bfloat16 l0 = __float2bfloat16_rn(r0 - __bfloat162float(m0));
-        const __nv_bfloat16 l1 = __float2bfloat16_rn(r1 - __bfloat162float(m1));
-        const uint32_t off = sw128_offset(j, k);
-        *reinterpret_cast<__nv_bfloat162*>(B0 + off) = __halves2bfloat162(h0, h1);
-        *reinterpret_cast<__nv_bfloat162*>(B0 + kTileB + off) = __halves2bfloat162(m0, m1);
-        *reinterpret_cast<__nv_bfloat162*>(B0 + 2 * kTileB + off) = __halves2bfloat162(l0, l1);
-      }
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    fail = __syncthreads_or(ok ? 0 : 1) != 0;
-    if (fail) break;
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // refill the stage of the previous chunk once its MMAs have finished reading it
-      if (c >= 1 && c - 1 + kTcStages < nchunk) {
-        const int sp = (c - 1) % kTcStages;
-        ok = mbar_wait(a_free + sp, ((c - 1) / kTcStages) & 1) && ok;
-        if (ok) {
-          mbar_expect_tx(full + sp, kTileA);
-          tma_load_2d(As + sp * kTileA, &mapX, (c - 1 + kTcStages) * kTcKC, row0, full + sp);
+#pragma unroll
+      for (int i = 0; i < kItems; ++i) {
+        const int it = warp + i * kTcWorkers;
+        if (it < nitems) {
+          const int j = (it >> 3) * 8 + jr, k = (it & 7) * 8 + kq * 2;
+          ureg[i] = make_float2(__ldg(Uc + (int64_t)k * p.ldu + j), __ldg(Uc + (int64_t)(k + 1) * p.ldu + j));
         }
       }
-      ok = mbar_wait(full + s, (c / kTcStages) & 1) && ok;
-      if (ok) {
+    };
+    load_chunk(0);
+#pragma unroll 1
+    for (int c = 0; c < nchunk && ok; ++c) {
+      const int b = c % kTcBufs;
+      if (c >= kTcBufs) ok = mbar_wait(b_free + b, ((c / kTcBufs) - 1) & 1);   // the MMAs that read it are done
+      if (!ok) break;
+      uint8_t* B0 = Bs + b * 3 * kTileB;
+#pragma unroll
+      for (int i = 0; i < kItems; ++i) {
+        const int it = warp + i * kTcWorkers;
+        if (it < nitems) {
+          const int j = (it >> 3) * 8 + jr, k = (it & 7) * 8 + kq * 2;
+          const float u0 = ureg[i].x, u1 = ureg[i].y;
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(u0), h1 = __float2bfloat16_rn(u1);
+          const float r0 = u0 - __bfloat162float(h0), r1 = u1 - __bfloat162float(h1);
+          const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(r0 - __bfloat162float(m0));
+          const __nv_bfloat16 l1 = __float2bfloat16_rn(r1 - __bfloat162float(m1));
+          const uint32_t off = sw128_offset(j, k);
+          *reinterpret_cast<__nv_bfloat162*>(B0 + off) = __halves2bfloat162(h0, h1);
+          *reinterpret_cast<__nv_bfloat162*>(B0 + term_bytes + off) = __halves2bfloat162(m0, m1);
+          *reinterpret_cast<__nv_bfloat162*>(B0 + 2 * term_bytes + off) = __halves2bfloat162(l0, l1);
+        }
+      }
+      if (c + 1 < nchunk) load_chunk(c + 1);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_ready + b);         // one arrival per warp: arrivals on one barrier serialise
+    }
+  } else if (warp == kTcWorkers) {
+    // ---- MMA issuer (one thread): 4 k-steps per chunk, then the commits that free the X stage and the
+    // factor buffer
+    if (lane == 0) {
+      const uint32_t a_base = smem_u32(As), b_base = smem_u32(Bs);
+#pragma unroll 1
+      for (int c = 0; c < nchunk && ok; ++c) {
+        const int s = c % kTcStages, b = c % kTcBufs;
+        ok = mbar_wait(b_ready + b, (c / kTcBufs) & 1) && mbar_wait(full + s, (c / kTcStages) & 1);
+        if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = smem_u32(As + s * kTileA);
-        const uint32_t b_addr = smem_u32(Bs + b * 3 * kTileB);
+        const uint64_t da0 = smem_desc_sw128(a_base + s * kTileA);
+        const uint64_t db0 = smem_desc_sw128(b_base + b * 3 * kTileB);
 #pragma unroll
-        for (int ks = 0; ks < kTcKC / 16; ++ks) {       // 16 bf16 = 32 bytes along k inside the swizzle row
-          const uint64_t da = smem_desc_sw128(a_addr + ks * 32);
-#pragma unroll
-          for (int t = 0; t < 3; ++t) {
-            const uint64_t db = smem_desc_sw128(b_addr + t * kTileB + ks * 32);
-            umma_bf16(tmem_d, da, db, idesc, (c | ks | t) ? 1u : 0u);
-          }
-        }
+        for (int ks = 0; ks < kTcKC / 16; ++ks)         // 16 bf16 = 32 bytes along k inside the swizzle row
+          umma_bf16(tmem_d, da0 + (uint64_t)(ks * 2), db0 + (uint64_t)(ks * 2), idesc, (c | ks) ? 1u : 0u);
+        umma_commit(a_free + s);
+        umma_commit(b_free + b);
       }
-      umma_commit(a_free + s);
-      umma_commit(b_free + b);
-      if (c == nchunk - 1) umma_commit(done);
+      umma_commit(done);
+    }
+  } else {
+    // ---- TMA producer (one thread): keeps kTcStages X tiles in flight
+    if (lane == 0) {
+#pragma unroll 1
+      for (int c = 0; c < nchunk && ok; ++c) {
+        const int s = c % kTcStages;
+        if (c >= kTcStages) ok = mbar_wait(a_free + s, ((c / kTcStages) - 1) & 1);
+        if (!ok) break;
+        mbar_expect_tx(full + s, kTileA);
+        tma_load_2d(As + s * kTileA, &mapX, c * kTcKC, row0, full + s);
+      }
     }
   }
+  if (warp < 8) ok = mbar_wait(done, 0) && ok;          // every reader of TMEM observes the completed phase
+  const bool fail = __syncthreads_or(ok ? 0 : 1) != 0;
   if (!fail) {
-    ok = mbar_wait(done, 0) && ok;                      // every thread observes the completed phase
-    fail = __syncthreads_or(ok ? 0 : 1) != 0;
-  }
-  if (!fail) {
-    // thread = row: warp w reads lanes 32 (w % 4) ..., warps 0-3 the columns [0, N/2), warps 4-7 the rest
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int half = N >> 1;                            // 8, 16, 24 or 32 columns per warp
-    const int col0 = (warp >> 2) * half;
-    const int row = row0 + (warp & 3) * 32 + lane;
-    const uint32_t taddr = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
-    for (int cc = 0; cc < half; cc += 8) {
-      uint32_t v[8];
-      asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                   : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                   : "r"(taddr + (uint32_t)cc)
-                   : "memory");
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (row < p.M) {
-        float* y = p.Y + (int64_t)row * p.ldy + col0 + cc;
-        *reinterpret_cast<float4*>(y) = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
-        *reinterpret_cast<float4*>(y + 4) = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
+    if (warp < 8) {
+      // thread = row: warp w reads lanes 32 (w % 4) ..., warps 0-3 the columns [0, N/2), warps 4-7 the rest
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int half = N >> 1;                          // 8, 16, 24 or 32 columns per warp
+      const int col0 = (warp >> 2) * half;
+      const int row = row0 + (warp & 3) * 32 + lane;
+      const uint32_t taddr = tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
+      for (int cc = 0; cc < half; cc += 8) {
+        uint32_t h[8], m[8], l[8];
+        tmem_ld8(taddr + (uint32_t)cc, h);
+        tmem_ld8(taddr + (uint32_t)(N + cc), m);
+        tmem_ld8(taddr + (uint32_t)(2 * N + cc), l);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < p.M) {
+          float o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)                   // small terms first
+            o[i] = (__uint_as_float(l[i]) + __uint_as_float(m[i])) + __uint_as_float(h[i]);
+          float* y = p.Y + (int64_t)row * p.ldy + col0 + cc;
+          *reinterpret_cast<float4*>(y) = make_float4(o[0], o[1], o[2], o[3]);
+          *reinterpret_cast<float4*>(y + 4) = make_float4(o[4], o[5], o[6], o[7]);
+        }
       }
     }
   } else if (tid == 0) {
@@ -248,7 +288,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(64) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(256) : "memory");
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -290,7 +330,7 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, cudaStream_t st) {
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorNotSupported;
-  static const size_t smem = 1024 + kTcStages * kTileA + 2 * 3 * kTileB + 16 * 8 + 16;
+  static const size_t smem = 1024 + kTcStages * kTileA + kTcBufs * 3 * kTileB + (2 * kTcStages + 2 * kTcBufs + 1) * 8 + 16;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
