@@ -139,6 +139,17 @@ void layout_compress(asi_plan* pl) {
     pl->off_Gp[m] = off;
     off = align_up(off + (size_t)pl->nchunk[m] * v.r * v.r * 8, 256);
   }
+  // bf16 operand of the tensor-core kernel: last-mode products of bf16 tensors with a wide factor
+  pl->off_tc = off;
+  pl->tc_bytes = 0;
+  {
+    const int m = pl->nd - 1;
+    const ModeView& v = pl->mv[m];
+    if (pl->bf16 && !pl->fast_compress && v.I == 1 && pl->r[m] % 16 == 0 && pl->r[m] >= 16 && pl->r[m] <= 64 &&
+        v.a % 64 == 0 && v.Q >= 128)
+      pl->tc_bytes = tc_scratch_bytes(v.a, pl->r[m]);
+  }
+  off = align_up(off + pl->tc_bytes, 256);
   pl->off_Rf = off;                                   // Cholesky factors of the fused path
   off = align_up(off + (size_t)ASI_MAX_MODES * kRfStride * 8, 256);
   for (int m = 0; m < ASI_MAX_MODES; ++m) pl->off_Pg[m] = 0;
@@ -181,6 +192,9 @@ void layout_compress(asi_plan* pl) {
     pl->launches_compress = 2 + pl->nd;                                    // reduction/QR pair, core chain
     for (int m = 0; m < pl->nd; ++m)
       pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
+    // tensor-core products are two launches (operand split + GEMM): V of the last mode, and the first
+    // core product when it contracts the last mode
+    if (pl->tc_bytes) pl->launches_compress += 1 + (pl->core_order[0] == pl->nd - 1 ? 1 : 0);
   }
 }
 
@@ -351,6 +365,8 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     a.si = 1;
     float* dst = (s == pl->nd - 1) ? core : reinterpret_cast<float*>(w + pl->off_T[s & 1]);
     a.Y = dst;
+    a.tc_scratch = w + pl->off_tc;
+    a.tc_scratch_bytes = pl->tc_bytes;
     ASI_CUDA(launch_modeprod(a, src_bf16, st));
     cd[m] = pl->r[m];
     src = dst;
@@ -583,6 +599,8 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     a.so = v.I * v.r;
     a.sj = 1;
     a.si = v.r;
+    a.tc_scratch = w + pl->off_tc;
+    a.tc_scratch_bytes = pl->tc_bytes;
     ASI_CUDA(launch_modeprod(a, pl->bf16, st));
     // P = A_m V
     s = expand_mode(pl, m, act, V, w, st);

@@ -336,7 +336,7 @@ static cudaError_t launch_modeprod_t(const ModeProdArgs& p, cudaStream_t st) {
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.a * p.n_out + (double)p.Q * p.n_out));
   if constexpr (std::is_same<TX, __nv_bfloat16>::value) {
     // a dense contraction with a wide factor: tensor cores (tcgen05), when the shape fits
-    const cudaError_t e = launch_tc_lastmode(p, st);
+    const cudaError_t e = launch_tc_lastmode(p, p.tc_scratch, p.tc_scratch_bytes, st);
     if (e != cudaErrorNotSupported) return e;
   }
   if (p.O == 1 && p.n_out <= 8 && p.si == 1 && p.Q % 4 == 0 && p.sj % 4 == 0 && p.Q >= (1 << 16) &&

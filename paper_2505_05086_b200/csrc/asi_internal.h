@@ -32,6 +32,8 @@ struct ModeProdArgs {
   int n_out;
   int64_t ldb_k, ldb_j;    // B(k, j) = B[k*ldb_k + j*ldb_j]
   int64_t so, sj, si;      // Y(o, j, i) = Y[o*so + j*sj + i*si]
+  void* tc_scratch = nullptr;      // device scratch for the tensor-core kernel's bf16 operand (optional)
+  size_t tc_scratch_bytes = 0;
 };
 
 // Pp[s](k, j) = sum_{q in split s} X(k, q) * V[q*r + j]
@@ -154,7 +156,8 @@ size_t sm_wgrad_smem(const SmWgradArgs& p, int R);
 int sm_wgrad_pitch(int J);
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st);
 // Tensor-core last-mode product of a bf16 tensor (tcgen05); cudaErrorNotSupported when the shape does not fit.
-cudaError_t launch_tc_lastmode(const ModeProdArgs& p, cudaStream_t st);
+cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st);
+size_t tc_scratch_bytes(int64_t K, int N);
 int tc_error_flag();   // != 0: a bounded wait of the tensor-core kernel expired
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
@@ -214,6 +217,7 @@ struct asi_plan {
   // compress workspace (byte offsets)
   size_t off_V, off_Pp[ASI_MAX_MODES], off_Pred[ASI_MAX_MODES], off_Gp[ASI_MAX_MODES], off_T[2];
   size_t off_Rf, off_Pg[ASI_MAX_MODES];
+  size_t off_tc, tc_bytes;         // bf16 operand of the tensor-core last-mode product (0 bytes: not used)
   int nsplit[ASI_MAX_MODES], nchunk[ASI_MAX_MODES];
   int64_t q_per_split[ASI_MAX_MODES];
   int core_order[ASI_MAX_MODES];

@@ -6,14 +6,13 @@
 // so one MMA of width 3 n per k-step (the three terms stacked as operand rows) yields three partial products
 // in TMEM whose sum reproduces the fp32 product to fp32 rounding.
 //
-// One CTA owns a 128-row tile of Y and walks K in chunks of 64, its warps in three roles that meet only
-// through mbarriers:
-//   * a producer thread keeps four X tiles [128 x 64] in flight by TMA (cp.async.bulk.tensor, 128-byte
-//     swizzle);
-//   * sixteen converter warps split the factor chunk [64 x n] into the three bf16 operands, written
-//     K-major in the same 128-byte-swizzled layout (four buffers);
-//   * an issuer thread launches 4 k-steps of tcgen05.mma (M = 128, N = 3 n, K = 16) per chunk and
-//     commits them to the mbarriers that free the X stage and the factor buffer;
+// k_tc_split writes the stacked operand [3 n][K] (bf16, K contiguous: hi rows, then mid, then lo) to
+// scratch memory once per product; k_tc_lastmode then streams both operands by TMA.  One CTA owns a
+// 128-row tile of Y and walks K in chunks of 64, its warps in three roles that meet only through mbarriers:
+//   * a producer thread keeps four stages in flight, each the X tile [128 x 64] and the operand tile
+//     [3 n x 64] (cp.async.bulk.tensor, 128-byte swizzle);
+//   * an issuer thread launches 4 k-steps of tcgen05.mma (M = 128, N = 3 n, K = 16) per chunk and commits
+//     them to the mbarrier that frees the stage;
 //   * eight warps then read the three accumulator groups with tcgen05.ld (lane = row), add them and store
 //     fp32 rows.
 // Every wait has a time limit; on expiry the kernel raises g_tc_error, frees its TMEM and returns.
@@ -30,16 +29,14 @@ namespace asi {
 
 namespace {
 
-constexpr int kTcWorkers = 16;      // converter warps (the first eight also run the epilogue)
+constexpr int kTcWorkers = 8;       // epilogue warps
 constexpr int kTcThreads = (kTcWorkers + 2) * 32;   // + the MMA issuer warp and the TMA producer warp
 constexpr int kTcM = 128;          // rows of Y per CTA (= TMEM lanes)
 constexpr int kTcKC = 64;          // k per chunk: 64 bf16 = one 128-byte swizzle row
 constexpr int kTcStages = 4;       // X stages in flight
-constexpr int kTcBufs = 4;         // factor-operand buffers: the chain MMA -> convert -> MMA of one buffer is
-                                   // ~3 K cycles long, four buffers keep the tensor pipe fed
 constexpr int kTcNMax = 64;
 constexpr uint32_t kTileA = kTcM * kTcKC * 2;       // 16 KB
-constexpr uint32_t kTileB = kTcNMax * kTcKC * 2;    // 8 KB per term
+constexpr uint32_t kTileB = 3 * kTcNMax * kTcKC * 2;   // 24 KB: the three terms stacked
 
 __device__ int g_tc_error = 0;
 
@@ -48,9 +45,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
@@ -122,28 +116,47 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {   /
                : "r"(taddr)
                : "memory");
 }
-// byte offset of element (row, k) of a K-major bf16 tile with 64 k per row in the 128-byte-swizzled layout
-__device__ __forceinline__ uint32_t sw128_offset(int row, int k) {
-  return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((((k >> 3) ^ (row & 7)) & 7) << 4) + (k & 7) * 2);
-}
-
 struct TcArgs {
-  const float* U;      // [K][ldu]
   float* Y;            // [M][ldy]
-  int M, N, K, ldu, ldy;
+  int M, N, K, ldy;
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX, TcArgs p) {
+// Bt[t*n + j][k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
+__global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, int ldu, int K, int N,
+                                                  __nv_bfloat16* __restrict__ Bt) {
+  __shared__ float tile[32][33];
+  const int k0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) {
+    const int k = k0 + r, j = j0 + tx;
+    tile[r][tx] = (k < K && j < N) ? U[(int64_t)k * ldu + j] : 0.f;
+  }
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {
+    const int j = j0 + r, k = k0 + tx;
+    if (j < N && k < K) {
+      const float u = tile[tx][r];
+      const __nv_bfloat16 h = __float2bfloat16_rn(u);
+      const float r1 = u - __bfloat162float(h);
+      const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+      const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+      Bt[(int64_t)j * K + k] = h;
+      Bt[(int64_t)(N + j) * K + k] = m;
+      Bt[(int64_t)(2 * N + j) * K + k] = l;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX,
+                                                                const __grid_constant__ CUtensorMap mapB, TcArgs p) {
   extern __shared__ __align__(1024) uint8_t tc_smem[];
-  // carve-up: X stages, factor buffers (3 terms each), then barriers
+  // carve-up: per stage the X tile and the operand tile, then barriers
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem) + 1023) & ~(uintptr_t)1023);
   uint8_t* As = base;                                   // [stages][16 KB]
-  uint8_t* Bs = As + kTcStages * kTileA;                // [kTcBufs][3][8 KB]
-  uint64_t* full = reinterpret_cast<uint64_t*>(Bs + kTcBufs * 3 * kTileB);   // [stages] X landed
-  uint64_t* a_free = full + kTcStages;                  // [stages] MMAs that read the stage are done
-  uint64_t* b_free = a_free + kTcStages;                // [bufs]   MMAs that read the factor buffer are done
-  uint64_t* b_ready = b_free + kTcBufs;                 // [bufs]   the converter warps have filled it
-  uint64_t* done = b_ready + kTcBufs;                         // all MMAs of the tile are done
+  uint8_t* Bs = As + kTcStages * kTileA;                // [stages][24 KB]
+  uint64_t* full = reinterpret_cast<uint64_t*>(Bs + kTcStages * kTileB);   // [stages] both tiles landed
+  uint64_t* s_free = full + kTcStages;                  // [stages] the MMAs that read the stage are done
+  uint64_t* done = s_free + kTcStages;                  // all MMAs of the tile are done
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -152,8 +165,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   const int N = p.N;
 
   if (tid == 0) {
-    for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(a_free + s, 1); }
-    for (int i = 0; i < kTcBufs; ++i) { mbar_init(b_free + i, 1); mbar_init(b_ready + i, kTcWorkers); }
+    for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(s_free + s, 1); }
     mbar_init(done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -171,94 +183,46 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   // The three bf16 terms of the factor are stacked along the operand's rows: one MMA of width 3 N per
   // k-step reads the X tile once and leaves the three partial products in three column groups of TMEM.
   const uint32_t idesc = instr_desc_bf16(kTcM, 3 * N);
-  const uint32_t term_bytes = (uint32_t)N * 128u;      // rows of one term in the swizzled operand tile
-  bool ok = true;                                      // this thread's waits so far
-  if (warp < kTcWorkers) {
-    // ---- converter warps: the factor chunk U[c*64 .. c*64+64)[0..N) as three bf16 operands, K-major,
-    // swizzled.  A warp covers 8 factor columns (operand rows) x one 16-byte chunk of k per item:
-    // conflict-free 4-byte shared-memory stores.  The values are fetched one chunk ahead.
-    constexpr int kItems = (kTcNMax / 8) * 8 / kTcWorkers;         // items per warp at N = 64
-    const int nitems = (N >> 3) * 8;
-    const int kq = lane & 3, jr = lane >> 2;
-    float2 ureg[kItems];
-    auto load_chunk = [&](int c) {
-      const float* Uc = p.U + (int64_t)c * kTcKC * p.ldu;
-#pragma unroll
-      for (int i = 0; i < kItems; ++i) {
-        const int it = warp + i * kTcWorkers;
-        if (it < nitems) {
-          const int j = (it >> 3) * 8 + jr, k = (it & 7) * 8 + kq * 2;
-          ureg[i] = make_float2(__ldg(Uc + (int64_t)k * p.ldu + j), __ldg(Uc + (int64_t)(k + 1) * p.ldu + j));
-        }
-      }
-    };
-    load_chunk(0);
-#pragma unroll 1
-    for (int c = 0; c < nchunk && ok; ++c) {
-      const int b = c % kTcBufs;
-      if (c >= kTcBufs) ok = mbar_wait(b_free + b, ((c / kTcBufs) - 1) & 1);   // the MMAs that read it are done
-      if (!ok) break;
-      uint8_t* B0 = Bs + b * 3 * kTileB;
-#pragma unroll
-      for (int i = 0; i < kItems; ++i) {
-        const int it = warp + i * kTcWorkers;
-        if (it < nitems) {
-          const int j = (it >> 3) * 8 + jr, k = (it & 7) * 8 + kq * 2;
-          const float u0 = ureg[i].x, u1 = ureg[i].y;
-          const __nv_bfloat16 h0 = __float2bfloat16_rn(u0), h1 = __float2bfloat16_rn(u1);
-          const float r0 = u0 - __bfloat162float(h0), r1 = u1 - __bfloat162float(h1);
-          const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
-          const __nv_bfloat16 l0 = __float2bfloat16_rn(r0 - __bfloat162float(m0));
-          const __nv_bfloat16 l1 = __float2bfloat16_rn(r1 - __bfloat162float(m1));
-          const uint32_t off = sw128_offset(j, k);
-          *reinterpret_cast<__nv_bfloat162*>(B0 + off) = __halves2bfloat162(h0, h1);
-          *reinterpret_cast<__nv_bfloat162*>(B0 + term_bytes + off) = __halves2bfloat162(m0, m1);
-          *reinterpret_cast<__nv_bfloat162*>(B0 + 2 * term_bytes + off) = __halves2bfloat162(l0, l1);
-        }
-      }
-      if (c + 1 < nchunk) load_chunk(c + 1);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
-      __syncwarp();
-      if (lane == 0) mbar_arrive(b_ready + b);         // one arrival per warp: arrivals on one barrier serialise
-    }
-  } else if (warp == kTcWorkers) {
-    // ---- MMA issuer (one thread): 4 k-steps per chunk, then the commits that free the X stage and the
-    // factor buffer
+  const uint32_t b_bytes = (uint32_t)(3 * N) * 128u;    // operand tile: 3 N rows of 64 bf16
+  bool ok = true;                                       // this thread's waits so far
+  if (warp == kTcWorkers) {
+    // ---- MMA issuer (one thread): 4 k-steps per chunk, then the commit that frees the stage
     if (lane == 0) {
       const uint32_t a_base = smem_u32(As), b_base = smem_u32(Bs);
 #pragma unroll 1
       for (int c = 0; c < nchunk && ok; ++c) {
-        const int s = c % kTcStages, b = c % kTcBufs;
-        ok = mbar_wait(b_ready + b, (c / kTcBufs) & 1) && mbar_wait(full + s, (c / kTcStages) & 1);
+        const int s = c % kTcStages;
+        ok = mbar_wait(full + s, (c / kTcStages) & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t da0 = smem_desc_sw128(a_base + s * kTileA);
-        const uint64_t db0 = smem_desc_sw128(b_base + b * 3 * kTileB);
+        const uint64_t db0 = smem_desc_sw128(b_base + s * kTileB);
 #pragma unroll
         for (int ks = 0; ks < kTcKC / 16; ++ks)         // 16 bf16 = 32 bytes along k inside the swizzle row
           umma_bf16(tmem_d, da0 + (uint64_t)(ks * 2), db0 + (uint64_t)(ks * 2), idesc, (c | ks) ? 1u : 0u);
-        umma_commit(a_free + s);
-        umma_commit(b_free + b);
+        umma_commit(s_free + s);
       }
       umma_commit(done);
     }
-  } else {
-    // ---- TMA producer (one thread): keeps kTcStages X tiles in flight
+  } else if (warp == kTcWorkers + 1) {
+    // ---- TMA producer (one thread): keeps kTcStages stages in flight
     if (lane == 0) {
 #pragma unroll 1
       for (int c = 0; c < nchunk && ok; ++c) {
         const int s = c % kTcStages;
-        if (c >= kTcStages) ok = mbar_wait(a_free + s, ((c / kTcStages) - 1) & 1);
+        if (c >= kTcStages) ok = mbar_wait(s_free + s, ((c / kTcStages) - 1) & 1);
         if (!ok) break;
-        mbar_expect_tx(full + s, kTileA);
+        mbar_expect_tx(full + s, kTileA + b_bytes);
         tma_load_2d(As + s * kTileA, &mapX, c * kTcKC, row0, full + s);
+        tma_load_2d(Bs + s * kTileB, &mapB, c * kTcKC, 0, full + s);
       }
     }
+  } else {
+    ok = mbar_wait(done, 0);                            // every reader of TMEM observes the completed phase
   }
-  if (warp < 8) ok = mbar_wait(done, 0) && ok;          // every reader of TMEM observes the completed phase
   const bool fail = __syncthreads_or(ok ? 0 : 1) != 0;
   if (!fail) {
-    if (warp < 8) {
+    if (warp < kTcWorkers) {
       // thread = row: warp w reads lanes 32 (w % 4) ..., warps 0-3 the columns [0, N/2), warps 4-7 the rest
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int half = N >> 1;                          // 8, 16, 24 or 32 columns per warp
@@ -310,36 +274,53 @@ EncodeFn encode_fn() {
 
 }  // namespace
 
-// Y[q][j] = sum_k X[q][k] U[k][j] on the tensor cores.  Returns cudaErrorNotSupported when the shape or the
+size_t tc_scratch_bytes(int64_t K, int N) { return (size_t)3 * N * K * 2; }
+
+// Y[q][j] = sum_k X[q][k] U[k][j] on the tensor cores.  `scratch` (device, 16-byte aligned, at least
+// tc_scratch_bytes(K, N)) receives the bf16 operand.  Returns cudaErrorNotSupported when the shape or the
 // alignment does not fit (the caller then takes the SIMT kernel).
-cudaError_t launch_tc_lastmode(const ModeProdArgs& p, cudaStream_t st) {
+cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
   const int64_t M = p.Q, K = p.a;
   const int N = p.n_out;
   if (p.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || K % kTcKC != 0 || K < kTcKC || M < kTcM ||
-      M >= (1ll << 31) || K >= (1ll << 31) || p.sj != 1 || p.so % 4 != 0 || p.ldb_j != 1 ||
-      (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u) || (K * 2) % 16 != 0)
+      M >= (1ll << 31) || K >= (1ll << 31) || p.sj != 1 || p.so % 4 != 0 || p.ldb_j != 1 || !scratch ||
+      scratch_bytes < tc_scratch_bytes(K, N) || (reinterpret_cast<uintptr_t>(scratch) & 15u) ||
+      (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u))
     return cudaErrorNotSupported;
   EncodeFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
-  CUtensorMap map;
-  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)kTcM};
+  CUtensorMap mapX, mapB;
   const cuuint32_t estr[2] = {1, 1};
-  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p.X), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorNotSupported;
-  static const size_t smem = 1024 + kTcStages * kTileA + kTcBufs * 3 * kTileB + (2 * kTcStages + 2 * kTcBufs + 1) * 8 + 16;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)kTcM};
+    if (enc(&mapX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p.X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)(3 * N)};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
+    if (enc(&mapB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, scratch, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
+  static const size_t smem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
     attr_err = cudaFuncSetAttribute(k_tc_lastmode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   });
   if (attr_err != cudaSuccess) return attr_err;
-  TcArgs a = {p.B, p.Y, (int)M, N, (int)K, (int)p.ldb_k, (int)p.so};
+  k_tc_split<<<dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
+      p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch));
+  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so};
   const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
-  k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(map, a);
+  k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
 }
 
