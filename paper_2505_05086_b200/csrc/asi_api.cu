@@ -147,7 +147,7 @@ void layout_compress(asi_plan* pl) {
     const ModeView& v = pl->mv[m];
     if (pl->bf16 && !pl->fast_compress && v.I == 1 && pl->r[m] % 16 == 0 && pl->r[m] >= 16 && pl->r[m] <= 64 &&
         v.a % 64 == 0 && v.Q >= 128)
-      pl->tc_bytes = tc_scratch_bytes(v.a, pl->r[m]);
+      pl->tc_bytes = tc_scratch_bytes(std::max(v.a, v.Q), pl->r[m]);    // the factor, then V for the expansion
   }
   off = align_up(off + pl->tc_bytes, 256);
   pl->off_Rf = off;                                   // Cholesky factors of the fused path
@@ -194,7 +194,11 @@ void layout_compress(asi_plan* pl) {
       pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
     // tensor-core products are two launches (operand split + GEMM): V of the last mode, and the first
     // core product when it contracts the last mode
-    if (pl->tc_bytes) pl->launches_compress += 1 + (pl->core_order[0] == pl->nd - 1 ? 1 : 0);
+    if (pl->tc_bytes) {
+      const ModeView& v = pl->mv[pl->nd - 1];
+      pl->launches_compress += 1 + (pl->core_order[0] == pl->nd - 1 ? 1 : 0);
+      if (v.a % 8 == 0 && v.a >= 128 && v.Q % 8 == 0) pl->launches_compress += 1;   // the expansion as well
+    }
   }
 }
 
@@ -389,6 +393,8 @@ asi_status_t expand_mode(const asi_plan* pl, int m, const void* act, const float
   e.r = v.r;
   e.nsplit = pl->nsplit[m];
   e.q_per_split = pl->q_per_split[m];
+  e.tc_scratch = w + pl->off_tc;
+  e.tc_scratch_bytes = pl->tc_bytes;
   ASI_CUDA(launch_expand(e, pl->bf16, st));
   return ASI_OK;
 }

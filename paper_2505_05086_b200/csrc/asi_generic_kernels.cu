@@ -423,6 +423,10 @@ template <typename TX>
 static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_EXPAND, st,
                  (double)p.Q * p.a * sizeof(TX) + 4.0 * ((double)p.Q * p.r + (double)p.nsplit * p.a * p.r));
+  if constexpr (std::is_same<TX, __nv_bfloat16>::value) {
+    const cudaError_t e = launch_tc_expand(p, p.tc_scratch, p.tc_scratch_bytes, st);   // tensor cores when it fits
+    if (e != cudaErrorNotSupported) return e;
+  }
   if (p.I == 1 && p.r >= 16 && p.a >= 64 && p.Q < (1 << 30) && p.a < (1 << 30)) {
     GemmArgs g = {p.X, p.V, p.Pp, (int)p.a, p.r, (int)p.Q, p.a, (int)p.q_per_split, 0};
     return launch_gemm_t<false, TX>(g, p.nsplit, st);

@@ -44,6 +44,8 @@ struct ExpandArgs {
   int64_t O, a, I, Q;
   int r, nsplit;
   int64_t q_per_split;
+  void* tc_scratch = nullptr;      // device scratch for the tensor-core kernel's bf16 operand (optional)
+  size_t tc_scratch_bytes = 0;
 };
 
 // One mode's P = A_m (A_m^T U) in a single pass (k_fiber); Pp: [grid][a][r] partials.
@@ -158,6 +160,7 @@ cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaS
 // Tensor-core last-mode product of a bf16 tensor (tcgen05); cudaErrorNotSupported when the shape does not fit.
 cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st);
 size_t tc_scratch_bytes(int64_t K, int N);
+cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st);
 int tc_error_flag();   // != 0: a bounded wait of the tensor-core kernel expired
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);

@@ -83,20 +83,24 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
       "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
-// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of 8 rows
-// 1024 bytes apart (start address, leading and stride offsets in 16-byte units; descriptor version 1)
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+// shared-memory matrix descriptor of a 128-byte-swizzled operand (start address, leading and stride byte
+// offsets in 16-byte units; descriptor version 1).  K-major: rows of 128 bytes along K, groups of 8 rows
+// 1024 bytes apart (stride offset), the leading offset is unused.  MN-major: rows of 128 bytes along M/N
+// (64 bf16), one row per K index, groups of 8 K-rows 1024 bytes apart (stride offset), the next 64 M/N
+// elements `lbo` bytes further (leading offset).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes = 16) {
   uint64_t d = 0;
   d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)1 << 16;                 // leading byte offset (unused by swizzled K-major layouts)
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
   d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
   d |= (uint64_t)1 << 46;                 // version
   d |= (uint64_t)2 << 61;                 // 128-byte swizzle
   return d;
 }
-// instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major
-__device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, B K-major, A K-major or MN-major
+__device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N, bool a_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
 }
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
   asm volatile(
@@ -117,8 +121,10 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {   /
                : "memory");
 }
 struct TcArgs {
-  float* Y;            // [M][ldy]
-  int M, N, K, ldy;
+  float* Y;            // [M][ldy]; CTA (., s) writes Y + s * y_split
+  int M, N, K, ldy;    // K: total extent of the contraction
+  int k_per_split;     // multiple of 64; CTA (., s) contracts [s * k_per_split, min(K, (s + 1) * k_per_split))
+  int64_t y_split;
 };
 
 // Bt[t*n + j][k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
@@ -147,8 +153,10 @@ __global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, i
   }
 }
 
-__global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX,
-                                                                const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+// A_MN = false: D[m][n] = sum_k X[m][k] B[n][k] (X K-major: tile [128 m x 64 k] in one TMA box);
+// A_MN = true:  D[m][n] = sum_k X[k][m] B[n][k] (X MN-major: tile [64 k x 128 m] as two boxes of 64 m).
+template <bool A_MN>
+__device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUtensorMap& mapB, const TcArgs& p) {
   extern __shared__ __align__(1024) uint8_t tc_smem[];
   // carve-up: per stage the X tile and the operand tile, then barriers
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem) + 1023) & ~(uintptr_t)1023);
@@ -161,8 +169,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row0 = blockIdx.x * kTcM;
-  const int nchunk = p.K / kTcKC;
+  const int k_begin = blockIdx.y * p.k_per_split;
+  const int k_end = (p.K - k_begin < p.k_per_split) ? p.K : k_begin + p.k_per_split;
+  const int nchunk = (k_end - k_begin + kTcKC - 1) / kTcKC;   // a ragged last chunk is zero-filled by TMA
   const int N = p.N;
+  float* Yout = p.Y + (int64_t)blockIdx.y * p.y_split;
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(s_free + s, 1); }
@@ -182,7 +193,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
 
   // The three bf16 terms of the factor are stacked along the operand's rows: one MMA of width 3 N per
   // k-step reads the X tile once and leaves the three partial products in three column groups of TMEM.
-  const uint32_t idesc = instr_desc_bf16(kTcM, 3 * N);
+  const uint32_t idesc = instr_desc_bf16(kTcM, 3 * N, A_MN);
   const uint32_t b_bytes = (uint32_t)(3 * N) * 128u;    // operand tile: 3 N rows of 64 bf16
   bool ok = true;                                       // this thread's waits so far
   if (warp == kTcWorkers) {
@@ -195,11 +206,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
         ok = mbar_wait(full + s, (c / kTcStages) & 1);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t da0 = smem_desc_sw128(a_base + s * kTileA);
+        // a k-step is 16 bf16: 32 bytes inside the swizzle row of a K-major tile, 16 rows (2048 bytes) of
+        // an MN-major tile (start-address field in 16-byte units)
+        const uint64_t da0 = smem_desc_sw128(a_base + s * kTileA, A_MN ? kTileA / 2 : 16);
         const uint64_t db0 = smem_desc_sw128(b_base + s * kTileB);
 #pragma unroll
-        for (int ks = 0; ks < kTcKC / 16; ++ks)         // 16 bf16 = 32 bytes along k inside the swizzle row
-          umma_bf16(tmem_d, da0 + (uint64_t)(ks * 2), db0 + (uint64_t)(ks * 2), idesc, (c | ks) ? 1u : 0u);
+        for (int ks = 0; ks < kTcKC / 16; ++ks)
+          umma_bf16(tmem_d, da0 + (uint64_t)(ks * (A_MN ? 128 : 2)), db0 + (uint64_t)(ks * 2), idesc,
+                    (c | ks) ? 1u : 0u);
         umma_commit(s_free + s);
       }
       umma_commit(done);
@@ -213,8 +227,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
         if (c >= kTcStages) ok = mbar_wait(s_free + s, ((c / kTcStages) - 1) & 1);
         if (!ok) break;
         mbar_expect_tx(full + s, kTileA + b_bytes);
-        tma_load_2d(As + s * kTileA, &mapX, c * kTcKC, row0, full + s);
-        tma_load_2d(Bs + s * kTileB, &mapB, c * kTcKC, 0, full + s);
+        const int kc = k_begin + c * kTcKC;
+        if (A_MN) {
+          tma_load_2d(As + s * kTileA, &mapX, row0, kc, full + s);
+          tma_load_2d(As + s * kTileA + kTileA / 2, &mapX, row0 + 64, kc, full + s);
+        } else {
+          tma_load_2d(As + s * kTileA, &mapX, kc, row0, full + s);
+        }
+        tma_load_2d(Bs + s * kTileB, &mapB, kc, 0, full + s);
       }
     }
   } else {
@@ -240,7 +260,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
 #pragma unroll
           for (int i = 0; i < 8; ++i)                   // small terms first
             o[i] = (__uint_as_float(l[i]) + __uint_as_float(m[i])) + __uint_as_float(h[i]);
-          float* y = p.Y + (int64_t)row * p.ldy + col0 + cc;
+          float* y = Yout + (int64_t)row * p.ldy + col0 + cc;
           *reinterpret_cast<float4*>(y) = make_float4(o[0], o[1], o[2], o[3]);
           *reinterpret_cast<float4*>(y + 4) = make_float4(o[4], o[5], o[6], o[7]);
         }
@@ -253,6 +273,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_cons
   __syncthreads();
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(256) : "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX,
+                                                                const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+  tc_gemm_body<false>(mapX, mapB, p);
+}
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_expand(const __grid_constant__ CUtensorMap mapX,
+                                                              const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+  tc_gemm_body<true>(mapX, mapB, p);
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -318,9 +347,57 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
       p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch));
-  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so};
+  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0};
   const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
   k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
+  return cudaGetLastError();
+}
+
+// Pp[s][k][j] = sum_{q in split s} X[q][k] V[q][j] on the tensor cores (the expansion P = A_m V of the last
+// mode, X bf16 [Q x a], V fp32 [Q x r]).  `scratch` as above, at least tc_scratch_bytes(Q, r).
+cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  const int64_t Q = e.Q, A = e.a;
+  const int N = e.r;
+  if (e.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || A % 8 != 0 || A < kTcM || Q % 8 != 0 || Q < kTcKC ||
+      Q >= (1ll << 31) || A >= (1ll << 31) || e.q_per_split % kTcKC != 0 || e.q_per_split >= (1ll << 31) ||
+      e.nsplit < 1 || !scratch || scratch_bytes < tc_scratch_bytes(Q, N) ||
+      (reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(e.X) & 15u) ||
+      (reinterpret_cast<uintptr_t>(e.Pp) & 15u))
+    return cudaErrorNotSupported;
+  EncodeFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  CUtensorMap mapX, mapB;
+  const cuuint32_t estr[2] = {1, 1};
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)A, (cuuint64_t)Q};
+    const cuuint64_t strides[1] = {(cuuint64_t)A * 2};
+    const cuuint32_t box[2] = {64, 64};
+    if (enc(&mapX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(e.X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)Q, (cuuint64_t)(3 * N)};
+    const cuuint64_t strides[1] = {(cuuint64_t)Q * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
+    if (enc(&mapB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, scratch, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
+  static const size_t smem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(k_tc_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  });
+  if (attr_err != cudaSuccess) return attr_err;
+  k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
+      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch));
+  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N};
+  dim3 grid((unsigned)((A + kTcM - 1) / kTcM), (unsigned)e.nsplit);
+  k_tc_expand<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
 }
 
