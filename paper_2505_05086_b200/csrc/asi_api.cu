@@ -139,16 +139,22 @@ void layout_compress(asi_plan* pl) {
     pl->off_Gp[m] = off;
     off = align_up(off + (size_t)pl->nchunk[m] * v.r * v.r * 8, 256);
   }
-  // bf16 operand of the tensor-core kernel: last-mode products of bf16 tensors with a wide factor
+  // bf16 operand of the tensor-core kernels: products of bf16 tensors with a wide factor (16..64 columns, a
+  // multiple of 16) over the last mode (a_m a multiple of 64, >= 128 fibers) or over a mode whose inner
+  // extent I is a multiple of 64; the same scratch then serves the mode's expansion (operand = V_m)
   pl->off_tc = off;
   pl->tc_bytes = 0;
-  {
-    const int m = pl->nd - 1;
-    const ModeView& v = pl->mv[m];
-    if (pl->bf16 && !pl->fast_compress && v.I == 1 && pl->r[m] % 16 == 0 && pl->r[m] >= 16 && pl->r[m] <= 64 &&
-        v.a % 64 == 0 && v.Q >= 128)
-      pl->tc_bytes = tc_scratch_bytes(std::max(v.a, v.Q), pl->r[m]);    // the factor, then V for the expansion
-  }
+  for (int m = 0; m < pl->nd; ++m) pl->tc_mode[m] = 0;
+  if (pl->bf16 && !pl->fast_compress)
+    for (int m = 0; m < pl->nd; ++m) {
+      const ModeView& v = pl->mv[m];
+      if (pl->r[m] % 16 != 0 || pl->r[m] < 16 || pl->r[m] > 64) continue;
+      const bool last = v.I == 1 && v.a % 64 == 0 && v.Q >= 128;
+      const bool inner = v.I >= 64 && v.I % 64 == 0 && v.O < 65536;
+      if (!last && !inner) continue;
+      pl->tc_mode[m] = last ? 1 : 2;
+      pl->tc_bytes = std::max(pl->tc_bytes, tc_scratch_bytes(std::max(v.a, v.Q), pl->r[m]));
+    }
   off = align_up(off + pl->tc_bytes, 256);
   pl->off_Rf = off;                                   // Cholesky factors of the fused path
   off = align_up(off + (size_t)ASI_MAX_MODES * kRfStride * 8, 256);
@@ -194,10 +200,14 @@ void layout_compress(asi_plan* pl) {
       pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
     // tensor-core products are two launches (operand split + GEMM): V of the last mode, and the first
     // core product when it contracts the last mode
-    if (pl->tc_bytes) {
-      const ModeView& v = pl->mv[pl->nd - 1];
-      pl->launches_compress += 1 + (pl->core_order[0] == pl->nd - 1 ? 1 : 0);
-      if (v.a % 8 == 0 && v.a >= 128 && v.Q % 8 == 0) pl->launches_compress += 1;   // the expansion as well
+    // a tensor-core product is two launches (operand split + GEMM): V_m, the expansion when it fits too,
+    // and the first core product when it contracts such a mode of the bf16 activation
+    for (int m = 0; m < pl->nd; ++m) {
+      if (!pl->tc_mode[m]) continue;
+      const ModeView& v = pl->mv[m];
+      pl->launches_compress += 1;
+      if (pl->tc_mode[m] == 2 || (v.a % 8 == 0 && v.a >= 128 && v.Q % 8 == 0)) pl->launches_compress += 1;
+      if (pl->core_order[0] == m) pl->launches_compress += 1;
     }
   }
 }

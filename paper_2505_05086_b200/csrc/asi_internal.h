@@ -220,7 +220,8 @@ struct asi_plan {
   // compress workspace (byte offsets)
   size_t off_V, off_Pp[ASI_MAX_MODES], off_Pred[ASI_MAX_MODES], off_Gp[ASI_MAX_MODES], off_T[2];
   size_t off_Rf, off_Pg[ASI_MAX_MODES];
-  size_t off_tc, tc_bytes;         // bf16 operand of the tensor-core last-mode product (0 bytes: not used)
+  size_t off_tc, tc_bytes;         // bf16 operand of the tensor-core products (0 bytes: not used)
+  int tc_mode[ASI_MAX_MODES];      // 0: SIMT, 1: last-mode tensor-core kernels, 2: inner-extent (token) kernels
   int nsplit[ASI_MAX_MODES], nchunk[ASI_MAX_MODES];
   int64_t q_per_split[ASI_MAX_MODES];
   int core_order[ASI_MAX_MODES];

@@ -83,6 +83,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
       "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+      : "memory");
+}
 // shared-memory matrix descriptor of a 128-byte-swizzled operand (start address, leading and stride byte
 // offsets in 16-byte units; descriptor version 1).  K-major: rows of 128 bytes along K, groups of 8 rows
 // 1024 bytes apart (stride offset), the leading offset is unused.  MN-major: rows of 128 bytes along M/N
@@ -125,11 +132,12 @@ struct TcArgs {
   int M, N, K, ldy;    // K: total extent of the contraction
   int k_per_split;     // multiple of 64; CTA (., s) contracts [s * k_per_split, min(K, (s + 1) * k_per_split))
   int64_t y_split;
+  int inner;           // kTcTokenExpand: K enumerates (o, i) with i < inner (a multiple of 64)
 };
 
-// Bt[t*n + j][k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
+// Bt[(t*n + j) * ldb + k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
 __global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, int ldu, int K, int N,
-                                                  __nv_bfloat16* __restrict__ Bt) {
+                                                  __nv_bfloat16* __restrict__ Bt, int64_t ldb) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -146,16 +154,22 @@ __global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, i
       const float r1 = u - __bfloat162float(h);
       const __nv_bfloat16 m = __float2bfloat16_rn(r1);
       const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
-      Bt[(int64_t)j * K + k] = h;
-      Bt[(int64_t)(N + j) * K + k] = m;
-      Bt[(int64_t)(2 * N + j) * K + k] = l;
+      Bt[(int64_t)j * ldb + k] = h;
+      Bt[(int64_t)(N + j) * ldb + k] = m;
+      Bt[(int64_t)(2 * N + j) * ldb + k] = l;
     }
   }
 }
 
-// A_MN = false: D[m][n] = sum_k X[m][k] B[n][k] (X K-major: tile [128 m x 64 k] in one TMA box);
-// A_MN = true:  D[m][n] = sum_k X[k][m] B[n][k] (X MN-major: tile [64 k x 128 m] as two boxes of 64 m).
-template <bool A_MN>
+// How the X operand of D[m][n] = sum_k A(m, k) B[n][k] is laid out in memory:
+//   kTcLast        X[m][k], k contiguous: one box [128 m x 64 k] (K-major);            CTA (mt, split of K)
+//   kTcLastExpand  X[k][m], m contiguous: two boxes [64 k x 64 m] (MN-major);          CTA (mt, split of K)
+//   kTcToken       X[o][k][m], m contiguous, one o per CTA row: two boxes (MN-major);  CTA (mt, o)
+//   kTcTokenExpand X[o][m][i], i contiguous, K = (o, i) flattened: one box (K-major);  CTA (mt, split of K)
+// Rows of a box that fall outside the tensor are zero-filled by TMA.
+enum TcMode { kTcLast = 0, kTcLastExpand = 1, kTcToken = 2, kTcTokenExpand = 3 };
+
+template <int MODE>
 __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUtensorMap& mapB, const TcArgs& p) {
   extern __shared__ __align__(1024) uint8_t tc_smem[];
   // carve-up: per stage the X tile and the operand tile, then barriers
@@ -168,9 +182,10 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUte
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr bool A_MN = (MODE == kTcLastExpand || MODE == kTcToken);
   const int row0 = blockIdx.x * kTcM;
-  const int k_begin = blockIdx.y * p.k_per_split;
-  const int k_end = (p.K - k_begin < p.k_per_split) ? p.K : k_begin + p.k_per_split;
+  const int k_begin = (MODE == kTcToken) ? 0 : blockIdx.y * p.k_per_split;
+  const int k_end = (MODE == kTcToken || p.K - k_begin < p.k_per_split) ? p.K : k_begin + p.k_per_split;
   const int nchunk = (k_end - k_begin + kTcKC - 1) / kTcKC;   // a ragged last chunk is zero-filled by TMA
   const int N = p.N;
   float* Yout = p.Y + (int64_t)blockIdx.y * p.y_split;
@@ -228,9 +243,15 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUte
         if (!ok) break;
         mbar_expect_tx(full + s, kTileA + b_bytes);
         const int kc = k_begin + c * kTcKC;
-        if (A_MN) {
+        if (MODE == kTcLastExpand) {
           tma_load_2d(As + s * kTileA, &mapX, row0, kc, full + s);
           tma_load_2d(As + s * kTileA + kTileA / 2, &mapX, row0 + 64, kc, full + s);
+        } else if (MODE == kTcToken) {
+          tma_load_3d(As + s * kTileA, &mapX, row0, kc, blockIdx.y, full + s);
+          tma_load_3d(As + s * kTileA + kTileA / 2, &mapX, row0 + 64, kc, blockIdx.y, full + s);
+        } else if (MODE == kTcTokenExpand) {
+          const int o = kc / p.inner;
+          tma_load_3d(As + s * kTileA, &mapX, kc - o * p.inner, row0, o, full + s);
         } else {
           tma_load_2d(As + s * kTileA, &mapX, kc, row0, full + s);
         }
@@ -277,11 +298,19 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUte
 
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_lastmode(const __grid_constant__ CUtensorMap mapX,
                                                                 const __grid_constant__ CUtensorMap mapB, TcArgs p) {
-  tc_gemm_body<false>(mapX, mapB, p);
+  tc_gemm_body<kTcLast>(mapX, mapB, p);
 }
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_expand(const __grid_constant__ CUtensorMap mapX,
                                                               const __grid_constant__ CUtensorMap mapB, TcArgs p) {
-  tc_gemm_body<true>(mapX, mapB, p);
+  tc_gemm_body<kTcLastExpand>(mapX, mapB, p);
+}
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_token(const __grid_constant__ CUtensorMap mapX,
+                                                             const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+  tc_gemm_body<kTcToken>(mapX, mapB, p);
+}
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_token_expand(const __grid_constant__ CUtensorMap mapX,
+                                                                    const __grid_constant__ CUtensorMap mapB, TcArgs p) {
+  tc_gemm_body<kTcTokenExpand>(mapX, mapB, p);
 }
 
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -303,12 +332,101 @@ EncodeFn encode_fn() {
 
 }  // namespace
 
-size_t tc_scratch_bytes(int64_t K, int N) { return (size_t)3 * N * K * 2; }
+size_t tc_scratch_bytes(int64_t K, int N) { return (size_t)3 * N * ((K + 63) / 64 * 64) * 2; }
+
+namespace {
+constexpr size_t kTcSmem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
+
+bool encode_bf16_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+                     const cuuint32_t* box) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box,
+             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+template <typename K>
+cudaError_t tc_opt_in(K kernel) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem);
+}
+
+// V[o][i][j] = sum_k X[o][k][i] U[k][j]: a middle mode of a bf16 token tensor (I = inner extent, a multiple of 64)
+cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  const int N = p.n_out;
+  const int64_t Kp = (p.a + 63) / 64 * 64;
+  if (p.I < 64 || p.I % 64 != 0 || p.O < 1 || p.O >= 65536 || N % 16 != 0 || N < 16 || N > kTcNMax || p.a < 1 ||
+      p.a >= (1ll << 31) || p.I >= (1ll << 31) || p.sj != 1 || p.si != N || p.so != p.I * N || p.ldb_j != 1 ||
+      !scratch || scratch_bytes < tc_scratch_bytes(p.a, N) || (reinterpret_cast<uintptr_t>(scratch) & 15u) ||
+      (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u))
+    return cudaErrorNotSupported;
+  CUtensorMap mapX, mapB;
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)p.I, (cuuint64_t)p.a, (cuuint64_t)p.O};
+    const cuuint64_t strides[2] = {(cuuint64_t)p.I * 2, (cuuint64_t)p.a * p.I * 2};
+    const cuuint32_t box[3] = {64, 64, 1};
+    if (!encode_bf16_map(&mapX, p.X, 3, dims, strides, box)) return cudaErrorNotSupported;
+  }
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)p.a, (cuuint64_t)(3 * N)};
+    const cuuint64_t strides[1] = {(cuuint64_t)Kp * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
+    if (!encode_bf16_map(&mapB, scratch, 2, dims, strides, box)) return cudaErrorNotSupported;
+  }
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] { attr_err = tc_opt_in(k_tc_token); });
+  if (attr_err != cudaSuccess) return attr_err;
+  k_tc_split<<<dim3((unsigned)((p.a + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
+      p.B, (int)p.ldb_k, (int)p.a, N, static_cast<__nv_bfloat16*>(scratch), Kp);
+  TcArgs a = {p.Y, (int)p.I, N, (int)p.a, N, (int)Kp, p.so, 0};
+  dim3 grid((unsigned)((p.I + kTcM - 1) / kTcM), (unsigned)p.O);
+  k_tc_token<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
+  return cudaGetLastError();
+}
+
+// Pp[s][k][j] = sum_{(o,i) in split s} X[o][k][i] V[o][i][j]: the expansion of a middle mode
+cudaError_t launch_tc_token_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  const int N = e.r;
+  const int64_t Q = e.Q;
+  if (e.I < 64 || e.I % 64 != 0 || e.O < 1 || e.O >= 65536 || N % 16 != 0 || N < 16 || N > kTcNMax || e.a < 1 ||
+      e.a >= (1ll << 31) || Q >= (1ll << 31) || e.q_per_split % kTcKC != 0 || e.q_per_split >= (1ll << 31) ||
+      e.nsplit < 1 || !scratch || scratch_bytes < tc_scratch_bytes(Q, N) ||
+      (reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(e.X) & 15u) ||
+      (reinterpret_cast<uintptr_t>(e.Pp) & 15u))
+    return cudaErrorNotSupported;
+  CUtensorMap mapX, mapB;
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)e.I, (cuuint64_t)e.a, (cuuint64_t)e.O};
+    const cuuint64_t strides[2] = {(cuuint64_t)e.I * 2, (cuuint64_t)e.a * e.I * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTcM, 1};
+    if (!encode_bf16_map(&mapX, e.X, 3, dims, strides, box)) return cudaErrorNotSupported;
+  }
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)Q, (cuuint64_t)(3 * N)};
+    const cuuint64_t strides[1] = {(cuuint64_t)Q * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
+    if (!encode_bf16_map(&mapB, scratch, 2, dims, strides, box)) return cudaErrorNotSupported;
+  }
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] { attr_err = tc_opt_in(k_tc_token_expand); });
+  if (attr_err != cudaSuccess) return attr_err;
+  k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
+      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
+  TcArgs a = {e.Pp, (int)e.a, N, (int)Q, N, (int)e.q_per_split, e.a * N, (int)e.I};
+  dim3 grid((unsigned)((e.a + kTcM - 1) / kTcM), (unsigned)e.nsplit);
+  k_tc_token_expand<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
+  return cudaGetLastError();
+}
+}  // namespace
+
 
 // Y[q][j] = sum_k X[q][k] U[k][j] on the tensor cores.  `scratch` (device, 16-byte aligned, at least
 // tc_scratch_bytes(K, N)) receives the bf16 operand.  Returns cudaErrorNotSupported when the shape or the
 // alignment does not fit (the caller then takes the SIMT kernel).
 cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  if (p.I != 1) return launch_tc_token(p, scratch, scratch_bytes, st);
   const int64_t M = p.Q, K = p.a;
   const int N = p.n_out;
   if (p.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || K % kTcKC != 0 || K < kTcKC || M < kTcM ||
@@ -346,8 +464,8 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
   });
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch));
-  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0};
+      p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch), K);
+  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0, 0};
   const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
   k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -356,6 +474,7 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
 // Pp[s][k][j] = sum_{q in split s} X[q][k] V[q][j] on the tensor cores (the expansion P = A_m V of the last
 // mode, X bf16 [Q x a], V fp32 [Q x r]).  `scratch` as above, at least tc_scratch_bytes(Q, r).
 cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+  if (e.I != 1) return launch_tc_token_expand(e, scratch, scratch_bytes, st);
   const int64_t Q = e.Q, A = e.a;
   const int N = e.r;
   if (e.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || A % 8 != 0 || A < kTcM || Q % 8 != 0 || Q < kTcKC ||
@@ -394,8 +513,8 @@ cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_
   });
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch));
-  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N};
+      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
+  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N, 0};
   dim3 grid((unsigned)((A + kTcM - 1) / kTcM), (unsigned)e.nsplit);
   k_tc_expand<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();

@@ -139,13 +139,16 @@ def test_linear_layers(dims, ranks, cout, rho, gen):
 
 # bf16 token layers whose last-mode products (V_3 = A_(3)^T U_3, the first core product and, when the token
 # count is a multiple of 8, the expansion P_3 = A_(3) V_3) take the tensor-core kernels: last dimension a
-# multiple of 64, last rank 16 / 32 / 48 / 64, at least 128 tokens; the token counts leave ragged tiles.
+# multiple of 64, last rank 16 / 32 / 48 / 64, at least 128 tokens; the token counts leave ragged tiles.  With
+# a token-mode rank of 16 / 32 the token-mode products V_2, P_2 run there as well (3-D TMA boxes).
 LINEAR_TC = [  # (dims, ranks, cout, rho, generating ranks)
     ((4, 40, 128), (3, 6, 16), 24, (0.6, 0.8, 0.93), (4, 12, 32)),
     ((2, 197, 192), (2, 8, 32), 40, (0.5, 0.85, 0.96), (2, 16, 64)),
     ((3, 100, 320), (3, 8, 48), 32, (0.6, 0.85, 0.975), (3, 16, 96)),
     ((8, 64, 256), (4, 8, 64), 48, (0.7, 0.85, 0.985), (8, 16, 128)),
     ((4, 48, 192), (3, 6, 32), 24, (0.6, 0.8, 0.96), (4, 12, 64)),      # expansion tile with 64 valid rows
+    ((4, 72, 128), (3, 16, 16), 24, (0.6, 0.93, 0.93), (4, 32, 32)),    # token mode on the tensor cores too
+    ((2, 197, 192), (2, 32, 32), 40, (0.5, 0.96, 0.96), (2, 64, 64)),   # 197 tokens: ragged K chunks and row tiles
 ]
 
 
