@@ -97,11 +97,12 @@ void layout_compress(asi_plan* pl) {
     const int64_t np = 256 / pl->dims[2], planes = pl->dims[0] * pl->dims[1];
     pl->plane_grid = (int)std::min<int64_t>((planes + np - 1) / np, 296);
   }
-  if (pl->small_rank)
+  // one-pass kernel for every mode with a rank <= 8 and a short fiber, whatever the other modes' ranks
+  if (!pl->fast_compress && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY))
     for (int m = 0; m < pl->nd; ++m) {
       if (pl->plane && m >= 2) continue;
       const ModeView& v = pl->mv[m];
-      if (v.a <= 128 && fiber_smem((int)v.a) <= kSmemLimit) {
+      if (pl->r[m] <= 8 && v.a <= 128 && fiber_smem((int)v.a) <= kSmemLimit) {
         pl->fiber[m] = true;
         pl->fiber_grid[m] = (int)std::min<int64_t>(fiber_tiles(v.O, v.a, v.I), 296);
       }
