@@ -1,13 +1,16 @@
-// Tensor-core kernel (sm_100a: tcgen05.mma, TMEM accumulator, TMA operand staging) for the one step of
-// the path that is a plain dense contraction: the last-mode product of a bf16 tensor with a wide factor,
-//   Y[q][j] = sum_k X[q][k] U[k][j],   X bf16 [Q x a] (k contiguous), U fp32 [a x n], n = 16..64,
-// i.e. V_3 = A_(3)^T U_3 and the first core product of token layers (Algorithm 1 on a B x N x D
-// activation).  X is exact in bf16; the fp32 factor is split into three bf16 terms (24 mantissa bits),
-// so one MMA of width 3 n per k-step (the three terms stacked as operand rows) yields three partial products
-// in TMEM whose sum reproduces the fp32 product to fp32 rounding.
+// Tensor-core kernels (sm_100a: tcgen05.mma, TMEM accumulator, TMA operand staging) for the steps of the
+// path that are plain dense contractions: products of a bf16 tensor with a wide fp32 factor (16..64
+// columns) in Algorithm 1 on token layers (B x N x D activations),
+//   k_tc_lastmode      Y[q][j]     = sum_k X[q][k] U[k][j]          V_3 = A_(3)^T U_3, first core product
+//   k_tc_expand        P[k][j]     = sum_q X[q][k] V[q][j]          P_3 = A_(3) V_3 (split-K partials)
+//   k_tc_token         V[o][i][j]  = sum_k X[o][k][i] U[k][j]       V_2 = A_(2)^T U_2, one sample o per CTA row
+//   k_tc_token_expand  P[k][j]     = sum_{o,i} X[o][k][i] V[o][i][j]  P_2 = A_(2) V_2 (split-K partials)
+// X is exact in bf16; the fp32 factor (U or V) is split into three bf16 terms (24 mantissa bits), so one
+// MMA of width 3 n per k-step (the three terms stacked as operand rows) yields three partial products in
+// TMEM whose sum reproduces the fp32 product to fp32 rounding.
 //
 // k_tc_split writes the stacked operand [3 n][K] (bf16, K contiguous: hi rows, then mid, then lo) to
-// scratch memory once per product; k_tc_lastmode then streams both operands by TMA.  One CTA owns a
+// scratch memory once per product; the GEMM kernel then streams both operands by TMA.  One CTA owns a
 // 128-row tile of Y and walks K in chunks of 64, its warps in three roles that meet only through mbarriers:
 //   * a producer thread keeps four stages in flight, each the X tile [128 x 64] and the operand tile
 //     [3 n x 64] (cp.async.bulk.tensor, 128-byte swizzle);
