@@ -60,6 +60,26 @@ def test_plan_query_matches_closed_forms(asi):
     assert p3.info.compressed_elems == O.compressed_elems((32, 197, 768), (8, 32, 64))
 
 
+@pytest.mark.parametrize("dims,ranks,on_tensor_cores", [
+    ((32, 197, 768), (8, 32, 64), True),      # ViT-Base MLP input: last mode and token mode both qualify
+    ((8, 64, 256), (4, 8, 64), True),         # last mode only
+    ((8, 64, 256), (4, 8, 60), False),        # rank not a multiple of 16
+    ((8, 64, 250), (4, 8, 64), False),        # feature extent not a multiple of the K chunk
+])
+def test_bf16_plans_pick_the_tensor_core_products_by_shape(asi, dims, ranks, on_tensor_cores):
+    """A bf16 plan whose dense products fit the tensor-core tiling enqueues the factor-split launches
+    and reserves their scratch; any other plan is launch-for-launch the fp32 plan."""
+    tc = asi.Plan("linear", dims, ranks, cout=128, bf16=True)
+    f32 = asi.Plan("linear", dims, ranks, cout=128)
+    more = tc.launch_count(0) - f32.launch_count(0)
+    extra = tc.info.compress_ws_bytes - f32.info.compress_ws_bytes
+    if on_tensor_cores:
+        assert more > 0 and extra > 0
+    else:
+        assert more == 0 and extra == 0
+    assert tc.launch_count(1) == f32.launch_count(1)
+
+
 @pytest.mark.parametrize("kw,code", [
     (dict(dims=(8, 32, 16, 16), ranks=(9, 8, 8, 8)), 3),            # r_1 > a_1
     (dict(dims=(8, 32, 16, 16), ranks=(0, 8, 8, 8)), 3),
