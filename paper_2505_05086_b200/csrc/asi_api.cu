@@ -196,11 +196,9 @@ void layout_compress(asi_plan* pl) {
   pl->compress_ws = off;
   pl->launches_compress = 3;
   if (!pl->fast_compress) {
-    pl->launches_compress = 2 + pl->nd;                                    // reduction/QR pair, core chain
+    pl->launches_compress = 2 + pl->nd + (pl->small_rank ? 0 : 1);         // reduction/QR kernels, core chain
     for (int m = 0; m < pl->nd; ++m)
       pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
-    // tensor-core products are two launches (operand split + GEMM): V of the last mode, and the first
-    // core product when it contracts the last mode
     // a tensor-core product is two launches (operand split + GEMM): V_m, the expansion when it fits too,
     // and the first core product when it contracts such a mode of the bf16 activation
     for (int m = 0; m < pl->nd; ++m) {

@@ -4,7 +4,7 @@
 //
 //   k_modeprod : Y = X x_m B^T-like small contraction over one mode (Sec. 3.2, m-mode product)
 //   k_expand   : P_m = A_m V_m, split over the columns of the unfolding (Algorithm 1)
-//   k_qr_gram / k_qr_solve : Orthogonalize(P) as Cholesky-QR with the Gram matrix and the
+//   k_qr_gram / k_qr_gsum / k_qr_solve : Orthogonalize(P) as Cholesky-QR with the Gram matrix and the
 //                triangular solve in fp64 -- in exact arithmetic the Gram-Schmidt basis
 //   k_conv_tail: terms 4 and 5 of C_ASI (appendix "Speedup")
 #include <cuda_bf16.h>
@@ -828,84 +828,242 @@ __global__ void __launch_bounds__(256) k_qr_gram(QRArgs args) {
   const QRMode M = args.m[blockIdx.y];
   const int c = blockIdx.x;
   if (c >= M.nchunk) return;
-  __shared__ double Ps[kQRRows][ASI_MAX_RANK];
+  __shared__ double Ps[kQRRows * ASI_MAX_RANK];      // this chunk's rows of P, pitch r
+  constexpr int kPer = 16;
+  static_assert(kQRRows * ASI_MAX_RANK == kPer * 256, "one thread holds 16 elements of a full chunk");
   const int tid = threadIdx.x;
   const int r = M.r;
   const int row0 = c * kQRRows;
-  for (int idx = tid; idx < kQRRows * r; idx += 256) {
-    const int rl = idx / r, j = idx % r;
-    const int row = row0 + rl;
-    double v = 0.0;
-    if (row < M.a) {
-      for (int s = 0; s < M.nsplit; ++s) v += (double)M.Pp[((int64_t)s * M.a + row) * r + j];
-      M.Pred[(int64_t)row * r + j] = v;
+  const int nrows = min(kQRRows, M.a - row0);
+  const int nval = nrows * r;                        // the chunk is one contiguous run of P
+  const int64_t base = (int64_t)row0 * r;
+  // A thread has 16 accumulators: `ethr` elements (a power of two) times 16 / ethr lanes that take
+  // every (16 / ethr)-th split, so 16 loads are in flight whatever the chunk's size; the lanes of
+  // an element then fold pairwise.  The order of the sum is fixed by (nval, nsplit) alone.
+  int ethr = 1, lg = 0;
+  while (ethr * 256 < nval) { ethr <<= 1; ++lg; }
+  const int ssub = 16 >> lg;
+  const int64_t sstride = (int64_t)M.a * r;
+  double acc[kPer];
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
+  for (int s0 = 0; s0 < M.nsplit; s0 += ssub) {
+    float t[kPer];
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const int idx = tid + (q & (ethr - 1)) * 256;
+      const int s = s0 + (q >> lg);
+      const bool on = idx < nval && s < M.nsplit;
+      // Every load is issued, from a clamped address when off, and nothing here touches its
+      // result: a use or a condition next to a load makes the following loads wait for it.
+      t[q] = __ldcg(M.Pp + (on ? s * sstride + base + idx : 0));
     }
-    Ps[rl][j] = v;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const bool on = tid + (q & (ethr - 1)) * 256 < nval && s0 + (q >> lg) < M.nsplit;
+      acc[q] += on ? (double)t[q] : 0.0;
+    }
+  }
+#pragma unroll
+  for (int h = kPer / 2; h >= 1; h >>= 1)
+    if (h >= ethr) {
+#pragma unroll
+      for (int q = 0; q < h; ++q) acc[q] += acc[q + h];
+    }
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    const int idx = tid + q * 256;
+    if (q < ethr && idx < nval) {
+      M.Pred[base + idx] = acc[q];
+      Ps[idx] = acc[q];
+    }
   }
   __syncthreads();
-  for (int idx = tid; idx < r * r; idx += 256) {
-    const int i = idx / r, j = idx % r;
-    if (j < i) continue;
-    double g = 0.0;
-#pragma unroll 8
-    for (int rl = 0; rl < kQRRows; ++rl) g = fma(Ps[rl][i], Ps[rl][j], g);
-    M.Gp[((int64_t)c * r + i) * r + j] = g;
+  // Thread (ti, tj) owns G[ti + 16x][tj + 16y]: per row of P it reads 4 + 4 values for 16 products.
+  const int ti = tid >> 4, tj = tid & 15;
+  double g[4][4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) g[x][y] = 0.0;
+  for (int rl = 0; rl < nrows; ++rl) {
+    const double* prow = Ps + rl * r;
+    double pi[4], pj[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      pi[t] = (ti + 16 * t < r) ? prow[ti + 16 * t] : 0.0;
+      pj[t] = (tj + 16 * t < r) ? prow[tj + 16 * t] : 0.0;
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) g[x][y] = fma(pi[x], pj[y], g[x][y]);
   }
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int i = ti + 16 * x, j = tj + 16 * y;
+      if (i < r && j < r && j >= i) M.Gp[((int64_t)c * r + i) * r + j] = g[x][y];
+    }
 }
 
+// k_qr_gsum: G = sum of the row chunks' shares, chunk by chunk in order, left in the place of
+// share 0, so that the solve kernel's CTAs read r*r numbers each instead of every share.  One
+// thread per element of the upper triangle, eight loads in flight.
+__global__ void __launch_bounds__(256) k_qr_gsum(QRArgs args) {
+  const QRMode M = args.m[blockIdx.y];
+  const int rr = M.r * M.r;
+  const int e = blockIdx.x * 256 + threadIdx.x;
+  if (e >= rr || (e % M.r) < (e / M.r)) return;
+  const double* G = M.Gp + e;
+  double acc = 0.0;
+#pragma unroll 8
+  for (int cc = 0; cc < M.nchunk; ++cc) acc += __ldcg(G + (int64_t)cc * rr);
+  M.Gp[e] = acc;
+}
+
+// k_qr_solve keeps the running Schur complement of the Cholesky factorisation and the rows it
+// solves in registers; shared memory carries only what one step hands to the next (the pivot
+// row, the next unknown of each row) and R^T for the row solve.
+constexpr int kQRPitch = ASI_MAX_RANK + 1;
+
 __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
+  static_assert(ASI_MAX_RANK == 64 && kQRRows == 64, "4 x 4 slots of stride 16; four threads per row");
   const QRMode M = args.m[blockIdx.y];
   const int c = blockIdx.x;
-  if (c >= M.nchunk) return;
-  __shared__ double G[ASI_MAX_RANK][ASI_MAX_RANK + 1];
+  const int row0 = c * kQRRows;
+  if (c >= M.nchunk || row0 >= M.a) return;
+  __shared__ double Rt[ASI_MAX_RANK * kQRPitch];      // Rt[k][j] = R[j][k], k > j
+  __shared__ double rowbuf[2][ASI_MAX_RANK];          // pivot row of step j in rowbuf[j & 1]
+  __shared__ double pub[2][kQRRows];                  // v_j of each row in pub[j & 1]
+  __shared__ double Rinv[ASI_MAX_RANK];               // 1 / R[j][j]
   __shared__ double s_trace;
   const int tid = threadIdx.x;
   const int r = M.r;
-  for (int idx = tid; idx < r * r; idx += 256) {
-    const int i = idx / r, j = idx % r;
-    double g = 0.0;
-    if (j >= i)
-      for (int cc = 0; cc < M.nchunk; ++cc) g += M.Gp[((int64_t)cc * r + i) * r + j];
-    G[i][j] = g;
+  const int ti = tid >> 4, tj = tid & 15;             // slot (x, y) of a thread is G[ti + 16x][tj + 16y]
+
+  // The rows of P this CTA solves: four threads per row, thread ql holds columns ql, ql + 4, ...
+  const int rowl = tid >> 2, ql = tid & 3;
+  const int row = row0 + rowl;
+  const bool live = row < M.a;                        // rows past the end are solved as zeros, unstored
+  double v[ASI_MAX_RANK / 4];
+  {
+    const double* prow = M.Pred + (int64_t)(live ? row : 0) * r;
+#pragma unroll
+    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+      const int k = ql + 4 * t;
+      v[t] = __ldcg(prow + (k < r ? k : 0));         // unconditional, selected afterwards
+    }
+#pragma unroll
+    for (int t = 0; t < ASI_MAX_RANK / 4; ++t)
+      if (!(live && ql + 4 * t < r)) v[t] = 0.0;
   }
+  // G = sum of the row chunks' shares, chunk by chunk in order (upper triangle).
+  double g[4][4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) g[x][y] = 0.0;
+  const int nsum = args.gsum ? 1 : M.nchunk;          // share 0 already holds the total
+  for (int cc = 0; cc < nsum; cc += 2) {              // two chunks' loads in flight, added in order
+    const double* Gc = M.Gp + (int64_t)cc * r * r;
+    const bool two = cc + 1 < nsum;
+    double t0[4][4], t1[4][4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        const int i = ti + 16 * x, k = tj + 16 * y;
+        const bool on = k < r && k >= i;
+        const int o = on ? i * r + k : 0;
+        t0[x][y] = __ldcg(Gc + o);                   // unconditional loads, selected afterwards
+        t1[x][y] = __ldcg(Gc + (two ? r * r : 0) + o);
+      }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        const int i = ti + 16 * x, k = tj + 16 * y;
+        const bool on = k < r && k >= i;
+        g[x][y] = (g[x][y] + (on ? t0[x][y] : 0.0)) + ((on && two) ? t1[x][y] : 0.0);
+      }
+  }
+  // Diagonal -> trace; row 0 -> the first pivot row.
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+    if (ti == tj && ti + 16 * x < r) Rinv[ti + 16 * x] = g[x][x];
+  if (ti == 0) {
+#pragma unroll
+    for (int y = 0; y < 4; ++y)
+      if (tj + 16 * y < r) rowbuf[0][tj + 16 * y] = g[0][y];
+  }
+  if (ql == 0) pub[0][rowl] = v[0];
   __syncthreads();
   if (tid == 0) {
     double t = 0.0;
-    for (int i = 0; i < r; ++i) t += G[i][i];
+    for (int i = 0; i < r; ++i) t += Rinv[i];
     s_trace = t;
   }
   __syncthreads();
   const double floor_d = 1e-12 * s_trace;
+  // Right-looking Cholesky, one barrier per column.  Step j reads the pivot row (row j of the
+  // Schur complement), updates the rows below it in registers, hands row j + 1 to the next step
+  // and leaves R[j][k] = G[j][k] / R[j][j] in Rt.
   for (int j = 0; j < r; ++j) {
-    double d = G[j][j];
+    const double* rb = rowbuf[j & 1];
+    double* nb = rowbuf[(j + 1) & 1];
+    double d = rb[j];
     if (!(d > floor_d)) {
       if (tid == 0 && c == 0) atomicMax(args.status, (int)ASI_ERR_RANK_DEFICIENT);
       d = (floor_d > 0.0) ? floor_d : 1.0;
     }
-    const double rjj = sqrt(d);
-    __syncthreads();
-    for (int k = j + 1 + tid; k < r; k += 256) G[j][k] /= rjj;
-    if (tid == 0) G[j][j] = rjj;
-    __syncthreads();
-    const int n = r - j - 1;
-    for (int idx = tid; idx < n * n; idx += 256) {
-      const int i = j + 1 + idx / n, k = j + 1 + idx % n;
-      if (k >= i) G[i][k] -= G[j][i] * G[j][k];
+    const double inv = rsqrt(d);
+    double ai[4], bk[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int i = ti + 16 * t, k = tj + 16 * t;
+      ai[t] = (i > j && i < r) ? rb[i] * inv : 0.0;
+      bk[t] = (k > j && k < r) ? rb[k] * inv : 0.0;
     }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        const int i = ti + 16 * x, k = tj + 16 * y;
+        g[x][y] = fma(-ai[x], bk[y], g[x][y]);       // ai, bk are 0 outside the trailing block
+        if (i == j + 1 && k >= i && k < r) nb[k] = g[x][y];
+      }
+    if (tid > j && tid < r) Rt[tid * kQRPitch + j] = rb[tid] * inv;
+    if (tid == 0) Rinv[j] = inv;
     __syncthreads();
   }
-  if (tid < kQRRows) {
-    const int row = c * kQRRows + tid;
-    if (row < M.a) {
-      double q[ASI_MAX_RANK];
-      const double* prow = M.Pred + (int64_t)row * r;
-      for (int j = 0; j < r; ++j) {
-        double v = prow[j];
-        for (int i = 0; i < j; ++i) v -= q[i] * G[i][j];
-        v /= G[j][j];
-        q[j] = v;
-        M.Uout[(int64_t)row * r + j] = (float)v;
-      }
+  // U = P R^{-1}, row by row: q_j = v_j / R[j][j], then v_k -= q_j R[j][k] for k > j.  The four
+  // threads of a row sit in one warp; every lane takes every step (the warp barriers are
+  // unconditional), and the thread that owns column j + 1 hands v_{j+1} to the next step.
+  for (int j = 0; j < r; ++j) {
+    double rt[ASI_MAX_RANK / 4];
+#pragma unroll
+    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+      const int k = ql + 4 * t;
+      rt[t] = (k > j && k < r) ? Rt[k * kQRPitch + j] : 0.0;
+    }
+    const double q = pub[j & 1][rowl] * Rinv[j];
+    double* np = pub[(j + 1) & 1];
+#pragma unroll
+    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+      const int k = ql + 4 * t;
+      v[t] = (k == j) ? q : fma(-q, rt[t], v[t]);     // rt = 0 leaves the solved and the unused columns alone
+      if (k == j + 1 && k < r) np[rowl] = v[t];
+    }
+    __syncwarp();
+  }
+  if (live) {
+    float* urow = M.Uout + (int64_t)row * r;
+#pragma unroll
+    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+      const int k = ql + 4 * t;
+      if (k < r) urow[k] = (float)v[t];
     }
   }
 }
@@ -925,7 +1083,12 @@ cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) 
   k_qr_gram<<<grid, 256, 0, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k_qr_solve<<<grid, 256, 0, st>>>(p);
+  k_qr_gsum<<<dim3(ASI_MAX_RANK * ASI_MAX_RANK / 256, (unsigned)nd), 256, 0, st>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  QRArgs q = p;
+  q.gsum = 1;
+  k_qr_solve<<<grid, 256, 0, st>>>(q);
   return cudaGetLastError();
 }
 

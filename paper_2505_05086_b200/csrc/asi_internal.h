@@ -78,6 +78,7 @@ struct QRMode {
 struct QRArgs {
   QRMode m[ASI_MAX_MODES];
   int* status;
+  int gsum;            // set by launch_qr: share 0 of Gp holds the whole of G (else k_qr_solve sums the shares)
 };
 
 // Z4[c', j, kh, kw] = sum_{i,h',w'} Z1[i,c',h',w'] Z3pad[i,j,h's+kh-p,w's+kw-p], then
