@@ -45,16 +45,27 @@ template <int KC, int TQ, int NT, typename TX>
 __device__ __forceinline__ void load_x_tile(float (*Xs)[TQ + 1], const TX* __restrict__ X, int64_t a,
                                             int64_t I, int64_t k0, int64_t q0, int64_t q_end) {
   const int tid = threadIdx.x;
+  // All the loads of a thread are issued first, from clamped addresses where the tile hangs over
+  // the edge, and selected when they are stored: a load under a condition, or next to the store of
+  // the one before, waits for its predecessor, and a chunk then costs KC * TQ / NT round trips.
+  static_assert((KC * TQ) % NT == 0 && NT % TQ == 0, "threads must tile the chunk");
+  constexpr int PER = KC * TQ / NT;
+  float v[PER];
   if (I == 1 && a >= 32) {
-    for (int idx = tid; idx < KC * TQ; idx += NT) {
+#pragma unroll
+    for (int t = 0; t < PER; ++t) {
+      const int idx = tid + t * NT;
+      const int64_t k = k0 + idx % KC, q = q0 + idx / KC;
+      const bool on = k < a && q < q_end;
+      v[t] = ld_as_float(X + (on ? q * a + k : 0));
+    }
+#pragma unroll
+    for (int t = 0; t < PER; ++t) {
+      const int idx = tid + t * NT;
       const int kl = idx % KC, ql = idx / KC;
-      const int64_t k = k0 + kl, q = q0 + ql;
-      float v = 0.f;
-      if (k < a && q < q_end) v = ld_as_float(X + q * a + k);
-      Xs[kl][ql] = v;
+      Xs[kl][ql] = (k0 + kl < a && q0 + ql < q_end) ? v[t] : 0.f;
     }
   } else {
-    static_assert(NT % TQ == 0, "threads must tile the columns");
     const int ql = tid % TQ;
     const int64_t q = q0 + ql;
     const bool qok = q < q_end;
@@ -63,11 +74,15 @@ __device__ __forceinline__ void load_x_tile(float (*Xs)[TQ + 1], const TX* __res
       const int64_t o = q / I, i = q - o * I;
       base = o * a * I + i;
     }
-    for (int kl = tid / TQ; kl < KC; kl += NT / TQ) {
-      const int64_t k = k0 + kl;
-      float v = 0.f;
-      if (qok && k < a) v = ld_as_float(X + base + k * I);
-      Xs[kl][ql] = v;
+#pragma unroll
+    for (int t = 0; t < PER; ++t) {
+      const int64_t k = k0 + tid / TQ + t * (NT / TQ);
+      v[t] = ld_as_float(X + ((qok && k < a) ? base + k * I : 0));
+    }
+#pragma unroll
+    for (int t = 0; t < PER; ++t) {
+      const int kl = tid / TQ + t * (NT / TQ);
+      Xs[kl][ql] = (qok && k0 + kl < a) ? v[t] : 0.f;
     }
   }
 }
