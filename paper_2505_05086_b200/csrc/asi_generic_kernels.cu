@@ -106,11 +106,24 @@ __global__ void __launch_bounds__(128) k_modeprod(ModeProdArgs p) {
 
   for (int64_t k0 = 0; k0 < p.a; k0 += KC) {
     load_x_tile<KC, TQ, NT, TX>(Xs, X, p.a, p.I, k0, q0, p.Q);
-    for (int idx = tid; idx < KC * R; idx += NT) {
-      const int kl = idx / R, j = idx % R;
-      const int64_t k = k0 + kl;
-      const int jj = j0 + j;
-      Bs[kl][j] = (k < p.a && jj < p.n_out) ? p.B[k * p.ldb_k + jj * p.ldb_j] : 0.f;
+    {
+      // the factor's chunk, its loads issued together like the tile's
+      static_assert((KC * R) % NT == 0, "threads must tile the factor chunk");
+      constexpr int PB = KC * R / NT;
+      float b[PB];
+#pragma unroll
+      for (int t = 0; t < PB; ++t) {
+        const int idx = tid + t * NT;
+        const int64_t k = k0 + idx / R;
+        const int jj = j0 + idx % R;
+        b[t] = p.B[(k < p.a && jj < p.n_out) ? k * p.ldb_k + jj * p.ldb_j : 0];
+      }
+#pragma unroll
+      for (int t = 0; t < PB; ++t) {
+        const int idx = tid + t * NT;
+        const int kl = idx / R, j = idx % R;
+        Bs[kl][j] = (k0 + kl < p.a && j0 + j < p.n_out) ? b[t] : 0.f;
+      }
     }
     __syncthreads();
     const int kmax = (int)((p.a - k0 < KC) ? (p.a - k0) : KC);
