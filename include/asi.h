@@ -73,6 +73,11 @@ typedef struct {
 /* Use only the shape-generic kernels even where a fused kernel covers the layer
  * (same results up to fp32 rounding; for testing and comparison). */
 #define ASI_FLAG_GENERIC_ONLY 1
+/* Test hook for the bounded device waits: on the fused small-map path the producer of the bulk copy arms
+ * its barrier but issues no copy, and the wait limit drops from one second to one millisecond, so the
+ * waiting CTAs run into the limit, record ASI_ERR_TIMEOUT in the status word and return.  The outputs
+ * of such a call are undefined; nothing faults and the workspace can be used again afterwards. */
+#define ASI_FLAG_TEST_EXPIRE_WAIT 2
 
 /* Sizes and the paper's closed forms for one plan. */
 typedef struct {
@@ -137,7 +142,8 @@ asi_status_t asi_init_factors(const asi_plan_t* plan, const void* act, const flo
  *   - A plan whose compress_ws_bytes exceeds ASI_STATIC_WS_MAX_BYTES is refused with
  *     ASI_ERR_WORKSPACE and nothing is enqueued (asi_last_cuda_error() then holds the two sizes).
  *   - The first call on each device looks up the array's device address (one runtime query, with
- *     that device current).  Make that first call before any stream capture begins.
+ *     that device current).  Make that first call before any stream capture begins.  The address is
+ *     remembered per device: after cudaDeviceReset it is stale, so do not reset a device between calls.
  *   - All calls on one device share the one array, and it keeps whatever the previous call left in
  *     it.  The words that must start at zero (status word, completion counters) are cleared by the
  *     call itself.  Two calls whose GPU work overlaps -- different streams, or several host threads
@@ -175,6 +181,11 @@ size_t asi_step_host_arena_bytes(const asi_plan_t* plan);
 asi_status_t asi_step_host(const asi_plan_t* plan, const void* act_host, const void* dY_host,
                            const float* U_prev_host, float* U_new_host, float* core_host,
                            float* dW_host, void* arena, size_t arena_bytes, void* stream);
+
+/* The device status of the last asi_step_host call on `arena` (its workspace sits inside the arena at
+ * an offset only the library knows).  Synchronises `stream`. */
+asi_status_t asi_step_host_status(const asi_plan_t* plan, const void* arena, void* stream,
+                                  asi_status_t* device_status);
 
 /* Reads the device status word of a workspace after synchronising `stream`.
  * *device_status is ASI_OK, ASI_ERR_RANK_DEFICIENT or ASI_ERR_TIMEOUT. */

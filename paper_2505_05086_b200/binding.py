@@ -26,11 +26,12 @@ ASI_F32, ASI_BF16 = 0, 1
 ASI_CONV2D, ASI_LINEAR = 0, 1
 ASI_MAX_MODES = 4
 ASI_STATIC_WS_MAX_BYTES = 4 << 20
+ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT = 1, 2
 
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
     "asi_init_factors",
-    "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host",
+    "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host", "asi_step_host_status",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
     "asi_profile_end", "asi_last_cuda_error",
 )
@@ -85,6 +86,7 @@ def lib():
     L.asi_step_host_arena_bytes.restype = sz
     L.asi_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_poll_status.argtypes = [vp, vp, vp, C.POINTER(i32)]
+    L.asi_step_host_status.argtypes = [vp, vp, vp, C.POINTER(i32)]
     L.asi_launch_count.argtypes = [vp, i32]
     L.asi_launch_count.restype = i32
     L.asi_profile_begin.argtypes = [i32, C.POINTER(vp), i32]
@@ -97,7 +99,7 @@ def lib():
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
                  "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
-                 "asi_poll_status"):
+                 "asi_poll_status", "asi_step_host_status"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -113,7 +115,7 @@ def _check(code, where):
 
 
 def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False, dilation=1,
-              generic_only=False):
+              generic_only=False, flags=0):
     d = LayerDesc()
     d.kind = ASI_CONV2D if kind == "conv" else ASI_LINEAR
     d.in_dtype = ASI_BF16 if bf16 else ASI_F32
@@ -129,7 +131,7 @@ def make_desc(kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=Fals
     d.kh, d.kw, d.stride_h, d.stride_w, d.pad_h, d.pad_w = kh, kw, sh, sw, ph, pw
     d.dil_h = d.dil_w = int(dilation)
     d.groups = int(groups)
-    d.flags = 1 if generic_only else 0
+    d.flags = (1 if generic_only else 0) | int(flags)
     return d
 
 
@@ -138,10 +140,10 @@ class Plan:
     integers (device or host addresses), ``stream`` is a CUDA stream handle (0 = default)."""
 
     def __init__(self, kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False,
-                 dilation=1, generic_only=False):
+                 dilation=1, generic_only=False, flags=0):
         self._h = C.c_void_p()
         self.desc = make_desc(kind, dims, ranks, cout, k, stride, pad, groups, bf16, dilation,
-                              generic_only)
+                              generic_only, flags)
         _check(lib().asi_plan_create(C.byref(self.desc), C.byref(self._h)), "asi_plan_create")
         self.kind = kind
         self.info = PlanInfo()
@@ -197,6 +199,11 @@ class Plan:
     def step_host(self, act_h, dY_h, U_prev_h, U_new_h, core_h, dW_h, arena, arena_bytes, stream=0):
         _check(lib().asi_step_host(self._h, act_h, dY_h, U_prev_h, U_new_h, core_h, dW_h, arena,
                                    arena_bytes, stream), "asi_step_host")
+
+    def step_host_status(self, arena, stream=0):
+        out = C.c_int32(0)
+        _check(lib().asi_step_host_status(self._h, arena, stream, C.byref(out)), "asi_step_host_status")
+        return out.value
 
     def poll_status(self, ws, stream=0):
         out = C.c_int32(0)

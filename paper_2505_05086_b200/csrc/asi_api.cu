@@ -121,8 +121,10 @@ void layout_compress(asi_plan* pl) {
     int64_t qps = (v.Q + ns - 1) / ns;
     qps = (qps + 63) / 64 * 64;
     ns = (v.Q + qps - 1) / qps;
-    if (pl->fast_compress)                                               // one partial per tile
-      ns = (m == 1) ? sm_pass1_role_c_ctas(pl->fast_S, (int)pl->dims[0]) : pl->n_tiles_b;
+    if (pl->fast_compress) {                                             // one partial per tile; the cold-start
+      ns = (m == 1) ? sm_pass1_role_c_ctas(pl->fast_S, (int)pl->dims[0]) : pl->n_tiles_b;   // expansion splits the
+      qps = ((v.Q + ns - 1) / ns + 63) / 64 * 64;                        // columns over the same count
+    }
     if (pl->fiber[m] || (pl->plane && m >= 2)) {                         // one partial per CTA of k_fiber /
       ns = pl->fiber[m] ? pl->fiber_grid[m] : pl->plane_grid;            // k_plane; the cold-start expansion
       qps = ((v.Q + ns - 1) / ns + 63) / 64 * 64;                        // uses the same count (empty splits
@@ -380,6 +382,7 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     a.Y = dst;
     a.tc_scratch = w + pl->off_tc;
     a.tc_scratch_bytes = pl->tc_bytes;
+    a.status = reinterpret_cast<int*>(w);
     ASI_CUDA(launch_modeprod(a, src_bf16, st));
     cd[m] = pl->r[m];
     src = dst;
@@ -404,6 +407,7 @@ asi_status_t expand_mode(const asi_plan* pl, int m, const void* act, const float
   e.q_per_split = pl->q_per_split[m];
   e.tc_scratch = w + pl->off_tc;
   e.tc_scratch_bytes = pl->tc_bytes;
+  e.status = reinterpret_cast<int*>(w);
   ASI_CUDA(launch_expand(e, pl->bf16, st));
   return ASI_OK;
 }
@@ -529,7 +533,19 @@ asi_status_t asi_plan_query(const asi_plan_t* pl, asi_plan_info_t* info) {
                        r1 * r2 * Co * HoWo * D2 + r2 * Co * C * D2;
     info->macs_C_vanilla = D2 * C * Co * B * HoWo;
   } else {
-    info->macs_C_ASI = 0.0;
+    // linear layers (Sec. 3.1 footnote): Z = dY x_1 U_1^T (x_2 U_2^T), Z4 = Z . core over the leading ranks,
+    // dW = Z4 U_last^T -- one term per contraction, like the five terms of the conv cost
+    const int nd = pl->nd;
+    const double Do = pl->d.cout, Din = pl->dims[nd - 1], rl = pl->r[nd - 1];
+    double macs = 0.0, lead = 1.0, rest = Do;
+    for (int m = 1; m < nd - 1; ++m) rest *= (double)pl->dims[m];
+    for (int m = 0; m < nd - 1; ++m) {
+      macs += lead * pl->r[m] * (double)pl->dims[m] * rest;      // contract mode m of the running tensor
+      lead *= pl->r[m];
+      if (m + 1 < nd - 1) rest /= (double)pl->dims[m + 1];
+    }
+    macs += lead * rl * Do + rl * Do * Din;
+    info->macs_C_ASI = macs;
     info->macs_C_vanilla = (double)pl->N * pl->d.cout;
   }
   return ASI_OK;
@@ -564,6 +580,8 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     a.B = (int)pl->dims[0];
     a.C = (int)pl->dims[1];
     a.n_tiles_b = pl->n_tiles_b;
+    a.stall_copy = (pl->d.flags & ASI_FLAG_TEST_EXPIRE_WAIT) ? 1 : 0;
+    a.wait_ns = a.stall_copy ? 1000000ull : 1000000000ull;      // 1 ms under the test hook, else 1 s
     ASI_CUDA(launch_sm_pass1(a, pl->fast_S, pl->fast_R, pl->bf16, st));
     return finish_compress(pl, act, U_new, core, w, U_prev, st);
   }
@@ -616,6 +634,7 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     a.si = v.r;
     a.tc_scratch = w + pl->off_tc;
     a.tc_scratch_bytes = pl->tc_bytes;
+    a.status = reinterpret_cast<int*>(w);
     ASI_CUDA(launch_modeprod(a, pl->bf16, st));
     // P = A_m V
     s = expand_mode(pl, m, act, V, w, st);
@@ -851,6 +870,20 @@ asi_status_t asi_step_host(const asi_plan_t* pl, const void* act_host, const voi
   return ASI_OK;
 }
 
+asi_status_t asi_step_host_status(const asi_plan_t* pl, const void* arena, void* stream,
+                                  asi_status_t* device_status) {
+  if (!pl || !arena || !device_status) return ASI_ERR_INVALID_ARG;
+  const size_t eb = elem_bytes(pl);
+  size_t off = 0;                                   // the same carve-up as asi_step_host
+  off = align_up(off + (size_t)pl->N * eb, 256);
+  off = align_up(off + (size_t)pl->dy_elems * eb, 256);
+  off = align_up(off + (size_t)pl->u_elems * 4, 256);
+  off = align_up(off + (size_t)pl->u_elems * 4, 256);
+  off = align_up(off + (size_t)pl->core_elems * 4, 256);
+  off = align_up(off + (size_t)pl->dw_elems * 4, 256);
+  return asi_poll_status(pl, static_cast<const char*>(arena) + off, stream, device_status);
+}
+
 asi_status_t asi_profile_begin(int32_t kernel_id, void** events, int32_t n_pairs) {
   if (kernel_id < 1 || !events || n_pairs < 1) return ASI_ERR_INVALID_ARG;
   g_prof.ev = reinterpret_cast<cudaEvent_t*>(events);
@@ -875,7 +908,6 @@ asi_status_t asi_poll_status(const asi_plan_t* pl, const void* ws, void* stream,
   int v = 0;
   ASI_CUDA(cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, st));
   ASI_CUDA(cudaStreamSynchronize(st));
-  if (v == 0 && pl->bf16 && tc_error_flag()) v = (int)ASI_ERR_TIMEOUT;   // a wait of the tensor-core kernel expired
   *device_status = static_cast<asi_status_t>(v);
   return ASI_OK;
 }

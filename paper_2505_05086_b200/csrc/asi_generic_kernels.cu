@@ -10,14 +10,30 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
-
+#include <map>
+#include <mutex>
 #include <type_traits>
+#include <utility>
 
 #include "asi_internal.h"
 
 namespace asi {
 
 ProfState g_prof = {0, nullptr, 0, 0, 0.0};
+
+cudaError_t opt_in_smem(const void* kernel, size_t need) {
+  static std::mutex lock;
+  static std::map<std::pair<int, const void*>, size_t> granted;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> guard(lock);
+  size_t& have = granted[std::make_pair(dev, kernel)];
+  if (need <= have) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+  if (e == cudaSuccess) have = need;
+  return e;
+}
 
 __device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
@@ -795,13 +811,9 @@ size_t plane_smem(int S) {
 
 template <int R, typename TX>
 static cudaError_t launch_plane_t(const PlaneArgs& p, int grid, cudaStream_t st) {
-  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
-  const size_t smem = plane_smem(p.S);
-  if (smem > granted) {
-    cudaError_t e = cudaFuncSetAttribute(k_plane<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    granted = smem;
-  }
+  const size_t smem = plane_smem(p.S);   // the default limit counts static shared memory too: always opt in
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_plane<R, TX>), smem);
+  if (e != cudaSuccess) return e;
   k_plane<R, TX><<<grid, 256, smem, st>>>(p);
   return cudaGetLastError();
 }
@@ -827,13 +839,9 @@ int64_t fiber_tiles(int64_t O, int64_t a, int64_t I) {
 
 template <int R, typename TX>
 static cudaError_t launch_fiber_t(const FiberArgs& p, int grid, cudaStream_t st) {
-  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = fiber_smem((int)p.a);
-  if (smem > granted) {
-    cudaError_t e = cudaFuncSetAttribute(k_fiber<R, TX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    granted = smem;
-  }
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_fiber<R, TX>), smem);
+  if (e != cudaSuccess) return e;
   k_fiber<R, TX><<<grid, 256, smem, st>>>(p);
   return cudaGetLastError();
 }
@@ -1271,20 +1279,38 @@ cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, c
                         (double)p.C * p.r2 + (double)p.Cout * (p.C / p.groups) * p.kh * p.kw));
   const int n_out = p.r2 * p.kh * p.kw;
   const int G = (n_out <= 256) ? 256 / n_out : 1;
-  k_conv_z4<<<dim3(p.Cout, nsp), 256, (size_t)G * n_out * sizeof(float), st>>>(p, Z4p, nsp);
-  cudaError_t e = cudaGetLastError();
+  const size_t smem = (size_t)G * n_out * sizeof(float);
+  cudaError_t e = cudaSuccess;
+  if (smem > 40 * 1024) {
+    e = opt_in_smem(reinterpret_cast<const void*>(k_conv_z4), smem);
+    if (e == cudaSuccess) e = opt_in_smem(reinterpret_cast<const void*>(k_conv_dw), smem);
+    if (e != cudaSuccess) return e;
+  }
+  k_conv_z4<<<dim3(p.Cout, nsp), 256, smem, st>>>(p, Z4p, nsp);
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_conv_dw<<<p.Cout, 256, (size_t)n_out * sizeof(float), st>>>(p, Z4p, nsp);
   return cudaGetLastError();
+}
+
+size_t conv_tail_smem(int r2, int kh, int kw) {
+  const int n_out = r2 * kh * kw;
+  const int nsplit_max = (n_out <= 128) ? 256 / n_out : 1;
+  const int G = (n_out <= 256) ? 256 / n_out : 1;            // k_conv_z4
+  const size_t tail = (size_t)(((n_out + 31) / 32) * 32 + (size_t)nsplit_max * n_out) * sizeof(float);
+  const size_t z4 = (size_t)G * n_out * sizeof(float);
+  return tail > z4 ? tail : z4;
 }
 
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st) {
   ProfScope prof(ASI_K_CONV_TAIL, st,
                  4.0 * ((double)p.r1 * p.Cout * p.Ho * p.Wo + (double)p.r1 * p.r2 * p.H * p.W +
                         (double)p.C * p.r2 + (double)p.Cout * (p.C / p.groups) * p.kh * p.kw));
-  const int n_out = p.r2 * p.kh * p.kw;
-  const int nsplit_max = (n_out <= 128) ? 256 / n_out : 1;
-  const size_t smem = (size_t)(((n_out + 31) / 32) * 32 + (size_t)nsplit_max * n_out) * sizeof(float);
+  const size_t smem = conv_tail_smem(p.r2, p.kh, p.kw);
+  if (smem > 40 * 1024) {
+    cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_conv_tail), smem);
+    if (e != cudaSuccess) return e;
+  }
   k_conv_tail<<<p.Cout, 256, smem, st>>>(p);
   return cudaGetLastError();
 }

@@ -34,6 +34,7 @@ struct ModeProdArgs {
   int64_t so, sj, si;      // Y(o, j, i) = Y[o*so + j*sj + i*si]
   void* tc_scratch = nullptr;      // device scratch for the tensor-core kernel's bf16 operand (optional)
   size_t tc_scratch_bytes = 0;
+  int* status = nullptr;           // status word of the caller's workspace (a tensor-core wait that expires lands there)
 };
 
 // Pp[s](k, j) = sum_{q in split s} X(k, q) * V[q*r + j]
@@ -46,6 +47,7 @@ struct ExpandArgs {
   int64_t q_per_split;
   void* tc_scratch = nullptr;      // device scratch for the tensor-core kernel's bf16 operand (optional)
   size_t tc_scratch_bytes = 0;
+  int* status = nullptr;           // status word of the caller's workspace
 };
 
 // One mode's P = A_m (A_m^T U) in a single pass (k_fiber); Pp: [grid][a][r] partials.
@@ -101,6 +103,8 @@ struct SmPass1Args {
   int64_t u_off[ASI_MAX_MODES];
   int r[ASI_MAX_MODES];
   int B, C, n_tiles_b;
+  unsigned long long wait_ns;   // limit of the bounded wait on the bulk-copy barrier
+  int stall_copy;               // test hook: the producer arms the barrier but issues no copy (the wait must expire)
 };
 // Fixed-order fp64 reduction of the per-tile partials of every P_m, plus per-chunk shares of
 // G_m = P_m^T P_m.
@@ -162,7 +166,6 @@ cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaS
 cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st);
 size_t tc_scratch_bytes(int64_t K, int N);
 cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st);
-int tc_error_flag();   // != 0: a bounded wait of the tensor-core kernel expired
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
 cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t st);
@@ -193,12 +196,17 @@ struct ProfScope {
   }
 };
 
+// Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to a (device, kernel) pair,
+// so the sizes already granted are remembered per device.
+cudaError_t opt_in_smem(const void* kernel, size_t need);
+
 cudaError_t launch_modeprod(const ModeProdArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_expand(const ExpandArgs& p, bool x_bf16, cudaStream_t st);
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_qr_solve(const QRArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_fiber(const FiberArgs& p, int grid, bool x_bf16, cudaStream_t st);
 size_t fiber_smem(int a);
+size_t conv_tail_smem(int r2, int kh, int kw);
 cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t st);
 size_t plane_smem(int S);
 int64_t fiber_tiles(int64_t O, int64_t a, int64_t I);

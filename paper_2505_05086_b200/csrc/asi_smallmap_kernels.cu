@@ -100,12 +100,12 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
 // Thread 0 waits for the staged tile with a time limit; every thread learns the outcome.  On expiry
 // the status word gets ASI_ERR_TIMEOUT and thread 0 gives the copies in flight one more bounded
 // wait before the CTA returns.
-__device__ __forceinline__ bool cta_wait_tile(uint64_t* bar, int* s_flag, int* status) {
+__device__ __forceinline__ bool cta_wait_tile(uint64_t* bar, int* s_flag, int* status, uint64_t limit_ns) {
   if (threadIdx.x == 0) {
-    bool ok = mbar_wait_bounded(bar, 0, 1000000000ull);
+    bool ok = mbar_wait_bounded(bar, 0, limit_ns);
     if (!ok) {
       atomicMax(status, (int)ASI_ERR_TIMEOUT);
-      mbar_wait_bounded(bar, 0, 1000000000ull);
+      mbar_wait_bounded(bar, 0, limit_ns);
     }
     *s_flag = ok ? 1 : 0;
   }
@@ -118,7 +118,7 @@ __device__ __forceinline__ bool cta_wait_tile(uint64_t* bar, int* s_flag, int* s
 }
 
 // Warp 0 stages one contiguous block in chunks of 16 KB.
-__device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char* src, uint32_t bytes) {
+__device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char* src, uint32_t bytes, bool stall) {
   constexpr uint32_t kChunk = 16384;
   const int lane = threadIdx.x & 31;
   if ((threadIdx.x >> 5) != 0) return;
@@ -127,7 +127,7 @@ __device__ __forceinline__ void stage_block(uint64_t* bar, char* dst, const char
     mbar_expect_tx(bar, bytes);
   }
   __syncwarp();
-  const int nchunk = (int)((bytes + kChunk - 1) / kChunk);
+  const int nchunk = stall ? 0 : (int)((bytes + kChunk - 1) / kChunk);
   for (int i = lane; i < nchunk; i += 32) {
     const uint32_t off = (uint32_t)i * kChunk;
     const uint32_t n = (bytes - off < kChunk) ? bytes - off : kChunk;
@@ -628,7 +628,8 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     float* Vp = (C >= (G - 1) * HWC) ? U2s : V2s + HWC * R;   // [G-1][HWC][R]: on top of U2s when it fits
     const TX* Xb = A + (int64_t)b * C * HW + hw0;
     if constexpr (kBulkC)
-      stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u);
+      stage_block(&s_bar, reinterpret_cast<char*>(Xs), reinterpret_cast<const char*>(Xb), (uint32_t)C * HW * 4u,
+                  p.stall_copy != 0);
     fac_issue_padded<R>(p.U_prev + p.u_off[1], U2s, C, p.r[1]);
     if constexpr (kBulkC) {
     } else if constexpr (NQ == 1) {
@@ -653,7 +654,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     }
     fac_wait();
     if constexpr (kBulkC) {
-      if (!cta_wait_tile(&s_bar, &s_flag, p.status)) return;
+      if (!cta_wait_tile(&s_bar, &s_flag, p.status, p.wait_ns)) return;
     } else {
       __syncthreads();
     }
@@ -1332,20 +1333,10 @@ size_t sm_wgrad_smem(const SmWgradArgs& p, int R) {
   return 4 * n + 64;
 }
 
-// Raises the kernel's dynamic shared memory limit to `need` bytes when it is below that.
-template <typename K>
-static cudaError_t opt_in_smem(K kernel, size_t* granted, size_t need) {
-  if (need <= *granted) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-  if (e == cudaSuccess) *granted = need;
-  return e;
-}
-
 template <int S, int R, typename TX>
 static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
-  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
-  const size_t smem = sm_pass1_smem(S, R, p.B, p.C);
-  cudaError_t e = opt_in_smem(k_sm_pass1<S, R, TX>, &granted, smem);
+  const size_t smem = sm_pass1_smem(S, R, p.B, p.C);   // the default limit counts static shared memory too: always opt in
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_pass1<S, R, TX>), smem);
   if (e != cudaSuccess) return e;
   k_sm_pass1<S, R, TX><<<p.n_tiles_b + sm_pass1_role_c_ctas(S, p.B), kNT, smem, st>>>(p);
   return cudaGetLastError();
@@ -1353,18 +1344,16 @@ static cudaError_t launch_pass1_t(const SmPass1Args& p, cudaStream_t st) {
 
 template <int S, int R, typename TX>
 static cudaError_t launch_core_t(const SmCoreArgs& p, cudaStream_t st) {
-  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = sm_core_smem(S, R, p.B);
-  cudaError_t e = opt_in_smem(k_sm_core<S, R, TX>, &granted, smem);
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_core<S, R, TX>), smem);
   if (e != cudaSuccess) return e;
   return launch_dependent(k_sm_core<S, R, TX>, dim3(p.n_tiles), dim3(kNT), smem, st, p);
 }
 
 template <int R, typename TX>
 static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
-  static size_t granted = 0;   // the default limit counts static shared memory too: always opt in
   const size_t smem = sm_wgrad_smem(p, R);
-  cudaError_t e = opt_in_smem(k_sm_wgrad<R, TX>, &granted, smem);
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_wgrad<R, TX>), smem);
   if (e != cudaSuccess) return e;
   k_sm_wgrad<R, TX><<<p.Cout / p.cpb, kNT, smem, st>>>(p);
   return cudaGetLastError();

@@ -18,7 +18,8 @@
 //     them to the mbarrier that frees the stage;
 //   * eight warps then read the three accumulator groups with tcgen05.ld (lane = row), add them and store
 //     fp32 rows.
-// Every wait has a time limit; on expiry the kernel raises g_tc_error, frees its TMEM and returns.
+// Every wait has a time limit; on expiry the kernel records ASI_ERR_TIMEOUT in the workspace's status word,
+// frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -40,8 +41,6 @@ constexpr int kTcStages = 4;       // X stages in flight
 constexpr int kTcNMax = 64;
 constexpr uint32_t kTileA = kTcM * kTcKC * 2;       // 16 KB
 constexpr uint32_t kTileB = 3 * kTcNMax * kTcKC * 2;   // 24 KB: the three terms stacked
-
-__device__ int g_tc_error = 0;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -136,6 +135,7 @@ struct TcArgs {
   int k_per_split;     // multiple of 64; CTA (., s) contracts [s * k_per_split, min(K, (s + 1) * k_per_split))
   int64_t y_split;
   int inner;           // kTcTokenExpand: K enumerates (o, i) with i < inner (a multiple of 64)
+  int* status;         // status word of the caller's workspace (may be null): ASI_ERR_TIMEOUT when a wait expires
 };
 
 // Bt[(t*n + j) * ldb + k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
@@ -290,8 +290,8 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUte
         }
       }
     }
-  } else if (tid == 0) {
-    atomicExch(&g_tc_error, 1);
+  } else if (tid == 0 && p.status) {
+    atomicMax(p.status, (int)ASI_ERR_TIMEOUT);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -349,10 +349,6 @@ bool encode_bf16_map(CUtensorMap* map, const void* base, int rank, const cuuint6
              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-template <typename K>
-cudaError_t tc_opt_in(K kernel) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem);
-}
 
 // V[o][i][j] = sum_k X[o][k][i] U[k][j]: a middle mode of a bf16 token tensor (I = inner extent, a multiple of 64)
 cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
@@ -376,13 +372,11 @@ cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch
     const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
     if (!encode_bf16_map(&mapB, scratch, 2, dims, strides, box)) return cudaErrorNotSupported;
   }
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] { attr_err = tc_opt_in(k_tc_token); });
+  const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_token), kTcSmem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((p.a + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
       p.B, (int)p.ldb_k, (int)p.a, N, static_cast<__nv_bfloat16*>(scratch), Kp);
-  TcArgs a = {p.Y, (int)p.I, N, (int)p.a, N, (int)Kp, p.so, 0};
+  TcArgs a = {p.Y, (int)p.I, N, (int)p.a, N, (int)Kp, p.so, 0, p.status};
   dim3 grid((unsigned)((p.I + kTcM - 1) / kTcM), (unsigned)p.O);
   k_tc_token<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -411,13 +405,11 @@ cudaError_t launch_tc_token_expand(const ExpandArgs& e, void* scratch, size_t sc
     const cuuint32_t box[2] = {(cuuint32_t)kTcKC, (cuuint32_t)(3 * N)};
     if (!encode_bf16_map(&mapB, scratch, 2, dims, strides, box)) return cudaErrorNotSupported;
   }
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] { attr_err = tc_opt_in(k_tc_token_expand); });
+  const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_token_expand), kTcSmem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
       e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
-  TcArgs a = {e.Pp, (int)e.a, N, (int)Q, N, (int)e.q_per_split, e.a * N, (int)e.I};
+  TcArgs a = {e.Pp, (int)e.a, N, (int)Q, N, (int)e.q_per_split, e.a * N, (int)e.I, e.status};
   dim3 grid((unsigned)((e.a + kTcM - 1) / kTcM), (unsigned)e.nsplit);
   k_tc_token_expand<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -459,16 +451,12 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorNotSupported;
   }
-  static const size_t smem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(k_tc_lastmode, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  });
+  const size_t smem = kTcSmem;
+  const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_lastmode), smem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
       p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch), K);
-  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0, 0};
+  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0, 0, p.status};
   const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
   k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -508,25 +496,15 @@ cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorNotSupported;
   }
-  static const size_t smem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(k_tc_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  });
+  const size_t smem = kTcSmem;
+  const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_expand), smem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
       e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
-  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N, 0};
+  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N, 0, e.status};
   dim3 grid((unsigned)((A + kTcM - 1) / kTcM), (unsigned)e.nsplit);
   k_tc_expand<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
-}
-
-int tc_error_flag() {
-  int v = 0;
-  cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int));
-  return v;
 }
 
 }  // namespace asi

@@ -6,6 +6,10 @@ from oracle import asi_oracle as O
 
 TOL_F32 = dict(proj=1e-4, core=1e-4, dw=5e-4)     # relative Frobenius error, fp32 inputs
 TOL_BF16 = dict(proj=2e-2, core=2e-2, dw=2e-2)    # bf16-input mode
+# Beside the norms: the largest element error of dW against the largest element of the reference.
+# Rounding errors are spread evenly, so this ratio sits near the Frobenius figure; a misplaced or
+# missing tap moves single elements by O(1) and fails it even where the norm would pass.
+DW_MAX_FACTOR = 4.0
 
 
 def make_runner(L, ranks=None, bf16=False, generic_only=False):
@@ -38,6 +42,7 @@ def compare_step(run, L, A, dY, U_prev):
         proj=max(O.rel_fro(O.projector(ug), O.projector(ur)) for ug, ur in zip(U_gpu, U_ref)),
         core=O.rel_fro(S_al, S_ref),
         dw=O.rel_fro(dW_gpu, dW_ref),
+        dw_max=float(np.max(np.abs(dW_gpu - dW_ref)) / max(np.max(np.abs(dW_ref)), 1e-300)),
         orth=max(np.linalg.norm(ug.astype(np.float64).T @ ug - np.eye(ug.shape[1])) for ug in U_gpu),
         sign=min(float(np.min(np.sum(ug * ur, axis=0))) for ug, ur in zip(U_gpu, U_ref)),
     )
@@ -48,5 +53,7 @@ def check(err, tol, what=""):
     assert err["proj"] <= tol["proj"], (what, err)
     assert err["core"] <= tol["core"], (what, err)
     assert err["dw"] <= tol["dw"], (what, err)
+    if "dw_max" in err:
+        assert err["dw_max"] <= DW_MAX_FACTOR * tol["dw"], (what, err)
     assert err["orth"] <= 1e-4, (what, err)
     assert err["sign"] > 0.0, (what, err)      # same Gram-Schmidt sign convention, no flips needed

@@ -58,6 +58,13 @@ def test_plan_query_matches_closed_forms(asi):
     p3 = asi.Plan("linear", (32, 197, 768), (8, 32, 64), cout=3072, bf16=True)
     assert p3.info.dw_elems == 3072 * 768 and p3.info.dy_elems == 32 * 197 * 3072
     assert p3.info.compressed_elems == O.compressed_elems((32, 197, 768), (8, 32, 64))
+    # cost of the linear backward, term by term: dY x_1 U_1^T, x_2 U_2^T, the contraction with the core
+    # over the leading ranks, and the expansion with U_3^T
+    B, N, Din, Dout, r1, r2, r3 = 32, 197, 768, 3072, 8, 32, 64
+    assert p3.info.macs_C_ASI == r1 * B * N * Dout + r1 * r2 * N * Dout + r1 * r2 * r3 * Dout + r3 * Dout * Din
+    assert p3.info.macs_C_vanilla == B * N * Din * Dout
+    p4 = asi.Plan("linear", (45, 33), (6, 9), cout=17)
+    assert p4.info.macs_C_ASI == 6 * 45 * 17 + 6 * 9 * 17 + 9 * 17 * 33
 
 
 @pytest.mark.parametrize("dims,ranks,on_tensor_cores", [

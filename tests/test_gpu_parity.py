@@ -203,6 +203,81 @@ def test_cold_start_with_explicit_gaussian_matrices():
     assert O.rel_fro(S_al, S_ref) < 1e-4
 
 
+def _cold_start_case(L, A, bf16, tol):
+    rng = np.random.default_rng(1)
+    n = int(np.prod(L.dims))
+    Omega = [rng.standard_normal((n // d, r)).astype(np.float32) for d, r in zip(L.dims, L.ranks)]
+    run = make_runner(L, bf16=bf16)
+    om = torch.from_numpy(np.concatenate([o.ravel() for o in Omega])).cuda()
+    run.init_factors(run.to_device(A), om)
+    assert run.ok()
+    S_ref, U_ref = O.asi_cold_start(A.astype(np.float64), [o.astype(np.float64) for o in Omega])
+    U_gpu = run.factors()
+    for ug, ur in zip(U_gpu, U_ref):
+        assert O.rel_fro(O.projector(ug), O.projector(ur)) < tol, L.dims
+    S_al, _ = O.sign_align(run.core_np(), U_gpu, U_ref)
+    assert O.rel_fro(S_al, S_ref) < tol, L.dims
+
+
+@pytest.mark.parametrize("dims,ranks", [((64, 512, 7, 7), (4, 4, 4, 4)), ((64, 256, 14, 14), (3, 3, 3, 4)),
+                                        ((8, 32, 16, 16), (4, 8, 8, 8))])
+def test_cold_start_on_fused_small_map_plans(dims, ranks):
+    """Branch t = 0 of Algorithm 1 on plans that take the fused kernels afterwards: the expansion
+    P_m = A_m Omega_m must cover every column of the unfolding whatever split count the plan uses."""
+    L = LayerSpec("t", "conv", dims, 8, 3, 1, 1, 1, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=17)
+    A, _ = st.next()
+    assert make_runner(L).plan.launch_count(0) == 3          # the fused plan
+    _cold_start_case(L, A, False, 1e-4)
+
+
+def test_cold_start_on_a_bf16_token_layer():
+    """Cold start through the tensor-core expansion kernels (bf16 tokens, last rank 32, token rank 16)."""
+    dims, ranks = (4, 72, 128), (3, 16, 32)
+    L = LayerSpec("t", "linear", dims, 24, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=29, rho=(0.6, 0.93, 0.96),
+                     gen_ranks=(4, 32, 64), bf16=True)
+    A, _ = st.next()
+    _cold_start_case(L, A, True, 1e-3)
+
+
+def test_ragged_case_at_the_benchmark_conditioning():
+    """Ranks 8 with the benchmark generator's decay 0.7 per index (condition number of the one-step map
+    about 150, what the single-conv configuration has), on sizes that leave ragged tiles."""
+    dims, ranks = (9, 21, 11, 13), (8, 8, 8, 8)
+    L = LayerSpec("t", "conv", dims, 10, 3, 1, 1, 1, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=41)      # rho = 0.7 in every mode
+    run = make_runner(L)
+    U_prev = st.u_prev0()
+    for t in range(2):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, TOL_F32, f"rho 0.7 rank 8 step {t}")
+
+
+def test_expired_device_wait_is_reported_and_the_workspace_recovers():
+    """The bounded waits of the kernels end in ASI_ERR_TIMEOUT instead of hanging.  With the test
+    flag the producer of the bulk copy issues nothing, so every waiting CTA runs into its (1 ms)
+    limit and returns; the next ordinary call on the same workspace is healthy again."""
+    from paper_2505_05086_b200.binding import ASI_ERR_TIMEOUT, ASI_FLAG_TEST_EXPIRE_WAIT, Plan
+    dims, ranks = (8, 12, 7, 7), (3, 4, 3, 2)
+    L = LayerSpec("t", "conv", dims, 10, 3, 1, 1, 1, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=7)
+    A, dY = st.next()
+    run = make_runner(L)
+    stalled = Plan("conv", dims, ranks, 10, 3, 1, 1, 1, flags=ASI_FLAG_TEST_EXPIRE_WAIT)
+    assert stalled.info.compress_ws_bytes == run.plan.info.compress_ws_bytes
+    run.set_factors(st.u_prev0())
+    act = run.to_device(A)
+    s = int(torch.cuda.current_stream().cuda_stream)
+    stalled.compress(act.data_ptr(), run.U[run.cur].data_ptr(), run.U[1 - run.cur].data_ptr(),
+                     run.core.data_ptr(), run.ws_c.data_ptr(), run.ws_c.numel(), s)
+    assert stalled.poll_status(run.ws_c.data_ptr(), s) == ASI_ERR_TIMEOUT
+    err, _ = compare_step(run, L, A, dY, st.u_prev0())       # same workspace, healthy plan
+    check(err, TOL_F32, "after an expired wait")
+    assert run.device_status() == 0
+
+
 def test_rank_deficient_iterate_is_reported_not_hidden():
     dims, ranks = (4, 6, 5, 5), (2, 3, 2, 2)
     L = LayerSpec("t", "conv", dims, 4, 3, 1, 1, 1, ranks=ranks)

@@ -60,6 +60,37 @@ def test_static_workspace_variant_matches_asi_compress(cfg_index, layer):
         U_prev = U_ref                            # warm start of the next call
 
 
+def test_shared_array_serves_plans_of_different_layouts_in_turn():
+    """A fused small-map plan and a generic-path plan alternate on the one built-in array: each call
+    finds the other plan's leftovers in a different layout and must still match asi_compress run on
+    a workspace of its own (the generic path clears the status word by a memset, the fused path in
+    its first kernel)."""
+    from paper_2505_05086_b200.binding import ASI_STATIC_WS_MAX_BYTES
+    cfg = get_config(0)
+    L = cfg.layers[0]
+    st = make_stream(cfg, 0)
+    runs = [make_runner(L), make_runner(L, generic_only=True)]
+    assert runs[0].plan.launch_count(0) == 3 and runs[1].plan.launch_count(0) > 3
+    dev = runs[0].device
+    U_prev = torch.from_numpy(_flat(st.u_prev0())).to(dev)
+    stream = int(torch.cuda.current_stream().cuda_stream)
+    for call in range(4):
+        run = runs[call % 2]
+        assert run.plan.info.compress_ws_bytes <= ASI_STATIC_WS_MAX_BYTES
+        A, _ = st.next()
+        act = run.to_device(A)
+        U_ref, U_new = torch.zeros_like(U_prev), torch.zeros_like(U_prev)
+        S_ref = torch.zeros(run.plan.info.core_elems, device=dev)
+        S_new = torch.zeros_like(S_ref)
+        run.plan.compress(act.data_ptr(), U_prev.data_ptr(), U_ref.data_ptr(), S_ref.data_ptr(),
+                          run.ws_c.data_ptr(), run.ws_c.numel(), stream)
+        run.plan.compress_static_ws(act.data_ptr(), U_prev.data_ptr(), U_new.data_ptr(), S_new.data_ptr(), stream)
+        torch.cuda.synchronize()
+        assert torch.equal(U_new, U_ref), call          # same kernels, same order of sums: the same bits
+        assert torch.equal(S_new, S_ref), call
+        U_prev = U_ref
+
+
 def test_static_workspace_variant_refuses_oversized_plans():
     from paper_2505_05086_b200.binding import ASI_ERR_WORKSPACE, ASI_STATIC_WS_MAX_BYTES, AsiError, Plan
     p = Plan("conv", (128, 64, 56, 56), (3, 3, 3, 3), cout=64, k=3, stride=1, pad=1)
