@@ -323,7 +323,7 @@ class Workload:
     """Device-resident inputs, runners and CUDA graphs of one configuration."""
 
     def __init__(self, ci, dev, use_graph, torch, n_host_sets=0):
-        from paper_2505_05086_b200.runner import LayerRunner
+        from paper_2505_05086_b200.runner import LayerRunner, StepRunner
         self.ci, self.cfg, self.torch = ci, get_config(ci), torch
         cfg = self.cfg
         self.nl = len(cfg.layers)
@@ -349,8 +349,13 @@ class Workload:
             self.dys.append(d_l)
             self.host.append(h_l)
         self.stream = torch.cuda.Stream(device=dev)
+        # the whole step through the batched entry points (one call forward, one call backward)
+        self.step = StepRunner(self.runners)
+        # for the graph every layer is a branch of its own (the layers of a step are independent of one another):
+        # measured faster than the batched launches on one branch, whose kernel stages run one after the other
         self.side = [torch.cuda.Stream(device=dev) for _ in range(self.nl)]
-        self.launches_per_step = sum(r.plan.launch_count(0) + r.plan.launch_count(1) for r in self.runners)
+        self.launches_per_step = (self._count_launches() if not use_graph else
+                                  sum(r.plan.launch_count(0) + r.plan.launch_count(1) for r in self.runners))
         with torch.cuda.stream(self.stream):
             for i in range(2):
                 self.step_direct(i)
@@ -373,14 +378,31 @@ class Workload:
                         cur.wait_stream(self.side[li])
                 self.graphs.append(g)
 
+    def _count_launches(self):
+        """Kernel launches of one step through the batched entry points: fused layers of one variant
+        (map size, rank bucket) share three compress launches and, per rank bucket, one wgrad launch."""
+        n, cvar, wvar = 0, {}, {}
+        for r in self.runners:
+            pl, d = r.plan, r.dims
+            if pl.launch_count(0) == 3:
+                key = (d[2], 4 if max(r.ranks) <= 4 else 8)
+                cvar[key] = cvar.get(key, 0) + 1
+            else:
+                n += pl.launch_count(0)
+            if pl.launch_count(1) == 1:
+                key = 4 if max(r.ranks) <= 4 else 8
+                wvar[key] = wvar.get(key, 0) + 1
+            else:
+                n += pl.launch_count(1)
+        n += sum(3 * -(-c // 8) for c in cvar.values()) + sum(-(-c // 8) for c in wvar.values())
+        return n
+
     def step_direct(self, i, only=None):
         s = i % self.sets
         if only != "wgrad":
-            for li in range(self.nl):
-                self.runners[li].compress(self.acts[li][s], self.stream)
+            self.step.compress([self.acts[li][s] for li in range(self.nl)], self.stream)
         if only != "compress":
-            for li in reversed(range(self.nl)):
-                self.runners[li].wgrad(self.dys[li][s], self.stream)
+            self.step.wgrad([self.dys[li][s] for li in range(self.nl)], self.stream)
 
     def run_step(self, i):
         if self.graphs is None:
@@ -618,8 +640,9 @@ def run_ours(args):
                    "ranks": [list(L.ranks) for L in cfg.layers], "in_dtype": "bf16" if cfg.bf16 else "f32",
                    "l2_policy": f"inputs larger than L2: {head['input_sets']} rotating input sets, "
                                 f"{head['input_bytes_rotated'] / 1e6:.0f} MB of act+dY",
-                   "launch": ("direct launches on one stream" if args.no_graph else
+                   "launch": ("asi_compress_batched + asi_wgrad_batched on one stream" if args.no_graph else
                               "CUDA-graph replay, one graph per input set, one branch per layer"),
+                   "single_stream_launch": "asi_compress_batched + asi_wgrad_batched, one call each per step",
                    "timing": f"{head['timed_blocks']} blocks of {args.steps} steps, {head['timed_ms_total']:.0f} ms "
                              f"of device time; ms_per_step = median block / steps",
                    "single_stream_direct_launch_value": head.get("single_stream_value"),

@@ -126,6 +126,21 @@ asi_status_t asi_compress(const asi_plan_t* plan, const void* act, const float* 
 asi_status_t asi_init_factors(const asi_plan_t* plan, const void* act, const float* omega,
                               float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
 
+/* The layers one training step handles together, in one call each way: Algorithm 1 is run for every
+ * fine-tuned layer at every step (Sec. 4 fine-tunes the last two to four layers), and the backward pass
+ * needs every layer's weight gradient.  Arrays of n entries, entry i as in asi_compress / asi_*_wgrad;
+ * every layer has its own workspace (distinct pointers).  Results are bit-identical to n separate
+ * calls.  Layers on the fused small-map path that share a kernel variant (map size, rank bucket, input
+ * type) share one launch per kernel stage -- a step of L such layers is 3 + 1 launches instead of
+ * 3L + L --, the others are enqueued one after another on `stream`.  Host-detectable errors are checked
+ * for all layers before anything is enqueued. */
+asi_status_t asi_compress_batched(const asi_plan_t* const* plans, const void* const* acts,
+                                  const float* const* U_prev, float* const* U_new, float* const* cores,
+                                  void* const* ws, const size_t* ws_bytes, int32_t n, void* stream);
+asi_status_t asi_wgrad_batched(const asi_plan_t* const* plans, const float* const* cores,
+                               const float* const* U, const void* const* dY, float* const* dW,
+                               void* const* ws, const size_t* ws_bytes, int32_t n, void* stream);
+
 /* asi_compress for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a deployment convenience, not part of the method.)
  *

@@ -30,7 +30,7 @@ ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT = 1, 2
 
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
-    "asi_init_factors",
+    "asi_init_factors", "asi_compress_batched", "asi_wgrad_batched",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host", "asi_step_host_status",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
     "asi_profile_end", "asi_last_cuda_error",
@@ -80,6 +80,9 @@ def lib():
     L.asi_compress.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_compress_static_ws.argtypes = [vp, vp, vp, vp, vp, vp]
     L.asi_init_factors.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    pvp, psz = C.POINTER(vp), C.POINTER(sz)
+    L.asi_compress_batched.argtypes = [pvp, pvp, pvp, pvp, pvp, pvp, psz, i32, vp]
+    L.asi_wgrad_batched.argtypes = [pvp, pvp, pvp, pvp, pvp, pvp, psz, i32, vp]
     L.asi_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_linear_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_step_host_arena_bytes.argtypes = [vp]
@@ -99,7 +102,7 @@ def lib():
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
                  "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
-                 "asi_poll_status", "asi_step_host_status"):
+                 "asi_poll_status", "asi_step_host_status", "asi_compress_batched", "asi_wgrad_batched"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -209,6 +212,30 @@ class Plan:
         out = C.c_int32(0)
         _check(lib().asi_poll_status(self._h, ws, stream, C.byref(out)), "asi_poll_status")
         return out.value
+
+
+class Batch:
+    """Argument arrays of asi_compress_batched / asi_wgrad_batched for a fixed list of plans.  The
+    arrays are built once (marshalling only) and can be re-used every step with new pointers."""
+
+    def __init__(self, plans):
+        self.plans = list(plans)
+        self.n = len(self.plans)
+        self._h = (C.c_void_p * self.n)(*[p.handle.value for p in self.plans])
+
+    def _arr(self, values):
+        return (C.c_void_p * self.n)(*[int(v) for v in values])
+
+    def compress(self, acts, U_prev, U_new, cores, ws, ws_bytes, stream=0):
+        sizes = (C.c_size_t * self.n)(*[int(v) for v in ws_bytes])
+        _check(lib().asi_compress_batched(self._h, self._arr(acts), self._arr(U_prev), self._arr(U_new),
+                                          self._arr(cores), self._arr(ws), sizes, self.n, stream),
+               "asi_compress_batched")
+
+    def wgrad(self, cores, U, dY, dW, ws, ws_bytes, stream=0):
+        sizes = (C.c_size_t * self.n)(*[int(v) for v in ws_bytes])
+        _check(lib().asi_wgrad_batched(self._h, self._arr(cores), self._arr(U), self._arr(dY), self._arr(dW),
+                                       self._arr(ws), sizes, self.n, stream), "asi_wgrad_batched")
 
 
 KERNEL_IDS = {"modeprod": 1, "expand": 2, "qr": 3, "conv_tail": 4, "sm_pass1": 5, "sm_core": 6,

@@ -4,6 +4,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "asi_internal.h"
 
@@ -107,6 +108,18 @@ void layout_compress(asi_plan* pl) {
         pl->fiber_grid[m] = (int)std::min<int64_t>(fiber_tiles(v.O, v.a, v.I), 296);
       }
     }
+  // register-tiled successors where the shape fits them (one partial per CTA, fewer and larger CTAs)
+  pl->plane2 = false;
+  for (int m = 0; m < ASI_MAX_MODES; ++m) pl->fiber2[m] = false;
+  if (pl->plane && plane2_supported((int)pl->dims[2], pl->dims[0] * pl->dims[1], pl->r[2], pl->r[3])) {
+    pl->plane2 = true;
+    pl->plane_grid = plane2_grid((int)pl->dims[2], pl->dims[0] * pl->dims[1], 296);
+  }
+  for (int m = 0; m < pl->nd; ++m)
+    if (pl->fiber[m] && fiber2_supported(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16)) {
+      pl->fiber2[m] = true;
+      pl->fiber_grid[m] = (int)std::min<int64_t>(fiber2_tiles(pl->mv[m].O, pl->mv[m].I), 296);
+    }
   int64_t vmax = 0;
   if (!pl->fast_compress)
     for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
@@ -195,10 +208,19 @@ void layout_compress(asi_plan* pl) {
     pl->off_T[t] = off;
     off = align_up(off + (size_t)tmax[t] * 4, 256);
   }
+  pl->core_tail = false;
+  pl->off_ctp = off;
+  if (pl->d.kind == ASI_CONV2D && !pl->fast_compress && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) &&
+      order[0] == 0 && order[1] == 1 && order[2] == 2 && order[3] == 3 &&
+      core_tail_supported(pl->r[1], pl->r[2], pl->r[3], (int)pl->dims[2], (int)pl->dims[3])) {
+    pl->core_tail = true;
+    off = align_up(off + 4 * core_tail_part_elems(pl->r[0], pl->r[1], pl->r[2], pl->r[3], (int)pl->dims[1],
+                                                  (int)pl->dims[2], (int)pl->dims[3]), 256);
+  }
   pl->compress_ws = off;
   pl->launches_compress = 3;
   if (!pl->fast_compress) {
-    pl->launches_compress = 2 + pl->nd + (pl->small_rank ? 0 : 1);         // reduction/QR kernels, core chain
+    pl->launches_compress = 2 + (pl->core_tail ? 2 : pl->nd) + (pl->small_rank ? 0 : 1);   // reduction/QR kernels, core chain
     for (int m = 0; m < pl->nd; ++m)
       pl->launches_compress += (pl->plane && m >= 2) ? (m == 2 ? 1 : 0) : pl->fiber[m] ? 1 : 2;
     // a tensor-core product is two launches (operand split + GEMM): V_m, the expansion when it fits too,
@@ -236,12 +258,15 @@ void layout_wgrad(asi_plan* pl) {
   }
   pl->conv_nsp = 1;
   pl->off_Z4p = off;
+  pl->conv_z3 = pl->d.kind == ASI_CONV2D && !pl->fast_wgrad && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) &&
+                pl->r[2] <= 8 && pl->r[3] <= 8;
+  if (pl->conv_z3) pl->launches_wgrad = 3;
   if (pl->d.kind == ASI_CONV2D && !pl->fast_wgrad && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) &&
       (int64_t)pl->r[0] * pl->Ho * pl->Wo >= 1024 && pl->d.cout < 296) {
     pl->conv_nsp = (int)std::min<int64_t>(16, std::max<int64_t>(2, 592 / pl->d.cout));
     pl->conv_nsp = (int)std::min<int64_t>(pl->conv_nsp, (int64_t)pl->r[0] * pl->Ho);
     off = align_up(off + (size_t)pl->conv_nsp * pl->d.cout * pl->r[1] * pl->d.kh * pl->d.kw * 4, 256);
-    pl->launches_wgrad = 5;
+    pl->launches_wgrad = pl->conv_z3 ? 4 : 5;
   }
   pl->wgrad_ws = off;
 }
@@ -263,6 +288,95 @@ thread_local char g_cuda_err[256] = "";
     }                                                                         \
   } while (0)
 
+// Argument blocks of the fused small-map kernels for one layer (shared by the single-layer and the
+// batched entry points).
+void build_fused_pass1(const asi_plan* pl, const void* act, const float* U_prev, char* w, SmPass1Args* a) {
+  a->act = act;
+  a->U_prev = U_prev;
+  for (int m = 0; m < 4; ++m) {
+    a->Pp[m] = reinterpret_cast<float*>(w + pl->off_Pp[m]);
+    a->u_off[m] = pl->u_off[m];
+    a->r[m] = pl->r[m];
+  }
+  a->status = reinterpret_cast<int*>(w);     // cleared by the kernel itself
+  a->B = (int)pl->dims[0];
+  a->C = (int)pl->dims[1];
+  a->n_tiles_b = pl->n_tiles_b;
+  a->stall_copy = (pl->d.flags & ASI_FLAG_TEST_EXPIRE_WAIT) ? 1 : 0;
+  a->wait_ns = a->stall_copy ? 1000000ull : 1000000000ull;      // 1 ms under the test hook, else 1 s
+}
+
+int build_fused_reduce(const asi_plan* pl, char* w, const float* gram_U_prev, SmReduceArgs* ra) {
+  int max_chunks = 1;
+  std::memset(ra, 0, sizeof(*ra));
+  for (int m = 0; m < pl->nd; ++m) {
+    ra->m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
+    ra->m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
+    ra->m[m].Gp = reinterpret_cast<double*>(w + pl->off_Gp[m]);
+    ra->m[m].a = (int)pl->dims[m];
+    ra->m[m].r = pl->r[m];
+    ra->m[m].nsplit = pl->nsplit[m];
+    ra->m[m].nchunk = pl->nchunk[m];
+    if (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) {
+      ra->m[m].gram = 1;
+      ra->m[m].nchunk = (int)((pl->dims[m] * pl->dims[m] + 24) / 25);   // ~25 Gram elements per CTA
+      ra->m[m].Pg = reinterpret_cast<double*>(w + pl->off_Pg[m]);
+      ra->m[m].U_prev = gram_U_prev + pl->u_off[m];
+    }
+    max_chunks = std::max(max_chunks, ra->m[m].nchunk);
+  }
+  ra->factor = 1;
+  ra->Rf = reinterpret_cast<double*>(w + pl->off_Rf);
+  ra->counter = reinterpret_cast<int*>(w) + 20;
+  ra->status = reinterpret_cast<int*>(w);
+  return max_chunks;
+}
+
+void build_fused_core(const asi_plan* pl, const void* act, float* U_new, float* core, char* w, bool gram_modes,
+                      SmCoreArgs* c) {
+  c->act = act;
+  c->U_new = U_new;
+  c->Rf = reinterpret_cast<const double*>(w + pl->off_Rf);
+  c->Tp = reinterpret_cast<float*>(w + pl->off_T[0]);
+  c->core = core;
+  c->status = reinterpret_cast<int*>(w);
+  c->counter = reinterpret_cast<int*>(w) + 16;
+  c->gcount = reinterpret_cast<int*>(w) + 64;
+  c->gs = pl->fold_gs;
+  c->Tg = reinterpret_cast<float*>(w + pl->off_T[1]);
+  for (int m = 0; m < 4; ++m) {
+    const bool gram = gram_modes && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2;
+    c->Pred[m] = reinterpret_cast<const double*>(w + (gram ? pl->off_Pg[m] : pl->off_Pred[m]));
+    c->u_off[m] = pl->u_off[m];
+    c->r[m] = pl->r[m];
+  }
+  c->B = (int)pl->dims[0];
+  c->C = (int)pl->dims[1];
+  c->n_tiles = pl->n_tiles_b;
+}
+
+// false: dY is not aligned as the staged copies of this plan need
+bool build_fused_wgrad(const asi_plan* pl, const float* core, const float* U, const void* dY, float* dW, char* w,
+                       SmWgradArgs* g) {
+  g->core = core; g->U = U; g->dY = dY; g->dW = dW;
+  for (int m = 0; m < 4; ++m) {
+    g->u_off[m] = pl->u_off[m];
+    g->r[m] = pl->r[m];
+  }
+  g->B = (int)pl->dims[0]; g->C = (int)pl->dims[1]; g->Cout = pl->d.cout;
+  g->H = (int)pl->dims[2]; g->W = (int)pl->dims[3]; g->Ho = (int)pl->Ho; g->Wo = (int)pl->Wo;
+  g->kh = pl->d.kh; g->kw = pl->d.kw; g->sh = pl->d.stride_h; g->sw = pl->d.stride_w;
+  g->ph = pl->d.pad_h; g->pw = pl->d.pad_w; g->groups = pl->d.groups; g->cpb = pl->cpb;
+  g->ncl = pl->wgrad_ncl;
+  g->pj = sm_wgrad_pitch(pl->cpb * (int)(pl->Ho * pl->Wo));
+  g->bulk = pl->wgrad_bulk ? 1 : 0;
+  if (g->bulk && (reinterpret_cast<uintptr_t>(dY) & 15u)) return false;
+  g->status = reinterpret_cast<int*>(w);
+  g->bulk_store = (((pl->dims[1] / pl->d.groups) * pl->d.kh * pl->d.kw) % 4 == 0 &&
+                   (reinterpret_cast<uintptr_t>(dW) & 15u) == 0) ? 1 : 0;
+  return true;
+}
+
 // U_m^{new} = Orthogonalize(P_m) for all modes given the split partials.
 // gram_U_prev != nullptr: the partials of modes 3 and 4 of a 7x7 or 14x14 map are Gram matrices A_m A_m^T
 // (written by the fused first pass) and P_m = G_m U_m^prev is formed during the reduction.
@@ -272,27 +386,7 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
   for (int m = 0; m < pl->nd; ++m) max_chunks = std::max(max_chunks, pl->nchunk[m]);
   if (pl->fast_compress) {
     SmReduceArgs ra;
-    std::memset(&ra, 0, sizeof(ra));
-    for (int m = 0; m < pl->nd; ++m) {
-      ra.m[m].Pp = reinterpret_cast<const float*>(w + pl->off_Pp[m]);
-      ra.m[m].Pred = reinterpret_cast<double*>(w + pl->off_Pred[m]);
-      ra.m[m].Gp = reinterpret_cast<double*>(w + pl->off_Gp[m]);
-      ra.m[m].a = (int)pl->dims[m];
-      ra.m[m].r = pl->r[m];
-      ra.m[m].nsplit = pl->nsplit[m];
-      ra.m[m].nchunk = pl->nchunk[m];
-      if (gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2) {
-        ra.m[m].gram = 1;
-        ra.m[m].nchunk = (int)((pl->dims[m] * pl->dims[m] + 24) / 25);   // ~25 Gram elements per CTA
-        ra.m[m].Pg = reinterpret_cast<double*>(w + pl->off_Pg[m]);
-        ra.m[m].U_prev = gram_U_prev + pl->u_off[m];
-        max_chunks = std::max(max_chunks, ra.m[m].nchunk);
-      }
-    }
-    ra.factor = 1;
-    ra.Rf = reinterpret_cast<double*>(w + pl->off_Rf);
-    ra.counter = reinterpret_cast<int*>(w) + 20;
-    ra.status = reinterpret_cast<int*>(w);
+    max_chunks = build_fused_reduce(pl, w, gram_U_prev, &ra);
     ASI_CUDA(launch_sm_reduce(ra, pl->nd, max_chunks, st));
     return ASI_OK;      // the core kernel solves for the rows of U_m
   }
@@ -328,6 +422,28 @@ asi_status_t orthogonalize_all(const asi_plan* pl, float* U_new, char* w, const 
   return ASI_OK;
 }
 
+// A mode product that streams a large tensor once: the register-tiled kernel when the shape fits it
+// (strided fibers, a <= 128, at most four outputs, contiguous outputs per (o, j)), else the general one.
+cudaError_t stream_modeprod(const asi_plan* pl, const ModeProdArgs& a, bool x_bf16, cudaStream_t st) {
+  const bool fits = !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) && a.si == 1 && a.ldb_j == 1 && a.sj == a.I &&
+                    a.so == (int64_t)a.n_out * a.I && a.Q * a.a >= (1 << 20) &&
+                    fiber2_supported(a.O, a.a, a.I, a.n_out, x_bf16) &&
+                    (reinterpret_cast<uintptr_t>(a.X) & 15u) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0;
+  if (!fits) return launch_modeprod(a, x_bf16, st);
+  Fiber2Args f;
+  std::memset(&f, 0, sizeof(f));
+  f.X = a.X;
+  f.U = a.B;
+  f.ldu = (int)a.ldb_k;
+  f.Y = a.Y;
+  f.y_so = a.so;
+  f.y_sj = a.sj;
+  f.O = a.O; f.I = a.I; f.a = (int)a.a; f.r = a.n_out;
+  f.n_tiles = fiber2_tiles(a.O, a.I);
+  f.project_only = 1;
+  return launch_fiber2(f, (int)std::min<int64_t>(f.n_tiles, 296), x_bf16, st);
+}
+
 // Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).
 asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, float* core,
                              char* w, const float* gram_U_prev, cudaStream_t st) {
@@ -335,25 +451,7 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
   if (qs != ASI_OK) return qs;
   if (pl->fast_compress) {
     SmCoreArgs c;
-    c.act = act;
-    c.U_new = U_new;
-    c.Rf = reinterpret_cast<const double*>(w + pl->off_Rf);
-    c.Tp = reinterpret_cast<float*>(w + pl->off_T[0]);
-    c.core = core;
-    c.status = reinterpret_cast<int*>(w);
-    c.counter = reinterpret_cast<int*>(w) + 16;
-    c.gcount = reinterpret_cast<int*>(w) + 64;
-    c.gs = pl->fold_gs;
-    c.Tg = reinterpret_cast<float*>(w + pl->off_T[1]);
-    for (int m = 0; m < 4; ++m) {
-      const bool gram = gram_U_prev && (pl->fast_S == 7 || pl->fast_S == 14) && m >= 2;
-      c.Pred[m] = reinterpret_cast<const double*>(w + (gram ? pl->off_Pg[m] : pl->off_Pred[m]));
-      c.u_off[m] = pl->u_off[m];
-      c.r[m] = pl->r[m];
-    }
-    c.B = (int)pl->dims[0];
-    c.C = (int)pl->dims[1];
-    c.n_tiles = pl->n_tiles_b;
+    build_fused_core(pl, act, U_new, core, w, gram_U_prev != nullptr, &c);
     ASI_CUDA(launch_sm_core(c, pl->fast_S, pl->fast_R, pl->bf16, st));
     return ASI_OK;
   }
@@ -383,10 +481,23 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
     a.tc_scratch = w + pl->off_tc;
     a.tc_scratch_bytes = pl->tc_bytes;
     a.status = reinterpret_cast<int*>(w);
-    ASI_CUDA(launch_modeprod(a, src_bf16, st));
+    ASI_CUDA(stream_modeprod(pl, a, src_bf16, st));
     cd[m] = pl->r[m];
     src = dst;
     src_bf16 = false;
+    if (s == 0 && pl->core_tail) {
+      CoreTailArgs t;
+      std::memset(&t, 0, sizeof(t));
+      t.T = dst;
+      t.U2 = U_new + pl->u_off[1]; t.U3 = U_new + pl->u_off[2]; t.U4 = U_new + pl->u_off[3];
+      t.part = reinterpret_cast<float*>(w + pl->off_ctp);
+      t.core = core;
+      t.counter = reinterpret_cast<int*>(w) + 32;
+      t.r1 = pl->r[0]; t.r2 = pl->r[1]; t.r3 = pl->r[2]; t.r4 = pl->r[3];
+      t.C = (int)pl->dims[1]; t.H = (int)pl->dims[2]; t.W = (int)pl->dims[3];
+      ASI_CUDA(launch_core_tail(t, st));
+      break;
+    }
   }
   return ASI_OK;
 }
@@ -569,19 +680,7 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     // fp32 tiles are staged by 16-byte asynchronous copies, which need 16-byte aligned sources
     if (!pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
     SmPass1Args a;
-    a.act = act;
-    a.U_prev = U_prev;
-    for (int m = 0; m < 4; ++m) {
-      a.Pp[m] = reinterpret_cast<float*>(w + pl->off_Pp[m]);
-      a.u_off[m] = pl->u_off[m];
-      a.r[m] = pl->r[m];
-    }
-    a.status = reinterpret_cast<int*>(w);     // cleared by the kernel itself
-    a.B = (int)pl->dims[0];
-    a.C = (int)pl->dims[1];
-    a.n_tiles_b = pl->n_tiles_b;
-    a.stall_copy = (pl->d.flags & ASI_FLAG_TEST_EXPIRE_WAIT) ? 1 : 0;
-    a.wait_ns = a.stall_copy ? 1000000ull : 1000000000ull;      // 1 ms under the test hook, else 1 s
+    build_fused_pass1(pl, act, U_prev, w, &a);
     ASI_CUDA(launch_sm_pass1(a, pl->fast_S, pl->fast_R, pl->bf16, st));
     return finish_compress(pl, act, U_new, core, w, U_prev, st);
   }
@@ -599,11 +698,30 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     g.r3 = pl->r[2];
     g.r4 = pl->r[3];
     g.vec4 = (!pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u) == 0) ? 1 : 0;
-    ASI_CUDA(launch_plane(g, pl->plane_grid, pl->bf16, st));
+    g.status = reinterpret_cast<int*>(w);
+    if (pl->plane2) {
+      if (reinterpret_cast<uintptr_t>(act) & 15u) return ASI_ERR_INVALID_ARG;   // bulk copies need 16-byte alignment
+      ASI_CUDA(launch_plane2(g, pl->plane_grid, pl->bf16, st));
+    } else {
+      ASI_CUDA(launch_plane(g, pl->plane_grid, pl->bf16, st));
+    }
   }
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
     if (pl->plane && m >= 2) continue;
+    if (pl->fiber2[m]) {
+      if (reinterpret_cast<uintptr_t>(act) & 15u) return ASI_ERR_INVALID_ARG;
+      Fiber2Args f;
+      std::memset(&f, 0, sizeof(f));
+      f.X = act;
+      f.U = U_prev + pl->u_off[m];
+      f.ldu = v.r;
+      f.Pp = reinterpret_cast<float*>(w + pl->off_Pp[m]);
+      f.O = v.O; f.I = v.I; f.a = (int)v.a; f.r = v.r;
+      f.n_tiles = fiber2_tiles(v.O, v.I);
+      ASI_CUDA(launch_fiber2(f, pl->fiber_grid[m], pl->bf16, st));
+      continue;
+    }
     if (pl->fiber[m]) {
       // both products of the mode in one pass; V stays on chip
       FiberArgs f;
@@ -641,6 +759,112 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     if (s != ASI_OK) return s;
   }
   return finish_compress(pl, act, U_new, core, w, nullptr, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Batched entry points: the layers a training step compresses together (Algorithm 1 runs once per
+// fine-tuned layer and step; Sec. 4 fine-tunes the last 2..4 layers).  Layers on the fused small-map path
+// that share a kernel variant go through ONE launch of each kernel stage, their argument blocks in a
+// table the CTAs index; the remaining layers are enqueued one after another on the same stream.
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct Variant {
+  int S, R, bf16;
+  bool operator==(const Variant& o) const { return S == o.S && R == o.R && bf16 == o.bf16; }
+};
+}  // namespace
+
+asi_status_t asi_compress_batched(const asi_plan_t* const* plans, const void* const* acts,
+                                  const float* const* U_prev, float* const* U_new, float* const* cores,
+                                  void* const* ws, const size_t* ws_bytes, int32_t n, void* stream) {
+  if (!plans || !acts || !U_prev || !U_new || !cores || !ws || !ws_bytes || n < 1 || n > 4096)
+    return ASI_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    const asi_plan* pl = plans[i];
+    if (!pl || !valid_ptr(acts[i]) || !valid_ptr(U_prev[i]) || !valid_ptr(U_new[i]) || !valid_ptr(cores[i]))
+      return ASI_ERR_INVALID_ARG;
+    if (U_prev[i] == U_new[i]) return ASI_ERR_INVALID_ARG;
+    const asi_status_t s = check_ws(ws[i], ws_bytes[i], pl->compress_ws);
+    if (s != ASI_OK) return s;
+    if (pl->fast_compress && !pl->bf16 && (reinterpret_cast<uintptr_t>(acts[i]) & 15u)) return ASI_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (ws[j] == ws[i]) return ASI_ERR_INVALID_ARG;            // every layer needs a workspace of its own
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::vector<char> done(n, 0);
+  const int maxb = sm_max_batch();
+  for (int i = 0; i < n; ++i) {
+    if (done[i] || !plans[i]->fast_compress) continue;
+    const Variant v = {plans[i]->fast_S, plans[i]->fast_R, plans[i]->bf16 ? 1 : 0};
+    std::vector<int> grp;
+    for (int j = i; j < n && (int)grp.size() < maxb; ++j) {
+      const asi_plan* q = plans[j];
+      if (!done[j] && q->fast_compress && v == Variant{q->fast_S, q->fast_R, q->bf16 ? 1 : 0}) grp.push_back(j);
+    }
+    const int g = (int)grp.size();
+    std::vector<SmPass1Args> pa(g);
+    std::vector<SmReduceArgs> ra(g);
+    std::vector<SmCoreArgs> ca(g);
+    std::vector<int> mc(g);
+    for (int k = 0; k < g; ++k) {
+      const int j = grp[k];
+      char* w = static_cast<char*>(ws[j]);
+      build_fused_pass1(plans[j], acts[j], U_prev[j], w, &pa[k]);
+      mc[k] = build_fused_reduce(plans[j], w, U_prev[j], &ra[k]);
+      build_fused_core(plans[j], acts[j], U_new[j], cores[j], w, true, &ca[k]);
+      done[j] = 1;
+    }
+    ASI_CUDA(launch_sm_pass1_batched(pa.data(), g, v.S, v.R, v.bf16 != 0, st));
+    ASI_CUDA(launch_sm_reduce_batched(ra.data(), mc.data(), g, st));
+    ASI_CUDA(launch_sm_core_batched(ca.data(), g, v.S, v.R, v.bf16 != 0, st));
+  }
+  for (int i = 0; i < n; ++i) {
+    if (done[i]) continue;
+    const asi_status_t s = asi_compress(plans[i], acts[i], U_prev[i], U_new[i], cores[i], ws[i], ws_bytes[i], stream);
+    if (s != ASI_OK) return s;
+  }
+  return ASI_OK;
+}
+
+asi_status_t asi_wgrad_batched(const asi_plan_t* const* plans, const float* const* cores, const float* const* U,
+                               const void* const* dY, float* const* dW, void* const* ws, const size_t* ws_bytes,
+                               int32_t n, void* stream) {
+  if (!plans || !cores || !U || !dY || !dW || !ws || !ws_bytes || n < 1 || n > 4096) return ASI_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    const asi_plan* pl = plans[i];
+    if (!pl || !valid_ptr(cores[i]) || !valid_ptr(U[i]) || !valid_ptr(dY[i]) || !valid_ptr(dW[i]))
+      return ASI_ERR_INVALID_ARG;
+    const asi_status_t s = check_ws(ws[i], ws_bytes[i], pl->wgrad_ws);
+    if (s != ASI_OK) return s;
+    if (pl->fast_wgrad && pl->wgrad_bulk && (reinterpret_cast<uintptr_t>(dY[i]) & 15u)) return ASI_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::vector<char> done(n, 0);
+  const int maxb = sm_max_batch();
+  for (int i = 0; i < n; ++i) {
+    if (done[i] || !plans[i]->fast_wgrad) continue;
+    const int R = plans[i]->fast_R, bf = plans[i]->bf16 ? 1 : 0;
+    std::vector<SmWgradArgs> wa;
+    for (int j = i; j < n && (int)wa.size() < maxb; ++j) {
+      const asi_plan* q = plans[j];
+      if (done[j] || !q->fast_wgrad || q->fast_R != R || (q->bf16 ? 1 : 0) != bf) continue;
+      SmWgradArgs g;
+      if (!build_fused_wgrad(q, cores[j], U[j], dY[j], dW[j], static_cast<char*>(ws[j]), &g))
+        return ASI_ERR_INVALID_ARG;
+      wa.push_back(g);
+      done[j] = 1;
+    }
+    ASI_CUDA(launch_sm_wgrad_batched(wa.data(), (int)wa.size(), R, bf != 0, st));
+  }
+  for (int i = 0; i < n; ++i) {
+    if (done[i]) continue;
+    const asi_plan* pl = plans[i];
+    const asi_status_t s = pl->d.kind == ASI_CONV2D
+        ? asi_conv_wgrad(pl, cores[i], U[i], dY[i], dW[i], ws[i], ws_bytes[i], stream)
+        : asi_linear_wgrad(pl, cores[i], U[i], dY[i], dW[i], ws[i], ws_bytes[i], stream);
+    if (s != ASI_OK) return s;
+  }
+  return ASI_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -710,22 +934,7 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
   char* w = static_cast<char*>(ws);
   if (pl->fast_wgrad) {
     SmWgradArgs g;
-    g.core = core; g.U = U; g.dY = dY; g.dW = dW;
-    for (int m = 0; m < 4; ++m) {
-      g.u_off[m] = pl->u_off[m];
-      g.r[m] = pl->r[m];
-    }
-    g.B = (int)pl->dims[0]; g.C = (int)pl->dims[1]; g.Cout = pl->d.cout;
-    g.H = (int)pl->dims[2]; g.W = (int)pl->dims[3]; g.Ho = (int)pl->Ho; g.Wo = (int)pl->Wo;
-    g.kh = pl->d.kh; g.kw = pl->d.kw; g.sh = pl->d.stride_h; g.sw = pl->d.stride_w;
-    g.ph = pl->d.pad_h; g.pw = pl->d.pad_w; g.groups = pl->d.groups; g.cpb = pl->cpb;
-    g.ncl = pl->wgrad_ncl;
-    g.pj = sm_wgrad_pitch(pl->cpb * (int)(pl->Ho * pl->Wo));
-    g.bulk = pl->wgrad_bulk ? 1 : 0;
-    if (g.bulk && (reinterpret_cast<uintptr_t>(dY) & 15u)) return ASI_ERR_INVALID_ARG;
-    g.status = reinterpret_cast<int*>(w);
-    g.bulk_store = (((pl->dims[1] / pl->d.groups) * pl->d.kh * pl->d.kw) % 4 == 0 &&
-                    (reinterpret_cast<uintptr_t>(dW) & 15u) == 0) ? 1 : 0;
+    if (!build_fused_wgrad(pl, core, U, dY, dW, w, &g)) return ASI_ERR_INVALID_ARG;
     ASI_CUDA(launch_sm_wgrad(g, pl->fast_R, pl->bf16, st));
     return ASI_OK;
   }
@@ -741,8 +950,12 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
   a.X = dY; a.B = U + pl->u_off[0]; a.Y = Z1;
   a.O = 1; a.a = B; a.I = per_sample; a.Q = per_sample;
   a.n_out = r1; a.ldb_k = r1; a.ldb_j = 1;
-  a.so = 0; a.sj = per_sample; a.si = 1;
-  ASI_CUDA(launch_modeprod(a, pl->bf16, st));
+  a.so = (int64_t)r1 * per_sample; a.sj = per_sample; a.si = 1;
+  ASI_CUDA(stream_modeprod(pl, a, pl->bf16, st));
+  if (pl->conv_z3) {
+    // terms 2-3 in one launch
+    ASI_CUDA(launch_z3(core, U + pl->u_off[2], U + pl->u_off[3], Z3, r1 * r2, r3, r4, (int)H, (int)W, st));
+  } else {
   // term 2: core x_3 U_3  -> [r1 r2, H, r4]
   a.X = core; a.B = U + pl->u_off[2]; a.Y = Z3a;
   a.O = (int64_t)r1 * r2; a.a = r3; a.I = r4; a.Q = a.O * a.I;
@@ -755,6 +968,7 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float
   a.n_out = (int)W; a.ldb_k = 1; a.ldb_j = r4;
   a.so = W; a.sj = 1; a.si = 1;
   ASI_CUDA(launch_modeprod(a, false, st));
+  }
   // terms 4 and 5
   ConvTailArgs t;
   t.Z1 = Z1; t.Z3 = Z3; t.U2 = U + pl->u_off[1]; t.dW = dW;

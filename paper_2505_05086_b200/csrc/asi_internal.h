@@ -68,6 +68,19 @@ struct PlaneArgs {
   float* Pp4;          // [grid][S][r4]
   int64_t n_planes;
   int S, r3, r4, vec4;
+  int* status = nullptr;   // status word of the workspace (k_plane2: an expired wait on the bulk copy)
+};
+
+// One mode with strided fibers, a <= 128, r <= 4 (k_fiber2): both products in one pass, or with
+// project_only the mode product Y[o][j][i] = sum_k X[o][k][i] U[k][j] alone.
+struct Fiber2Args {
+  const void* X;
+  const float* U;      // U[k * ldu + j]
+  float* Pp;           // [grid][a][r] partials of P (not project_only)
+  float* Y;            // project_only: Y[o * y_so + j * y_sj + i]
+  int64_t y_so, y_sj;
+  int64_t O, I, n_tiles;
+  int ldu, a, r, project_only, nstage;
 };
 
 struct QRMode {
@@ -169,6 +182,12 @@ cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_
 cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cudaStream_t st);
 cudaError_t launch_sm_core(const SmCoreArgs& p, int S, int R, bool bf16, cudaStream_t st);
 cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t st);
+// the same kernels over several layers of one variant in one launch each (n <= sm_max_batch())
+int sm_max_batch();
+cudaError_t launch_sm_pass1_batched(const SmPass1Args* a, int n, int S, int R, bool bf16, cudaStream_t st);
+cudaError_t launch_sm_reduce_batched(const SmReduceArgs* a, const int* max_chunks, int n, cudaStream_t st);
+cudaError_t launch_sm_core_batched(const SmCoreArgs* a, int n, int S, int R, bool bf16, cudaStream_t st);
+cudaError_t launch_sm_wgrad_batched(const SmWgradArgs* a, int n, int R, bool bf16, cudaStream_t st);
 
 // Benchmark timing aid (asi_profile_begin / asi_profile_end).
 struct ProfState {
@@ -209,9 +228,30 @@ size_t fiber_smem(int a);
 size_t conv_tail_smem(int r2, int kh, int kw);
 cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t st);
 size_t plane_smem(int S);
+bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16);
+int64_t fiber2_tiles(int64_t O, int64_t I);
+cudaError_t launch_fiber2(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st);
+// core = T x_2 U_2^T x_3 U_3^T x_4 U_4^T for T [r1][C][H][W] in one launch (k_core_tail)
+struct CoreTailArgs {
+  const float* T;
+  const float *U2, *U3, *U4;
+  float* part;         // [r1][chunks x splits][r2 r3 r4] partial cores
+  float* core;
+  int* counter;        // zero on entry, zero again on exit
+  int r1, r2, r3, r4, C, H, W, RH, cper;
+};
+bool core_tail_supported(int r2, int r3, int r4, int H, int W);
+size_t core_tail_part_elems(int r1, int r2, int r3, int r4, int C, int H, int W);
+cudaError_t launch_core_tail(const CoreTailArgs& p, cudaStream_t st);
+cudaError_t launch_z3(const float* core, const float* U3, const float* U4, float* Z3, int r12, int r3, int r4,
+                      int H, int W, cudaStream_t st);
+bool plane2_supported(int S, int64_t n_planes, int r3, int r4);
+int plane2_grid(int S, int64_t n_planes, int max_ctas);
+cudaError_t launch_plane2(const PlaneArgs& p, int grid, bool bf16, cudaStream_t st);
 int64_t fiber_tiles(int64_t O, int64_t a, int64_t I);
 cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
 cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, cudaStream_t st);
+
 
 }  // namespace asi
 
@@ -239,6 +279,9 @@ struct asi_plan {
   // wgrad workspace (byte offsets)
   size_t off_Z[3], off_Z4p;
   int conv_nsp;                    // > 1: terms 4-5 in two launches with conv_nsp partial Z4 per channel
+  bool conv_z3;                    // terms 2-3 in one launch (k_z3)
+  bool core_tail;                  // the core products after the first in one launch
+  size_t off_ctp;                  // partial cores of that launch
   size_t wgrad_ws;
 
   int launches_compress, launches_wgrad;
@@ -250,5 +293,7 @@ struct asi_plan {
   int fiber_grid[ASI_MAX_MODES];
   bool plane;                      // modes 3 and 4 together by the whole-plane kernel
   int plane_grid;
+  bool fiber2[ASI_MAX_MODES];      // ... by its register-tiled successor (ranks <= 4, 16-byte aligned rows)
+  bool plane2;                     // 28 x 28 and 56 x 56 planes, ranks <= 4
   int fast_S, fast_R, n_tiles_b, cpb, wgrad_ncl, fold_gs;
 };

@@ -421,7 +421,7 @@ __device__ __forceinline__ void gram14_slot(int o, int& rl, int& e) {
 // k_sm_pass1
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
-__global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
+__device__ __forceinline__ void sm_pass1_cta(const SmPass1Args& p, const int bid) {
   constexpr bool kBulk = std::is_same<TX, float>::value;
   constexpr bool kGram = (S == 7);                   // modes 3, 4 as Gram matrices A_m A_m^T (7 x 7)
   constexpr bool kGram14 = (S == 14);                // ... as 14 x 14 Gram matrices in four 7 x 7 blocks
@@ -437,13 +437,13 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
   const TX* __restrict__ A = reinterpret_cast<const TX*>(p.act);
   const int B = p.B, C = p.C;
 
-  if (blockIdx.x == 0 && tid < 241) p.status[tid == 0 ? 0 : 15 + tid] = 0;  // status word, counters 16..255
+  if (bid == 0 && tid < 241) p.status[tid == 0 ? 0 : 15 + tid] = 0;  // status word, counters 16..255
   pdl_launch_dependents();
 
   constexpr int kNQ = (S == 7) ? 1 : 4;             // role-C CTAs per sample
-  if ((int)blockIdx.x >= B * kNQ) {
+  if (bid >= B * kNQ) {
     // ---------------- role B: modes 1, 3, 4 on tile [B x J] ----------------
-    const int tile = blockIdx.x - B * kNQ;
+    const int tile = bid - B * kNQ;
     float* Xs = smem;                                // [B][PJ]
     float* U1s = Xs + B * PJ;                        // [B][R]
     float* U3s = U1s + B * R;                        // [S][R]
@@ -619,7 +619,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     constexpr int PC = role_c_pitch(S);
     constexpr int G = kNT / HWC;
     constexpr bool kBulkC = kBulk && NQ == 1;
-    const int b = blockIdx.x / NQ, q = blockIdx.x % NQ;
+    const int b = bid / NQ, q = bid % NQ;
     const int hw0 = (S == 14) ? (q == 0 ? 0 : 4 + 48 * q) : q * HWC;     // first position of this part
     const int nval = (S == 14 && q > 0) ? 48 : HWC;                      // positions it holds
     float* Xs = smem;                                // [C][PC]
@@ -660,7 +660,7 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
     }
     project_channels<HWC, PC, R>(Xs, U2s, Vp, V2s, C);
     // expansion: P2[c,:] = sum_hw X[c,hw] V2[hw,:], one channel row per thread
-    float* P2 = p.Pp[1] + (int64_t)blockIdx.x * C * p.r[1];
+    float* P2 = p.Pp[1] + (int64_t)bid * C * p.r[1];
     for (int c = tid; c < C; c += kNT) {
       const float* row = Xs + c * PC;
       float acc[R];
@@ -686,6 +686,31 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
   }
 }
 
+// A launch over several layers at once: the CTAs of layer l are [first[l], first[l + 1]).
+constexpr int kMaxBatch = 8;
+template <typename Args>
+struct SmBatch {
+  Args a[kMaxBatch];
+  int first[kMaxBatch + 1];
+  int n;
+};
+template <typename Args>
+__device__ __forceinline__ int batch_layer(const SmBatch<Args>& b, int bid) {
+  int l = 0;
+  while (l + 1 < b.n && bid >= b.first[l + 1]) ++l;
+  return l;
+}
+
+template <int S, int R, typename TX>
+__global__ void __launch_bounds__(kNT, 2) k_sm_pass1(const __grid_constant__ SmPass1Args p) {
+  sm_pass1_cta<S, R, TX>(p, (int)blockIdx.x);
+}
+template <int S, int R, typename TX>
+__global__ void __launch_bounds__(kNT, 2) k_sm_pass1_b(const __grid_constant__ SmBatch<SmPass1Args> b) {
+  const int l = batch_layer(b, (int)blockIdx.x);
+  sm_pass1_cta<S, R, TX>(b.a[l], (int)blockIdx.x - b.first[l]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_sm_reduce: CTA (c, m) sums rows [16 c, 16 c + 16) of the per-tile partials of P_m in fp64 in a
 // fixed order (thread (e, sg) takes the partials s == sg (mod SG); the SG sums meet in shared memory
@@ -695,10 +720,9 @@ __global__ void __launch_bounds__(kNT, 2) k_sm_pass1(SmPass1Args p) {
 // core kernel: it sums the shares of P_m^T P_m (a Gram mode: forms P_m = G_m U_m^prev first), and
 // leaves the Cholesky factor R_m and 1 / diag(R_m) in args.Rf.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
+__device__ __forceinline__ void sm_reduce_cta(const SmReduceArgs& args, const int c, const int mode) {
   constexpr int RM = 8, RPC = kRedRows;
-  const SmReduceMode M = args.m[blockIdx.y];
-  const int c = blockIdx.x;
+  const SmReduceMode& M = args.m[mode];
   pdl_launch_dependents();
   if (c >= M.nchunk) return;
   pdl_wait();                                      // the partials come from the previous kernel
@@ -766,7 +790,7 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
   __shared__ float Ups[16 * RM];
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = (atomicAdd(args.counter + blockIdx.y, 1) == M.nchunk - 1);
+  if (tid == 0) s_last = (atomicAdd(args.counter + mode, 1) == M.nchunk - 1);
   __syncthreads();
   if (!s_last) return;
   __threadfence();
@@ -837,12 +861,20 @@ __global__ void __launch_bounds__(kRedNT) k_sm_reduce(SmReduceArgs args) {
       if (in1 && i1 > j && k1 >= i1) Gs[i1][k1] -= Gs[j][i1] * Gs[j][k1];
       __syncwarp();
     }
-    double* Rf = args.Rf + blockIdx.y * kRfStride;
+    double* Rf = args.Rf + mode * kRfStride;
     if (in0) Rf[i0 * RM + k0] = Gs[i0][k0];
     if (in1) Rf[i1 * RM + k1] = Gs[i1][k1];
     if (lane < r) Rf[RM * RM + lane] = Dinv[lane];
-    if (lane == 0) args.counter[blockIdx.y] = 0;
+    if (lane == 0) args.counter[mode] = 0;
   }
+}
+
+__global__ void __launch_bounds__(kRedNT) k_sm_reduce(const __grid_constant__ SmReduceArgs args) {
+  sm_reduce_cta(args, (int)blockIdx.x, (int)blockIdx.y);
+}
+__global__ void __launch_bounds__(kRedNT) k_sm_reduce_b(const __grid_constant__ SmBatch<SmReduceArgs> b) {
+  const int l = batch_layer(b, (int)blockIdx.x);
+  sm_reduce_cta(b.a[l], (int)blockIdx.x - b.first[l], (int)blockIdx.y);
 }
 
 // <<<>>> with the programmatic-stream-serialization attribute
@@ -880,7 +912,7 @@ cudaError_t launch_sm_reduce(const SmReduceArgs& p, int nd, int max_chunks, cuda
 //   T[i,j,k,l] = Y x_3 U3^T x_4 U4^T  -> per-tile partial core, summed in two ordered levels.
 // ---------------------------------------------------------------------------------------------
 template <int S, int R, typename TX>
-__global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
+__device__ __forceinline__ void sm_core_cta(const SmCoreArgs& p, const int bid) {
   constexpr int HW = S * S;
   constexpr int CC = (S == 7) ? 4 : 1;
   constexpr int J = CC * HW;
@@ -890,7 +922,7 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   __shared__ int s_last;
   __shared__ double Rs[4][kRfStride];   // per mode: rows of R_m (pitch 8), then 1 / diag(R_m) at [64..]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int B = p.B, C = p.C, tile = blockIdx.x;
+  const int B = p.B, C = p.C, tile = bid;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
   float* Xs = smem;                     // [B][PJ]
   float* U1s = Xs + B * PJ;             // [B][R]
@@ -1057,6 +1089,16 @@ __global__ void __launch_bounds__(kNT) k_sm_core(SmCoreArgs p) {
   if (tid == 0) *p.counter = 0;
 }
 
+template <int S, int R, typename TX>
+__global__ void __launch_bounds__(kNT) k_sm_core(const __grid_constant__ SmCoreArgs p) {
+  sm_core_cta<S, R, TX>(p, (int)blockIdx.x);
+}
+template <int S, int R, typename TX>
+__global__ void __launch_bounds__(kNT) k_sm_core_b(const __grid_constant__ SmBatch<SmCoreArgs> b) {
+  const int l = batch_layer(b, (int)blockIdx.x);
+  sm_core_cta<S, R, TX>(b.a[l], (int)blockIdx.x - b.first[l]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // k_sm_wgrad: CTA owns cpb consecutive output channels, i.e. the dY tile [B x J], J = cpb*Ho*Wo
 // contiguous values per sample (staged by 16-byte cp.async when fp32 and 16-byte aligned).
@@ -1153,7 +1195,7 @@ __device__ __forceinline__ void wgrad_expand_rows(const SmWgradArgs& p, const fl
 }
 
 template <int R, typename TX>
-__global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
+__device__ __forceinline__ void sm_wgrad_cta(const SmWgradArgs& p, const int bid) {
   extern __shared__ __align__(128) float smem[];
   const int tid = threadIdx.x;
   const int r1 = p.r[0], r2 = p.r[1], r3 = p.r[2], r4 = p.r[3];
@@ -1161,7 +1203,7 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   const int J = p.cpb * HoWo;                        // dY columns of this CTA, contiguous per sample
   const int PJ = p.pj;
   const int NH = batch_groups(kNT, J);
-  const int c0 = blockIdx.x * p.cpb;
+  const int c0 = bid * p.cpb;
   const int n_out = p.cpb * r2 * kk;
   // staging blocks of term 5 reuse the tile's space: ncl channels per round, doubled when rounds follow
   const int n_stage = (p.cpb > p.ncl ? 2 : 1) * p.ncl * (p.C / p.groups) * kk;
@@ -1291,6 +1333,16 @@ __global__ void __launch_bounds__(kNT) k_sm_wgrad(SmWgradArgs p) {
   wgrad_expand_rows<R>(p, Z4s, U2s, Ys, c0);
 }
 
+template <int R, typename TX>
+__global__ void __launch_bounds__(kNT) k_sm_wgrad(const __grid_constant__ SmWgradArgs p) {
+  sm_wgrad_cta<R, TX>(p, (int)blockIdx.x);
+}
+template <int R, typename TX>
+__global__ void __launch_bounds__(kNT) k_sm_wgrad_b(const __grid_constant__ SmBatch<SmWgradArgs> b) {
+  const int l = batch_layer(b, (int)blockIdx.x);
+  sm_wgrad_cta<R, TX>(b.a[l], (int)blockIdx.x - b.first[l]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // host-side launchers
 // ---------------------------------------------------------------------------------------------
@@ -1375,9 +1427,7 @@ static cudaError_t launch_wgrad_t(const SmWgradArgs& p, cudaStream_t st) {
 
 cudaError_t launch_sm_pass1(const SmPass1Args& p, int S, int R, bool bf16, cudaStream_t st) {
   const size_t eb = bf16 ? 2 : 4;
-  double bytes = (double)p.B * p.C * S * S * eb;
-  const double m34 = (S == 7 || S == 14) ? 2.0 * S * S : (double)S * (p.r[2] + p.r[3]);
-  bytes += 4.0 * ((double)p.n_tiles_b * (p.B * p.r[0] + m34) + (double)p.B * p.C * p.r[1]);
+  const double bytes = (double)p.B * p.C * S * S * eb;      // the activation, read once
   ProfScope prof(ASI_K_SM_PASS1, st, bytes);
   ASI_DISPATCH_SR(launch_pass1_t, p);
 }
@@ -1395,6 +1445,117 @@ cudaError_t launch_sm_wgrad(const SmWgradArgs& p, int R, bool bf16, cudaStream_t
                      4.0 * (double)p.Cout * (p.C / p.groups) * p.kh * p.kw);
   if (R == 4) return bf16 ? launch_wgrad_t<4, __nv_bfloat16>(p, st) : launch_wgrad_t<4, float>(p, st);
   return bf16 ? launch_wgrad_t<8, __nv_bfloat16>(p, st) : launch_wgrad_t<8, float>(p, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Batched launches: the same kernels over the tiles of up to kMaxBatch layers of one variant (map size,
+// rank bucket, input type) in one grid.  The per-layer argument blocks travel as a kernel parameter; a CTA
+// finds its layer from the table of first CTA indices.
+// ---------------------------------------------------------------------------------------------
+int sm_max_batch() { return kMaxBatch; }
+
+template <int S, int R, typename TX>
+static cudaError_t launch_pass1_bt(const SmBatch<SmPass1Args>& b, size_t smem, cudaStream_t st) {
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_pass1_b<S, R, TX>), smem);
+  if (e != cudaSuccess) return e;
+  k_sm_pass1_b<S, R, TX><<<b.first[b.n], kNT, smem, st>>>(b);
+  return cudaGetLastError();
+}
+template <int S, int R, typename TX>
+static cudaError_t launch_core_bt(const SmBatch<SmCoreArgs>& b, size_t smem, cudaStream_t st) {
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_core_b<S, R, TX>), smem);
+  if (e != cudaSuccess) return e;
+  return launch_dependent(k_sm_core_b<S, R, TX>, dim3(b.first[b.n]), dim3(kNT), smem, st, b);
+}
+template <int R, typename TX>
+static cudaError_t launch_wgrad_bt(const SmBatch<SmWgradArgs>& b, size_t smem, cudaStream_t st) {
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_sm_wgrad_b<R, TX>), smem);
+  if (e != cudaSuccess) return e;
+  k_sm_wgrad_b<R, TX><<<b.first[b.n], kNT, smem, st>>>(b);
+  return cudaGetLastError();
+}
+
+#define ASI_DISPATCH_SRB(FN, ARGS, SMEM)                                       \
+  do {                                                                         \
+    if (S == 7) {                                                              \
+      if (R == 4) return bf16 ? FN<7, 4, __nv_bfloat16>(ARGS, SMEM, st) : FN<7, 4, float>(ARGS, SMEM, st);   \
+      return bf16 ? FN<7, 8, __nv_bfloat16>(ARGS, SMEM, st) : FN<7, 8, float>(ARGS, SMEM, st);               \
+    }                                                                          \
+    if (S == 14) {                                                             \
+      if (R == 4) return bf16 ? FN<14, 4, __nv_bfloat16>(ARGS, SMEM, st) : FN<14, 4, float>(ARGS, SMEM, st); \
+      return bf16 ? FN<14, 8, __nv_bfloat16>(ARGS, SMEM, st) : FN<14, 8, float>(ARGS, SMEM, st);             \
+    }                                                                          \
+    if (R == 4) return bf16 ? FN<16, 4, __nv_bfloat16>(ARGS, SMEM, st) : FN<16, 4, float>(ARGS, SMEM, st);   \
+    return bf16 ? FN<16, 8, __nv_bfloat16>(ARGS, SMEM, st) : FN<16, 8, float>(ARGS, SMEM, st);               \
+  } while (0)
+
+cudaError_t launch_sm_pass1_batched(const SmPass1Args* a, int n, int S, int R, bool bf16, cudaStream_t st) {
+  if (n < 1 || n > kMaxBatch) return cudaErrorInvalidValue;
+  SmBatch<SmPass1Args> b;
+  size_t smem = 0;
+  double bytes = 0.0;
+  b.n = n;
+  b.first[0] = 0;
+  for (int l = 0; l < n; ++l) {
+    b.a[l] = a[l];
+    b.first[l + 1] = b.first[l] + a[l].n_tiles_b + sm_pass1_role_c_ctas(S, a[l].B);
+    const size_t need = sm_pass1_smem(S, R, a[l].B, a[l].C);
+    if (need > smem) smem = need;
+    bytes += (double)a[l].B * a[l].C * S * S * (bf16 ? 2 : 4);
+  }
+  ProfScope prof(ASI_K_SM_PASS1, st, bytes);
+  ASI_DISPATCH_SRB(launch_pass1_bt, b, smem);
+}
+
+cudaError_t launch_sm_reduce_batched(const SmReduceArgs* a, const int* max_chunks, int n, cudaStream_t st) {
+  if (n < 1 || n > kMaxBatch) return cudaErrorInvalidValue;
+  SmBatch<SmReduceArgs> b;
+  b.n = n;
+  b.first[0] = 0;
+  for (int l = 0; l < n; ++l) {
+    b.a[l] = a[l];
+    b.first[l + 1] = b.first[l] + max_chunks[l];
+  }
+  ProfScope prof(ASI_K_QR, st, 0.0);
+  return launch_dependent(k_sm_reduce_b, dim3((unsigned)b.first[n], 4), dim3(kRedNT), 0, st, b);
+}
+
+cudaError_t launch_sm_core_batched(const SmCoreArgs* a, int n, int S, int R, bool bf16, cudaStream_t st) {
+  if (n < 1 || n > kMaxBatch) return cudaErrorInvalidValue;
+  SmBatch<SmCoreArgs> b;
+  size_t smem = 0;
+  double bytes = 0.0;
+  b.n = n;
+  b.first[0] = 0;
+  for (int l = 0; l < n; ++l) {
+    b.a[l] = a[l];
+    b.first[l + 1] = b.first[l] + a[l].n_tiles;
+    const size_t need = sm_core_smem(S, R, a[l].B);
+    if (need > smem) smem = need;
+    bytes += (double)a[l].B * a[l].C * S * S * (bf16 ? 2 : 4);
+  }
+  ProfScope prof(ASI_K_SM_CORE, st, bytes);
+  ASI_DISPATCH_SRB(launch_core_bt, b, smem);
+}
+
+cudaError_t launch_sm_wgrad_batched(const SmWgradArgs* a, int n, int R, bool bf16, cudaStream_t st) {
+  if (n < 1 || n > kMaxBatch) return cudaErrorInvalidValue;
+  SmBatch<SmWgradArgs> b;
+  size_t smem = 0;
+  double bytes = 0.0;
+  b.n = n;
+  b.first[0] = 0;
+  for (int l = 0; l < n; ++l) {
+    b.a[l] = a[l];
+    b.first[l + 1] = b.first[l] + a[l].Cout / a[l].cpb;
+    const size_t need = sm_wgrad_smem(a[l], R);
+    if (need > smem) smem = need;
+    bytes += (double)a[l].B * a[l].Cout * a[l].Ho * a[l].Wo * (bf16 ? 2 : 4) +
+             4.0 * (double)a[l].Cout * (a[l].C / a[l].groups) * a[l].kh * a[l].kw;
+  }
+  ProfScope prof(ASI_K_SM_WGRAD, st, bytes);
+  if (R == 4) return bf16 ? launch_wgrad_bt<4, __nv_bfloat16>(b, smem, st) : launch_wgrad_bt<4, float>(b, smem, st);
+  return bf16 ? launch_wgrad_bt<8, __nv_bfloat16>(b, smem, st) : launch_wgrad_bt<8, float>(b, smem, st);
 }
 
 }  // namespace asi

@@ -5,7 +5,7 @@ from __future__ import annotations
 import numpy as np
 import torch
 
-from .binding import ASI_OK, Plan
+from .binding import ASI_OK, Batch, Plan
 
 
 def _stream_handle(stream=None):
@@ -81,3 +81,26 @@ class LayerRunner:
 
     def ok(self):
         return self.device_status() == ASI_OK
+
+
+class StepRunner:
+    """The layers of one training step behind the batched entry points: one asi_compress_batched call
+    for the forward pass, one asi_wgrad_batched call for the backward pass."""
+
+    def __init__(self, runners):
+        self.runners = list(runners)
+        self.batch = Batch([r.plan for r in self.runners])
+
+    def compress(self, acts, stream=None):
+        rs = self.runners
+        self.batch.compress([a.data_ptr() for a in acts], [r.U[r.cur].data_ptr() for r in rs],
+                            [r.U[1 - r.cur].data_ptr() for r in rs], [r.core.data_ptr() for r in rs],
+                            [r.ws_c.data_ptr() for r in rs], [r.ws_c.numel() for r in rs], _stream_handle(stream))
+        for r in rs:
+            r.cur = 1 - r.cur
+
+    def wgrad(self, dys, stream=None):
+        rs = self.runners
+        self.batch.wgrad([r.core.data_ptr() for r in rs], [r.U[r.cur].data_ptr() for r in rs],
+                         [d.data_ptr() for d in dys], [r.dW.data_ptr() for r in rs],
+                         [r.ws_w.data_ptr() for r in rs], [r.ws_w.numel() for r in rs], _stream_handle(stream))

@@ -135,3 +135,24 @@ def test_host_detectable_call_errors_enqueue_nothing(asi):
     assert L.asi_step_host(h, None, None, None, None, None, None, None, 0, None) == 1
     assert L.asi_step_host_arena_bytes(h) >= ws
     assert p.launch_count(0) > 0 and p.launch_count(1) > 0
+
+
+def test_batched_entry_points_validate_before_enqueuing(asi):
+    """Null arrays, an empty batch and two layers sharing one workspace are refused on the host."""
+    from paper_2505_05086_b200.binding import ASI_ERR_INVALID_ARG, ASI_ERR_WORKSPACE
+    L = asi.lib()
+    p = asi.Plan("conv", (8, 12, 7, 7), (3, 4, 3, 2), cout=10, k=3, stride=1, pad=1)
+    n = 2
+    h = (C.c_void_p * n)(p.handle.value, p.handle.value)
+    fake = (C.c_void_p * n)(4096, 8192)              # never dereferenced: the calls fail before any launch
+    other = (C.c_void_p * n)(12288, 16384)
+    same_ws = (C.c_void_p * n)(256 * 100, 256 * 100)
+    big = (C.c_size_t * n)(1 << 30, 1 << 30)
+    small = (C.c_size_t * n)(16, 16)
+    assert L.asi_compress_batched(None, fake, fake, other, fake, fake, big, n, None) == ASI_ERR_INVALID_ARG
+    assert L.asi_compress_batched(h, fake, fake, other, fake, fake, big, 0, None) == ASI_ERR_INVALID_ARG
+    assert L.asi_compress_batched(h, fake, fake, fake, fake, fake, big, n, None) == ASI_ERR_INVALID_ARG    # U_new aliases U_prev
+    assert L.asi_compress_batched(h, fake, fake, other, fake, same_ws, big, n, None) == ASI_ERR_INVALID_ARG
+    assert L.asi_compress_batched(h, fake, fake, other, fake, fake, small, n, None) == ASI_ERR_WORKSPACE
+    assert L.asi_wgrad_batched(h, fake, fake, None, fake, fake, big, n, None) == ASI_ERR_INVALID_ARG
+    assert L.asi_wgrad_batched(h, fake, fake, fake, fake, fake, small, n, None) == ASI_ERR_WORKSPACE
