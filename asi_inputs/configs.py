@@ -129,7 +129,15 @@ def get_config(index: int, energy: float = None, bf16: bool = None) -> Config:
              LayerSpec("mlp.fc2(3072->768)", "linear", (32, 197, 3072), 768, ranks=(8, 32, 64)))
         return Config(4, "vit-base-mlp", L, steps=20, bf16=True if bf16 is None else bool(bf16),
                       rho_rule="rank-scaled")
-    raise ValueError("config index 0..4")
+    if index == 5:
+        # LLM-shaped tokens (appendix, TinyLlama experiment: batch 8, up to 512 tokens, 2048-wide, a single
+        # rank of 20): the rank-range rule r_m <= a_m clips the batch mode to 8
+        L = (LayerSpec("attn.proj(2048->2048)", "linear", (8, 512, 2048), 2048, ranks=(8, 20, 20)),
+             LayerSpec("mlp.up(2048->5632)", "linear", (8, 512, 2048), 5632, ranks=(8, 20, 20)),
+             LayerSpec("mlp.down(5632->2048)", "linear", (8, 512, 5632), 2048, ranks=(8, 20, 20)))
+        return Config(5, "llm-tokens", L, steps=20, bf16=True if bf16 is None else bool(bf16),
+                      rho_rule="rank-scaled")
+    raise ValueError("config index 0..5")
 
 
 def layer_seed(cfg_index: int, layer_index: int) -> int:

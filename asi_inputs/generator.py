@@ -132,6 +132,20 @@ class LayerStream:
         """fp32 previous-step factors handed to step 0."""
         return [u.astype(np.float32) for u in self._U_prev0]
 
+    def skip(self, n: int):
+        """Advances the stream by n steps without building the tensors: only the drift of the generating
+        factors is replayed (each step seeds its own generator, so nothing else carries over)."""
+        for _ in range(int(n)):
+            rng = np.random.default_rng(self.seed + 1 + self._step)
+            if self._step > 0:
+                self._Ustar = [_rotate(u, rng, self.theta) for u in self._Ustar]
+            self._step += 1
+
+    def u_prev_now(self):
+        """fp32 previous-step factors for the NEXT step: the leading generating columns as they stand,
+        i.e. one drift step before the tensor that next() returns (the rule u_prev0() follows at step 0)."""
+        return [np.ascontiguousarray(u[:, :r]).astype(np.float32) for u, r in zip(self._Ustar, self.ranks)]
+
     def next(self):
         """Returns (A, dY) of the next training step as float32 arrays
         (bf16-representable when ``bf16``); generating factors drift first for

@@ -43,7 +43,7 @@ extern "C" {
 typedef enum {
   ASI_OK = 0,
   ASI_ERR_INVALID_ARG = 1,    /* null pointer, bad enum, non-positive size, aliasing */
-  ASI_ERR_UNSUPPORTED = 2,    /* dilation != 1, rank > 64, ndim out of range */
+  ASI_ERR_UNSUPPORTED = 2,    /* dilation != 1, rank > 128, ndim out of range */
   ASI_ERR_RANK_RANGE = 3,     /* r_m outside [1, min(a_m, b_m)] (Algorithm 1, inputs) */
   ASI_ERR_WORKSPACE = 4,      /* workspace too small or misaligned */
   ASI_ERR_CUDA = 5,           /* a CUDA runtime call failed */
@@ -55,7 +55,7 @@ typedef enum { ASI_F32 = 0, ASI_BF16 = 1 } asi_dtype_t;
 typedef enum { ASI_CONV2D = 0, ASI_LINEAR = 1 } asi_kind_t;
 
 #define ASI_MAX_MODES 4
-#define ASI_MAX_RANK 64
+#define ASI_MAX_RANK 128
 
 /* One trained layer.  conv: ndim = 4, dims = (B,C,H,W).  linear: ndim = 2 or 3,
  * dims = (B[,N],Din), cout = Dout and the conv fields are ignored. */
@@ -64,7 +64,7 @@ typedef struct {
   int32_t in_dtype;              /* asi_dtype_t of act and dY */
   int32_t ndim;
   int64_t dims[ASI_MAX_MODES];
-  int32_t ranks[ASI_MAX_MODES];  /* 1 <= r_m <= min(a_m, b_m), r_m <= 64 */
+  int32_t ranks[ASI_MAX_MODES];  /* 1 <= r_m <= min(a_m, b_m), r_m <= ASI_MAX_RANK */
   int32_t cout;
   int32_t kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, groups;
   int32_t flags;                 /* ASI_FLAG_* bits, 0 for defaults */
@@ -186,6 +186,32 @@ asi_status_t asi_conv_wgrad(const asi_plan_t* plan, const float* core, const flo
  *   dW [out] device fp32 [Dout, Din]. */
 asi_status_t asi_linear_wgrad(const asi_plan_t* plan, const float* core, const float* U,
                               const void* dY, float* dW, void* ws, size_t ws_bytes, void* stream);
+
+/* Rank selection aids (run once per layer before training, not per step).
+ *
+ * asi_mode_spectrum: for every mode m the leading eigenvalues of A_m A_m^T -- the squared singular values
+ * of the mode-m unfolding, whose partial sums are the "explained variance" HOSVD_eps truncates by
+ * (Sec. 3.2) -- in descending order, and the mode's total energy trace(A_m A_m^T) = ||A||_F^2.
+ *   eig     [out] device fp64 [ndim][ASI_SPECTRUM_MAX], zero-padded; for a_m <= ASI_SPECTRUM_MAX the whole
+ *           spectrum (Jacobi), otherwise the ASI_SPECTRUM_MAX leading Ritz values of a block subspace
+ *           iteration on A_m A_m^T (the leading ones converged to fp64 accuracy, the trailing ones lower
+ *           bounds)
+ *   energy  [out] device fp64 [ndim]
+ *   ws      device scratch of at least asi_spectrum_ws_bytes(plan), 256-byte aligned
+ * asi_pick_ranks: the HOSVD_eps rule on those numbers: r_m = the smallest r whose leading eigenvalues
+ * hold a fraction >= eps of the mode's energy, clipped to [1, min(r_max, a_m, b_m)] (Algorithm 1, rank
+ * range);  ranks [out] device int32 [ndim].
+ * asi_perplexity: the activation perplexity of Sec. 3.3 for one layer, ||dW - dW_approx||_F over n fp32
+ * values;  out [out] device fp64 [1];  ws of at least asi_perplexity_ws_bytes(). */
+#define ASI_SPECTRUM_MAX 128
+size_t asi_spectrum_ws_bytes(const asi_plan_t* plan);
+asi_status_t asi_mode_spectrum(const asi_plan_t* plan, const void* act, double* eig, double* energy, void* ws,
+                               size_t ws_bytes, void* stream);
+asi_status_t asi_pick_ranks(const asi_plan_t* plan, const double* eig, const double* energy, double eps,
+                            int32_t r_max, int32_t* ranks, void* stream);
+size_t asi_perplexity_ws_bytes(void);
+asi_status_t asi_perplexity(const float* dW, const float* dW_approx, int64_t n, double* out, void* ws,
+                            size_t ws_bytes, void* stream);
 
 /* One whole layer-step from HOST buffers (pinned memory recommended): copies
  * act, dY and U_prev to the caller's device arena, runs asi_compress and the

@@ -31,6 +31,7 @@ ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT = 1, 2
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
     "asi_init_factors", "asi_compress_batched", "asi_wgrad_batched",
+    "asi_spectrum_ws_bytes", "asi_mode_spectrum", "asi_pick_ranks", "asi_perplexity_ws_bytes", "asi_perplexity",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host", "asi_step_host_status",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
     "asi_profile_end", "asi_last_cuda_error",
@@ -85,6 +86,13 @@ def lib():
     L.asi_wgrad_batched.argtypes = [pvp, pvp, pvp, pvp, pvp, pvp, psz, i32, vp]
     L.asi_conv_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_linear_wgrad.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_spectrum_ws_bytes.argtypes = [vp]
+    L.asi_spectrum_ws_bytes.restype = sz
+    L.asi_mode_spectrum.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+    L.asi_pick_ranks.argtypes = [vp, vp, vp, C.c_double, i32, vp, vp]
+    L.asi_perplexity_ws_bytes.argtypes = []
+    L.asi_perplexity_ws_bytes.restype = sz
+    L.asi_perplexity.argtypes = [vp, vp, C.c_int64, vp, vp, sz, vp]
     L.asi_step_host_arena_bytes.argtypes = [vp]
     L.asi_step_host_arena_bytes.restype = sz
     L.asi_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -102,7 +110,8 @@ def lib():
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
                  "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
-                 "asi_poll_status", "asi_step_host_status", "asi_compress_batched", "asi_wgrad_batched"):
+                 "asi_poll_status", "asi_step_host_status", "asi_compress_batched", "asi_wgrad_batched",
+                 "asi_mode_spectrum", "asi_pick_ranks", "asi_perplexity"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -196,6 +205,15 @@ class Plan:
         else:
             self.linear_wgrad(core, U, dY, dW, ws, ws_bytes, stream)
 
+    def spectrum_ws_bytes(self):
+        return lib().asi_spectrum_ws_bytes(self._h)
+
+    def mode_spectrum(self, act, eig, energy, ws, ws_bytes, stream=0):
+        _check(lib().asi_mode_spectrum(self._h, act, eig, energy, ws, ws_bytes, stream), "asi_mode_spectrum")
+
+    def pick_ranks(self, eig, energy, eps, r_max, ranks, stream=0):
+        _check(lib().asi_pick_ranks(self._h, eig, energy, float(eps), int(r_max), ranks, stream), "asi_pick_ranks")
+
     def step_host_arena_bytes(self):
         return lib().asi_step_host_arena_bytes(self._h)
 
@@ -236,6 +254,15 @@ class Batch:
         sizes = (C.c_size_t * self.n)(*[int(v) for v in ws_bytes])
         _check(lib().asi_wgrad_batched(self._h, self._arr(cores), self._arr(U), self._arr(dY), self._arr(dW),
                                        self._arr(ws), sizes, self.n, stream), "asi_wgrad_batched")
+
+
+def perplexity(dW, dW_approx, n, out, ws, ws_bytes, stream=0):
+    """asi_perplexity: ||dW - dW_approx||_F into the device double `out`."""
+    _check(lib().asi_perplexity(dW, dW_approx, int(n), out, ws, ws_bytes, stream), "asi_perplexity")
+
+
+def perplexity_ws_bytes():
+    return lib().asi_perplexity_ws_bytes()
 
 
 KERNEL_IDS = {"modeprod": 1, "expand": 2, "qr": 3, "conv_tail": 4, "sm_pass1": 5, "sm_core": 6,

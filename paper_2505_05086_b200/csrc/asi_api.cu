@@ -1035,6 +1035,35 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
   return ASI_OK;
 }
 
+size_t asi_spectrum_ws_bytes(const asi_plan_t* pl) { return pl ? spectrum_ws_bytes(pl) : 0; }
+
+asi_status_t asi_mode_spectrum(const asi_plan_t* pl, const void* act, double* eig, double* energy, void* ws,
+                               size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(act) || !eig || !energy) return ASI_ERR_INVALID_ARG;
+  const asi_status_t s = check_ws(ws, ws_bytes, spectrum_ws_bytes(pl));
+  if (s != ASI_OK) return s;
+  ASI_CUDA(launch_mode_spectrum(pl, act, eig, energy, static_cast<char*>(ws), static_cast<cudaStream_t>(stream)));
+  return ASI_OK;
+}
+
+asi_status_t asi_pick_ranks(const asi_plan_t* pl, const double* eig, const double* energy, double eps,
+                            int32_t r_max, int32_t* ranks, void* stream) {
+  if (!pl || !eig || !energy || !ranks || !(eps > 0.0) || !(eps <= 1.0) || r_max < 1) return ASI_ERR_INVALID_ARG;
+  ASI_CUDA(launch_pick_ranks(pl, eig, energy, eps, r_max, ranks, static_cast<cudaStream_t>(stream)));
+  return ASI_OK;
+}
+
+size_t asi_perplexity_ws_bytes(void) { return perplexity_ws_bytes(); }
+
+asi_status_t asi_perplexity(const float* dW, const float* dW_approx, int64_t n, double* out, void* ws,
+                            size_t ws_bytes, void* stream) {
+  if (!dW || !dW_approx || !out || n < 1) return ASI_ERR_INVALID_ARG;
+  const asi_status_t s = check_ws(ws, ws_bytes, perplexity_ws_bytes());
+  if (s != ASI_OK) return s;
+  ASI_CUDA(launch_perplexity(dW, dW_approx, n, out, static_cast<double*>(ws), static_cast<cudaStream_t>(stream)));
+  return ASI_OK;
+}
+
 size_t asi_step_host_arena_bytes(const asi_plan_t* pl) {
   if (!pl) return 0;
   const size_t eb = elem_bytes(pl);

@@ -471,7 +471,7 @@ static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
     const cudaError_t e = launch_tc_expand(p, p.tc_scratch, p.tc_scratch_bytes, st);   // tensor cores when it fits
     if (e != cudaErrorNotSupported) return e;
   }
-  if (p.I == 1 && p.r >= 16 && p.a >= 64 && p.Q < (1 << 30) && p.a < (1 << 30)) {
+  if (p.I == 1 && p.r >= 16 && p.r <= 64 && p.a >= 64 && p.Q < (1 << 30) && p.a < (1 << 30)) {
     GemmArgs g = {p.X, p.V, p.Pp, (int)p.a, p.r, (int)p.Q, p.a, (int)p.q_per_split, 0};
     return launch_gemm_t<false, TX>(g, p.nsplit, st);
   }
@@ -482,7 +482,8 @@ static cudaError_t launch_expand_t(const ExpandArgs& p, cudaStream_t st) {
     case 8: k_expand<8, TX><<<grid, 256, 0, st>>>(p); break;
     case 16: k_expand<16, TX><<<grid, 256, 0, st>>>(p); break;
     case 32: k_expand<32, TX><<<grid, 256, 0, st>>>(p); break;
-    default: k_expand<64, TX><<<grid, 256, 0, st>>>(p); break;
+    case 64: k_expand<64, TX><<<grid, 256, 0, st>>>(p); break;
+    default: k_expand<128, TX><<<grid, 256, 0, st>>>(p); break;
   }
   return cudaGetLastError();
 }
@@ -863,10 +864,10 @@ cudaError_t launch_fiber(const FiberArgs& p, int grid, bool x_bf16, cudaStream_t
 __global__ void __launch_bounds__(256) k_qr_gram(QRArgs args) {
   const QRMode M = args.m[blockIdx.y];
   const int c = blockIdx.x;
-  if (c >= M.nchunk) return;
-  __shared__ double Ps[kQRRows * ASI_MAX_RANK];      // this chunk's rows of P, pitch r
+  if (c >= M.nchunk || M.r > kQRMaxRank) return;   // ranks above 64 take the k_qrb_* kernels
+  __shared__ double Ps[kQRRows * kQRMaxRank];      // this chunk's rows of P, pitch r
   constexpr int kPer = 16;
-  static_assert(kQRRows * ASI_MAX_RANK == kPer * 256, "one thread holds 16 elements of a full chunk");
+  static_assert(kQRRows * kQRMaxRank == kPer * 256, "one thread holds 16 elements of a full chunk");
   const int tid = threadIdx.x;
   const int r = M.r;
   const int row0 = c * kQRRows;
@@ -951,7 +952,7 @@ __global__ void __launch_bounds__(256) k_qr_gsum(QRArgs args) {
   const QRMode M = args.m[blockIdx.y];
   const int rr = M.r * M.r;
   const int e = blockIdx.x * 256 + threadIdx.x;
-  if (e >= rr || (e % M.r) < (e / M.r)) return;
+  if (M.r > kQRMaxRank || e >= rr || (e % M.r) < (e / M.r)) return;
   const double* G = M.Gp + e;
   double acc = 0.0;
 #pragma unroll 8
@@ -962,18 +963,18 @@ __global__ void __launch_bounds__(256) k_qr_gsum(QRArgs args) {
 // k_qr_solve keeps the running Schur complement of the Cholesky factorisation and the rows it
 // solves in registers; shared memory carries only what one step hands to the next (the pivot
 // row, the next unknown of each row) and R^T for the row solve.
-constexpr int kQRPitch = ASI_MAX_RANK + 1;
+constexpr int kQRPitch = kQRMaxRank + 1;
 
 __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
-  static_assert(ASI_MAX_RANK == 64 && kQRRows == 64, "4 x 4 slots of stride 16; four threads per row");
+  static_assert(kQRMaxRank == 64 && kQRRows == 64, "4 x 4 slots of stride 16; four threads per row");
   const QRMode M = args.m[blockIdx.y];
   const int c = blockIdx.x;
   const int row0 = c * kQRRows;
-  if (c >= M.nchunk || row0 >= M.a) return;
-  __shared__ double Rt[ASI_MAX_RANK * kQRPitch];      // Rt[k][j] = R[j][k], k > j
-  __shared__ double rowbuf[2][ASI_MAX_RANK];          // pivot row of step j in rowbuf[j & 1]
+  if (c >= M.nchunk || row0 >= M.a || M.r > kQRMaxRank) return;
+  __shared__ double Rt[kQRMaxRank * kQRPitch];      // Rt[k][j] = R[j][k], k > j
+  __shared__ double rowbuf[2][kQRMaxRank];          // pivot row of step j in rowbuf[j & 1]
   __shared__ double pub[2][kQRRows];                  // v_j of each row in pub[j & 1]
-  __shared__ double Rinv[ASI_MAX_RANK];               // 1 / R[j][j]
+  __shared__ double Rinv[kQRMaxRank];               // 1 / R[j][j]
   __shared__ double s_trace;
   const int tid = threadIdx.x;
   const int r = M.r;
@@ -983,16 +984,16 @@ __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
   const int rowl = tid >> 2, ql = tid & 3;
   const int row = row0 + rowl;
   const bool live = row < M.a;                        // rows past the end are solved as zeros, unstored
-  double v[ASI_MAX_RANK / 4];
+  double v[kQRMaxRank / 4];
   {
     const double* prow = M.Pred + (int64_t)(live ? row : 0) * r;
 #pragma unroll
-    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+    for (int t = 0; t < kQRMaxRank / 4; ++t) {
       const int k = ql + 4 * t;
       v[t] = __ldcg(prow + (k < r ? k : 0));         // unconditional, selected afterwards
     }
 #pragma unroll
-    for (int t = 0; t < ASI_MAX_RANK / 4; ++t)
+    for (int t = 0; t < kQRMaxRank / 4; ++t)
       if (!(live && ql + 4 * t < r)) v[t] = 0.0;
   }
   // G = sum of the row chunks' shares, chunk by chunk in order (upper triangle).
@@ -1078,16 +1079,16 @@ __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
   // threads of a row sit in one warp; every lane takes every step (the warp barriers are
   // unconditional), and the thread that owns column j + 1 hands v_{j+1} to the next step.
   for (int j = 0; j < r; ++j) {
-    double rt[ASI_MAX_RANK / 4];
+    double rt[kQRMaxRank / 4];
 #pragma unroll
-    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+    for (int t = 0; t < kQRMaxRank / 4; ++t) {
       const int k = ql + 4 * t;
       rt[t] = (k > j && k < r) ? Rt[k * kQRPitch + j] : 0.0;
     }
     const double q = pub[j & 1][rowl] * Rinv[j];
     double* np = pub[(j + 1) & 1];
 #pragma unroll
-    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+    for (int t = 0; t < kQRMaxRank / 4; ++t) {
       const int k = ql + 4 * t;
       v[t] = (k == j) ? q : fma(-q, rt[t], v[t]);     // rt = 0 leaves the solved and the unused columns alone
       if (k == j + 1 && k < r) np[rowl] = v[t];
@@ -1097,7 +1098,7 @@ __global__ void __launch_bounds__(256) k_qr_solve(QRArgs args) {
   if (live) {
     float* urow = M.Uout + (int64_t)row * r;
 #pragma unroll
-    for (int t = 0; t < ASI_MAX_RANK / 4; ++t) {
+    for (int t = 0; t < kQRMaxRank / 4; ++t) {
       const int k = ql + 4 * t;
       if (k < r) urow[k] = (float)v[t];
     }
@@ -1110,6 +1111,122 @@ cudaError_t launch_qr_solve(const QRArgs& p, int nd, int max_chunks, cudaStream_
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Orthogonalize for ranks 65..128: the same Cholesky-QR in fp64 in plain kernels (these ranks are rare
+// and the matrices small: a x r with r <= 128).  k_qrb_reduce sums the column-split partials in split
+// order, k_qrb_gram forms G = P^T P (one thread per entry of the upper triangle, rows in order),
+// k_qrb_chol factors G = R^T R in one CTA (shared memory), k_qrb_solve solves u R = p one row per thread.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_qrb_reduce(QRArgs args) {
+  const QRMode M = args.m[blockIdx.y];
+  if (M.r <= kQRMaxRank) return;
+  const int64_t n = (int64_t)M.a * M.r;
+  for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < n; e += (int64_t)gridDim.x * 256) {
+    double acc = 0.0;
+    for (int s0 = 0; s0 < M.nsplit; s0 += 8) {
+      float t[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) t[q] = __ldcg(M.Pp + (int64_t)((s0 + q < M.nsplit) ? (s0 + q) : 0) * n + e);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) acc += (s0 + q < M.nsplit) ? (double)t[q] : 0.0;
+    }
+    M.Pred[e] = acc;
+  }
+}
+
+__global__ void __launch_bounds__(256) k_qrb_gram(QRArgs args) {
+  const QRMode M = args.m[blockIdx.y];
+  const int r = M.r;
+  if (r <= kQRMaxRank) return;
+  const int e = blockIdx.x * 256 + threadIdx.x;
+  if (e >= r * r) return;
+  const int i = e / r, j = e - i * r;
+  if (j < i) return;
+  double g = 0.0;
+#pragma unroll 4
+  for (int k = 0; k < M.a; ++k) g = fma(__ldcg(M.Pred + (int64_t)k * r + i), __ldcg(M.Pred + (int64_t)k * r + j), g);
+  M.Gp[e] = g;
+}
+
+__global__ void __launch_bounds__(1024) k_qrb_chol(QRArgs args) {
+  extern __shared__ double qb_G[];                 // [r][r + 1]
+  __shared__ double s_d;
+  const QRMode M = args.m[blockIdx.x];
+  const int r = M.r, tid = threadIdx.x, P = r + 1;
+  if (r <= kQRMaxRank) return;
+  for (int e = tid; e < r * r; e += 1024) {
+    const int i = e / r, j = e - i * r;
+    qb_G[i * P + j] = (j >= i) ? M.Gp[e] : 0.0;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int i = 0; i < r; ++i) t += qb_G[i * P + i];
+    s_d = 1e-12 * t;
+  }
+  __syncthreads();
+  const double floor_d = s_d;
+  for (int j = 0; j < r; ++j) {
+    double d = qb_G[j * P + j];
+    if (!(d > floor_d)) {
+      if (tid == 0) atomicMax(args.status, (int)ASI_ERR_RANK_DEFICIENT);
+      d = (floor_d > 0.0) ? floor_d : 1.0;
+    }
+    const double inv = rsqrt(d);
+    __syncthreads();
+    for (int k = j + tid; k < r; k += 1024) qb_G[j * P + k] = (k == j) ? d * inv : qb_G[j * P + k] * inv;
+    __syncthreads();
+    const int nrem = r - j - 1;
+    for (int e = tid; e < nrem * nrem; e += 1024) {
+      const int i = j + 1 + e / nrem, k = j + 1 + e % nrem;
+      if (k >= i) qb_G[i * P + k] -= qb_G[j * P + i] * qb_G[j * P + k];
+    }
+    __syncthreads();
+  }
+  for (int e = tid; e < r * r; e += 1024) {
+    const int i = e / r, j = e - i * r;
+    M.Gp[e] = (j >= i) ? qb_G[i * P + j] : 0.0;    // R, upper triangular
+  }
+}
+
+__global__ void __launch_bounds__(128) k_qrb_solve(QRArgs args) {
+  extern __shared__ double qb_R[];                 // [r][r]
+  const QRMode M = args.m[blockIdx.y];
+  const int r = M.r;
+  if (r <= kQRMaxRank) return;
+  for (int e = threadIdx.x; e < r * r; e += 128) qb_R[e] = M.Gp[e];
+  __syncthreads();
+  const int row = blockIdx.x * 128 + threadIdx.x;
+  if (row >= M.a) return;
+  double u[2 * kQRMaxRank];
+  const double* prow = M.Pred + (int64_t)row * r;
+  for (int j = 0; j < r; ++j) {
+    double s = prow[j];
+    for (int i = 0; i < j; ++i) s = fma(-u[i], qb_R[i * r + j], s);
+    u[j] = s / qb_R[j * r + j];
+  }
+  float* urow = M.Uout + (int64_t)row * r;
+  for (int j = 0; j < r; ++j) urow[j] = (float)u[j];
+}
+
+static cudaError_t launch_qr_big(const QRArgs& p, int nd, cudaStream_t st) {
+  int amax = 1, rmax = 1;
+  for (int m = 0; m < nd; ++m)
+    if (p.m[m].r > kQRMaxRank) {
+      amax = std::max(amax, p.m[m].a);
+      rmax = std::max(rmax, p.m[m].r);
+    }
+  k_qrb_reduce<<<dim3(64, (unsigned)nd), 256, 0, st>>>(p);
+  k_qrb_gram<<<dim3((unsigned)((rmax * rmax + 255) / 256), (unsigned)nd), 256, 0, st>>>(p);
+  const size_t chol_smem = (size_t)rmax * (rmax + 1) * sizeof(double), solve_smem = (size_t)rmax * rmax * sizeof(double);
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_qrb_chol), chol_smem);
+  if (e == cudaSuccess) e = opt_in_smem(reinterpret_cast<const void*>(k_qrb_solve), solve_smem);
+  if (e != cudaSuccess) return e;
+  k_qrb_chol<<<nd, 1024, chol_smem, st>>>(p);
+  k_qrb_solve<<<dim3((unsigned)((amax + 127) / 128), (unsigned)nd), 128, solve_smem, st>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) {
   double qr_bytes = 0.0;
   for (int m = 0; m < nd; ++m)
@@ -1119,13 +1236,17 @@ cudaError_t launch_qr(const QRArgs& p, int nd, int max_chunks, cudaStream_t st) 
   k_qr_gram<<<grid, 256, 0, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k_qr_gsum<<<dim3(ASI_MAX_RANK * ASI_MAX_RANK / 256, (unsigned)nd), 256, 0, st>>>(p);
+  k_qr_gsum<<<dim3(kQRMaxRank * kQRMaxRank / 256, (unsigned)nd), 256, 0, st>>>(p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   QRArgs q = p;
   q.gsum = 1;
   k_qr_solve<<<grid, 256, 0, st>>>(q);
-  return cudaGetLastError();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  for (int m = 0; m < nd; ++m)
+    if (p.m[m].r > kQRMaxRank) return launch_qr_big(p, nd, st);
+  return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------------------------

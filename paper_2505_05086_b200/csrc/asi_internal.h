@@ -7,6 +7,8 @@
 
 #include "asi.h"
 
+struct asi_plan;
+
 namespace asi {
 
 // Mode-m view of a contiguous tensor: element (o, k, i) at o*a*I + k*I + i.
@@ -20,6 +22,7 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 constexpr int kStatusBytes = 1024;    // status word (int 0), completion counters (ints 16..255)
 constexpr int kQRRows = 64;          // rows per CTA in the orthonormalisation kernels
+constexpr int kQRMaxRank = 64;       // ranks the register-resident Cholesky-QR kernels cover (above: k_qrb_*)
 constexpr int kExpandKC = 32;        // rows of P per CTA in the expand kernel
 
 // Y(o, j, i) = sum_k X(o, k, i) * B(k, j): the small-mode contraction that serves the
@@ -253,6 +256,17 @@ cudaError_t launch_conv_tail(const ConvTailArgs& p, cudaStream_t st);
 cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, cudaStream_t st);
 
 
+}  // namespace asi
+
+namespace asi {
+// rank selection aids (asi_spectrum_kernels.cu)
+size_t spectrum_ws_bytes(const struct ::asi_plan* pl);
+cudaError_t launch_mode_spectrum(const struct ::asi_plan* pl, const void* act, double* eig, double* energy, char* w,
+                                 cudaStream_t st);
+cudaError_t launch_pick_ranks(const struct ::asi_plan* pl, const double* eig, const double* energy, double eps,
+                              int r_max, int* ranks, cudaStream_t st);
+size_t perplexity_ws_bytes();
+cudaError_t launch_perplexity(const float* x, const float* y, int64_t n, double* out, double* part, cudaStream_t st);
 }  // namespace asi
 
 struct asi_plan {

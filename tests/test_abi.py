@@ -91,7 +91,7 @@ def test_bf16_plans_pick_the_tensor_core_products_by_shape(asi, dims, ranks, on_
     (dict(dims=(8, 32, 16, 16), ranks=(9, 8, 8, 8)), 3),            # r_1 > a_1
     (dict(dims=(8, 32, 16, 16), ranks=(0, 8, 8, 8)), 3),
     (dict(dims=(200, 2, 2, 2), ranks=(9, 1, 1, 1)), 3),            # r_1 > b_1 = 8
-    (dict(dims=(128, 128, 8, 8), ranks=(65, 8, 8, 8)), 2),         # rank above the supported 64
+    (dict(dims=(256, 256, 8, 8), ranks=(129, 8, 8, 8)), 2),        # rank above the supported 128
     (dict(dims=(8, 32, 16, 16), ranks=(4, 8, 8, 8), dilation=2), 2),
     (dict(dims=(8, 32, 16, 16), ranks=(4, 8, 8, 8), groups=3), 1),
     (dict(dims=(8, 32, 16, 16), ranks=(4, 8, 8, 8), k=0), 1),

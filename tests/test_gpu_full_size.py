@@ -20,6 +20,39 @@ def _layer_steps(cfg, li, steps, tol, generic_only=False):
         check(err, tol, f"{cfg.name}/{L.name}/step{t}: {err}")
 
 
+def _first_steps_and_last(cfg, li, tol, first=3):
+    """Steps 0..first-1 teacher-forced on the oracle's factors, then the last step of the configuration's
+    stream: the generator is advanced without building tensors, and the step starts from the generating
+    factors one drift step back (the rule step 0 follows)."""
+    L = cfg.layers[li]
+    st = make_stream(cfg, li)
+    run = make_runner(L, bf16=cfg.bf16)
+    U_prev = st.u_prev0()
+    for t in range(first):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, tol, f"{cfg.name}/{L.name}/step{t}: {err}")
+    st.skip(cfg.steps - 1 - first)
+    U_prev = st.u_prev_now()
+    A, dY = st.next()
+    err, _ = compare_step(run, L, A, dY, U_prev)
+    check(err, tol, f"{cfg.name}/{L.name}/step{cfg.steps - 1}: {err}")
+
+
+@pytest.mark.parametrize("li", range(10))
+@pytest.mark.parametrize("bf16", [False, True])
+def test_config4_resnet34_sweep_at_the_benchmark_ranks(li, bf16):
+    """Every shape of the sweep at the 90 % ranks bench.py uses, default kernels, fp32 and bf16 inputs:
+    steps 0-2 and step 19 of the 20-step stream."""
+    _first_steps_and_last(get_config(3, energy=0.9, bf16=bf16), li, TOL_BF16 if bf16 else TOL_F32)
+
+
+@pytest.mark.parametrize("ci,li", [(1, 0), (1, 1), (2, 0), (2, 2), (2, 4), (4, 0), (4, 1), (5, 0), (5, 2)])
+def test_last_step_of_the_other_streams(ci, li):
+    cfg = get_config(ci)
+    _first_steps_and_last(cfg, li, TOL_BF16 if cfg.bf16 else TOL_F32, first=1)
+
+
 @pytest.mark.parametrize("generic_only", [False, True])
 @pytest.mark.parametrize("li", [0, 1, 2, 3])
 def test_config2_resnet18_last4(li, generic_only):
@@ -51,3 +84,8 @@ def test_config4_resnet34_shapes_bf16(li):
 @pytest.mark.parametrize("li", [0, 1])
 def test_config5_vit_mlp_bf16(li):
     _layer_steps(get_config(4), li, 2, TOL_BF16)
+
+
+@pytest.mark.parametrize("li", [0, 1, 2])
+def test_config6_llm_tokens_bf16(li):
+    _layer_steps(get_config(5), li, 2, TOL_BF16)

@@ -170,6 +170,21 @@ def test_bf16_linear_layers_on_tensor_cores(dims, ranks, cout, rho, gen):
         assert run.ok()
 
 
+def test_ranks_above_64_take_the_plain_orthogonalize_kernels():
+    """Ranks 65..128 (here 96 in the feature mode and 72 in the token mode) run through the generic
+    contraction kernels and the plain fp64 Cholesky-QR; spectra are kept flat enough for fp32."""
+    dims, ranks = (4, 150, 200), (3, 72, 96)
+    L = LayerSpec("t", "linear", dims, 24, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=61, rho=(0.6, 0.985, 0.99),
+                     gen_ranks=(4, 144, 192))
+    run = make_runner(L)
+    U_prev = st.u_prev0()
+    for t in range(2):
+        A, dY = st.next()
+        err, U_prev = compare_step(run, L, A, dY, U_prev)
+        check(err, TOL_F32, f"ranks {ranks} step {t}")
+
+
 def test_bf16_input_mode_small():
     dims, ranks = (6, 20, 9, 9), (3, 4, 3, 3)
     L = LayerSpec("t", "conv", dims, 10, 3, 1, 1, 1, ranks=ranks)

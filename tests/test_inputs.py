@@ -54,3 +54,23 @@ def test_bf16_rounding_is_nearest_even():
     x = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 2 ** -7, 1.0 + 3 * 2 ** -8, -2.5], dtype=np.float32)
     np.testing.assert_array_equal(round_to_bf16(x),
                                   np.array([1.0, 1.0, 1.0 + 2 ** -7, 1.0 + 2 ** -6, -2.5], np.float32))
+
+
+def test_skip_replays_the_drift_exactly():
+    from asi_inputs.generator import LayerStream
+    kw = dict(dims=(4, 6, 5, 5), ranks=(2, 3, 2, 2), dy_shape=(4, 3, 5, 5), seed=77)
+    a, b = LayerStream(**kw), LayerStream(**kw)
+    for _ in range(5):
+        a.next()
+    b.skip(5)
+    A1, d1 = a.next()
+    A2, d2 = b.next()
+    np.testing.assert_array_equal(A1, A2)
+    np.testing.assert_array_equal(d1, d2)
+    # the previous-step factors offered before a step span (nearly) the subspace that step will find
+    c = LayerStream(**kw)
+    c.skip(3)
+    U = c.u_prev_now()
+    assert [u.shape for u in U] == [(4, 2), (6, 3), (5, 2), (5, 2)]
+    for u in U:
+        assert np.allclose(u.T @ u, np.eye(u.shape[1]), atol=1e-5)
