@@ -4,7 +4,7 @@
 // plain and exact-minded (fp64 accumulation, fixed summation orders), not tuned.
 //
 //   k_gram / k_gram_sum : G_m = A_m A_m^T (a_m x a_m, fp64): 32 x 32 output blocks, the contraction split
-//                         over CTAs, fp32 products summed 32 at a time into fp64, the splits added in order
+//                         over CTAs, products and sums in fp64, the splits added in order
 //   k_sub_* (a_m > 128) : block subspace iteration on G_m with 128 vectors -- Y = G X, Gram-Schmidt twice
 //                         per column (one CTA), ten rounds -- then H = X^T G X, whose eigenvalues are the
 //                         leading Ritz values of G_m
@@ -61,17 +61,12 @@ __global__ void __launch_bounds__(256) k_gram(const TX* __restrict__ X, int64_t 
       Bs[kl][ql] = (qok && (int64_t)bj * 32 + kl < a) ? vb[t] : 0.f;
     }
     __syncthreads();
-    float p[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll 8
-    for (int ql = 0; ql < 32; ++ql) {
-      const float a0 = As[ty][ql], a1 = As[ty + 16][ql], b0 = Bs[tx][ql], b1 = Bs[tx + 16][ql];
-      p[0][0] = fmaf(a0, b0, p[0][0]); p[0][1] = fmaf(a0, b1, p[0][1]);
-      p[1][0] = fmaf(a1, b0, p[1][0]); p[1][1] = fmaf(a1, b1, p[1][1]);
+    for (int ql = 0; ql < 32; ++ql) {                 // fp64 products: the small eigenvalues need them
+      const double a0 = As[ty][ql], a1 = As[ty + 16][ql], b0 = Bs[tx][ql], b1 = Bs[tx + 16][ql];
+      acc[0][0] = fma(a0, b0, acc[0][0]); acc[0][1] = fma(a0, b1, acc[0][1]);
+      acc[1][0] = fma(a1, b0, acc[1][0]); acc[1][1] = fma(a1, b1, acc[1][1]);
     }
-#pragma unroll
-    for (int x = 0; x < 2; ++x)
-#pragma unroll
-      for (int y = 0; y < 2; ++y) acc[x][y] += (double)p[x][y];
     __syncthreads();
   }
   double* G = Gp + (int64_t)blockIdx.z * a * a;
