@@ -94,11 +94,11 @@ def layer_costs(L, bf16):
             if m + 1 < len(lead_dims):
                 rest /= lead_dims[m + 1]
         wg += lead * r[-1] * L.cout + r[-1] * L.cout * Din
-    # contractions the library runs on the tensor cores: bf16 token layers, factor width 16..64 (x16)
+    # contractions the library runs on the tensor cores: bf16 token layers, factor width 16..64 (a multiple of 4)
     tc = 0.0
     if bf16 and L.kind == "linear":
         for m, rm in enumerate(r):
-            if rm % 16 == 0 and 16 <= rm <= 64 and m >= 1:
+            if rm % 4 == 0 and 16 <= rm <= 64 and m >= 1:
                 tc += macs_modes[m]
     return {"act_bytes": N * eb, "dy_bytes": dy * eb, "dw_bytes": dw * 4,
             "flops": 2.0 * (sum(macs_modes) + core + wg), "flops_tensor": 2.0 * tc}

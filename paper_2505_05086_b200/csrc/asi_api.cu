@@ -164,7 +164,7 @@ void layout_compress(asi_plan* pl) {
   if (pl->bf16 && !pl->fast_compress)
     for (int m = 0; m < pl->nd; ++m) {
       const ModeView& v = pl->mv[m];
-      if (pl->r[m] % 16 != 0 || pl->r[m] < 16 || pl->r[m] > 64) continue;
+      if (pl->r[m] % 4 != 0 || pl->r[m] < 16 || pl->r[m] > 64) continue;   // factor zero-padded to 16 x
       const bool last = v.I == 1 && v.a % 64 == 0 && v.Q >= 128;
       const bool inner = v.I >= 64 && v.I % 64 == 0 && v.O < 65536;
       if (!last && !inner) continue;

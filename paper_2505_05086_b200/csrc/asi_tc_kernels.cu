@@ -136,17 +136,18 @@ struct TcArgs {
   int64_t y_split;
   int inner;           // kTcTokenExpand: K enumerates (o, i) with i < inner (a multiple of 64)
   int* status;         // status word of the caller's workspace (may be null): ASI_ERR_TIMEOUT when a wait expires
+  int nv;              // columns of Y that exist (a multiple of 4, N - 15 <= nv <= N): the factor is zero-padded to N
 };
 
 // Bt[(t*n + j) * ldb + k] = t-th bf16 term of U[k][j] (hi, mid, lo: U = hi + mid + lo to 24 bits)
-__global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, int ldu, int K, int N,
+__global__ void __launch_bounds__(256) k_tc_split(const float* __restrict__ U, int ldu, int K, int N, int nv,
                                                   __nv_bfloat16* __restrict__ Bt, int64_t ldb) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   for (int r = ty; r < 32; r += 8) {
     const int k = k0 + r, j = j0 + tx;
-    tile[r][tx] = (k < K && j < N) ? U[(int64_t)k * ldu + j] : 0.f;
+    tile[r][tx] = (k < K && j < nv) ? U[(int64_t)k * ldu + j] : 0.f;     // columns nv..N-1 of the operand are zero
   }
   __syncthreads();
   for (int r = ty; r < 32; r += 8) {
@@ -285,8 +286,8 @@ __device__ __forceinline__ void tc_gemm_body(const CUtensorMap& mapX, const CUte
           for (int i = 0; i < 8; ++i)                   // small terms first
             o[i] = (__uint_as_float(l[i]) + __uint_as_float(m[i])) + __uint_as_float(h[i]);
           float* y = Yout + (int64_t)row * p.ldy + col0 + cc;
-          *reinterpret_cast<float4*>(y) = make_float4(o[0], o[1], o[2], o[3]);
-          *reinterpret_cast<float4*>(y + 4) = make_float4(o[4], o[5], o[6], o[7]);
+          if (col0 + cc < p.nv) *reinterpret_cast<float4*>(y) = make_float4(o[0], o[1], o[2], o[3]);
+          if (col0 + cc + 4 < p.nv) *reinterpret_cast<float4*>(y + 4) = make_float4(o[4], o[5], o[6], o[7]);
         }
       }
     }
@@ -335,7 +336,7 @@ EncodeFn encode_fn() {
 
 }  // namespace
 
-size_t tc_scratch_bytes(int64_t K, int N) { return (size_t)3 * N * ((K + 63) / 64 * 64) * 2; }
+size_t tc_scratch_bytes(int64_t K, int N) { return (size_t)3 * ((N + 15) / 16 * 16) * ((K + 63) / 64 * 64) * 2; }
 
 namespace {
 constexpr size_t kTcSmem = 1024 + kTcStages * (kTileA + kTileB) + (2 * kTcStages + 1) * 8 + 16;
@@ -352,10 +353,10 @@ bool encode_bf16_map(CUtensorMap* map, const void* base, int rank, const cuuint6
 
 // V[o][i][j] = sum_k X[o][k][i] U[k][j]: a middle mode of a bf16 token tensor (I = inner extent, a multiple of 64)
 cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
-  const int N = p.n_out;
+  const int nv = p.n_out, N = (nv + 15) / 16 * 16;       // the factor is zero-padded to a multiple of 16 columns
   const int64_t Kp = (p.a + 63) / 64 * 64;
-  if (p.I < 64 || p.I % 64 != 0 || p.O < 1 || p.O >= 65536 || N % 16 != 0 || N < 16 || N > kTcNMax || p.a < 1 ||
-      p.a >= (1ll << 31) || p.I >= (1ll << 31) || p.sj != 1 || p.si != N || p.so != p.I * N || p.ldb_j != 1 ||
+  if (p.I < 64 || p.I % 64 != 0 || p.O < 1 || p.O >= 65536 || nv % 4 != 0 || nv < 16 || N > kTcNMax || p.a < 1 ||
+      p.a >= (1ll << 31) || p.I >= (1ll << 31) || p.sj != 1 || p.si != nv || p.so != p.I * nv || p.ldb_j != 1 ||
       !scratch || scratch_bytes < tc_scratch_bytes(p.a, N) || (reinterpret_cast<uintptr_t>(scratch) & 15u) ||
       (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u))
     return cudaErrorNotSupported;
@@ -375,8 +376,8 @@ cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch
   const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_token), kTcSmem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((p.a + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      p.B, (int)p.ldb_k, (int)p.a, N, static_cast<__nv_bfloat16*>(scratch), Kp);
-  TcArgs a = {p.Y, (int)p.I, N, (int)p.a, N, (int)Kp, p.so, 0, p.status};
+      p.B, (int)p.ldb_k, (int)p.a, N, nv, static_cast<__nv_bfloat16*>(scratch), Kp);
+  TcArgs a = {p.Y, (int)p.I, N, (int)p.a, nv, (int)Kp, p.so, 0, p.status, nv};
   dim3 grid((unsigned)((p.I + kTcM - 1) / kTcM), (unsigned)p.O);
   k_tc_token<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -384,9 +385,9 @@ cudaError_t launch_tc_token(const ModeProdArgs& p, void* scratch, size_t scratch
 
 // Pp[s][k][j] = sum_{(o,i) in split s} X[o][k][i] V[o][i][j]: the expansion of a middle mode
 cudaError_t launch_tc_token_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st) {
-  const int N = e.r;
+  const int nv = e.r, N = (nv + 15) / 16 * 16;
   const int64_t Q = e.Q;
-  if (e.I < 64 || e.I % 64 != 0 || e.O < 1 || e.O >= 65536 || N % 16 != 0 || N < 16 || N > kTcNMax || e.a < 1 ||
+  if (e.I < 64 || e.I % 64 != 0 || e.O < 1 || e.O >= 65536 || nv % 4 != 0 || nv < 16 || N > kTcNMax || e.a < 1 ||
       e.a >= (1ll << 31) || Q >= (1ll << 31) || e.q_per_split % kTcKC != 0 || e.q_per_split >= (1ll << 31) ||
       e.nsplit < 1 || !scratch || scratch_bytes < tc_scratch_bytes(Q, N) ||
       (reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(e.X) & 15u) ||
@@ -408,8 +409,8 @@ cudaError_t launch_tc_token_expand(const ExpandArgs& e, void* scratch, size_t sc
   const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_token_expand), kTcSmem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
-  TcArgs a = {e.Pp, (int)e.a, N, (int)Q, N, (int)e.q_per_split, e.a * N, (int)e.I, e.status};
+      e.V, nv, (int)Q, N, nv, static_cast<__nv_bfloat16*>(scratch), Q);
+  TcArgs a = {e.Pp, (int)e.a, N, (int)Q, nv, (int)e.q_per_split, e.a * nv, (int)e.I, e.status, nv};
   dim3 grid((unsigned)((e.a + kTcM - 1) / kTcM), (unsigned)e.nsplit);
   k_tc_token_expand<<<grid, kTcThreads, kTcSmem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -423,8 +424,8 @@ cudaError_t launch_tc_token_expand(const ExpandArgs& e, void* scratch, size_t sc
 cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scratch_bytes, cudaStream_t st) {
   if (p.I != 1) return launch_tc_token(p, scratch, scratch_bytes, st);
   const int64_t M = p.Q, K = p.a;
-  const int N = p.n_out;
-  if (p.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || K % kTcKC != 0 || K < kTcKC || M < kTcM ||
+  const int nv = p.n_out, N = (nv + 15) / 16 * 16;
+  if (p.I != 1 || nv % 4 != 0 || nv < 16 || N > kTcNMax || K % kTcKC != 0 || K < kTcKC || M < kTcM ||
       M >= (1ll << 31) || K >= (1ll << 31) || p.sj != 1 || p.so % 4 != 0 || p.ldb_j != 1 || !scratch ||
       scratch_bytes < tc_scratch_bytes(K, N) || (reinterpret_cast<uintptr_t>(scratch) & 15u) ||
       (reinterpret_cast<uintptr_t>(p.X) & 15u) || (reinterpret_cast<uintptr_t>(p.Y) & 15u))
@@ -455,8 +456,8 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
   const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_lastmode), smem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      p.B, (int)p.ldb_k, (int)K, N, static_cast<__nv_bfloat16*>(scratch), K);
-  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0, 0, p.status};
+      p.B, (int)p.ldb_k, (int)K, N, nv, static_cast<__nv_bfloat16*>(scratch), K);
+  TcArgs a = {p.Y, (int)M, N, (int)K, (int)p.so, (int)K, 0, 0, p.status, nv};
   const unsigned grid = (unsigned)((M + kTcM - 1) / kTcM);
   k_tc_lastmode<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();
@@ -467,8 +468,8 @@ cudaError_t launch_tc_lastmode(const ModeProdArgs& p, void* scratch, size_t scra
 cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_bytes, cudaStream_t st) {
   if (e.I != 1) return launch_tc_token_expand(e, scratch, scratch_bytes, st);
   const int64_t Q = e.Q, A = e.a;
-  const int N = e.r;
-  if (e.I != 1 || N % 16 != 0 || N < 16 || N > kTcNMax || A % 8 != 0 || A < kTcM || Q % 8 != 0 || Q < kTcKC ||
+  const int nv = e.r, N = (nv + 15) / 16 * 16;
+  if (e.I != 1 || nv % 4 != 0 || nv < 16 || N > kTcNMax || A % 8 != 0 || A < kTcM || Q % 8 != 0 || Q < kTcKC ||
       Q >= (1ll << 31) || A >= (1ll << 31) || e.q_per_split % kTcKC != 0 || e.q_per_split >= (1ll << 31) ||
       e.nsplit < 1 || !scratch || scratch_bytes < tc_scratch_bytes(Q, N) ||
       (reinterpret_cast<uintptr_t>(scratch) & 15u) || (reinterpret_cast<uintptr_t>(e.X) & 15u) ||
@@ -500,8 +501,8 @@ cudaError_t launch_tc_expand(const ExpandArgs& e, void* scratch, size_t scratch_
   const cudaError_t attr_err = opt_in_smem(reinterpret_cast<const void*>(k_tc_expand), smem);
   if (attr_err != cudaSuccess) return attr_err;
   k_tc_split<<<dim3((unsigned)((Q + 31) / 32), (unsigned)((N + 31) / 32)), 256, 0, st>>>(
-      e.V, N, (int)Q, N, static_cast<__nv_bfloat16*>(scratch), Q);
-  TcArgs a = {e.Pp, (int)A, N, (int)Q, N, (int)e.q_per_split, A * N, 0, e.status};
+      e.V, nv, (int)Q, N, nv, static_cast<__nv_bfloat16*>(scratch), Q);
+  TcArgs a = {e.Pp, (int)A, N, (int)Q, nv, (int)e.q_per_split, A * nv, 0, e.status, nv};
   dim3 grid((unsigned)((A + kTcM - 1) / kTcM), (unsigned)e.nsplit);
   k_tc_expand<<<grid, kTcThreads, smem, st>>>(mapX, mapB, a);
   return cudaGetLastError();

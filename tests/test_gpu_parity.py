@@ -149,6 +149,8 @@ LINEAR_TC = [  # (dims, ranks, cout, rho, generating ranks)
     ((4, 48, 192), (3, 6, 32), 24, (0.6, 0.8, 0.96), (4, 12, 64)),      # expansion tile with 64 valid rows
     ((4, 72, 128), (3, 16, 16), 24, (0.6, 0.93, 0.93), (4, 32, 32)),    # token mode on the tensor cores too
     ((2, 197, 192), (2, 32, 32), 40, (0.5, 0.96, 0.96), (2, 64, 64)),   # 197 tokens: ragged K chunks and row tiles
+    ((4, 72, 128), (3, 20, 24), 24, (0.6, 0.94, 0.95), (4, 40, 48)),    # ranks 20 / 24: factors zero-padded to 32 columns
+    ((3, 128, 256), (3, 20, 36), 32, (0.6, 0.94, 0.965), (3, 40, 72)),  # rank 36 padded to 48
 ]
 
 
