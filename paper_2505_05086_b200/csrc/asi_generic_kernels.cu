@@ -317,16 +317,20 @@ __global__ void __launch_bounds__(256) k_rowstream(ModeProdArgs p) {
   const int k1 = (k0 + kper < a) ? k0 + kper : a;
   if (live) {
     const TX* X = reinterpret_cast<const TX*>(p.X) + q;
-    for (; k0 + UNR <= k1; k0 += UNR) {
+    // batches of UNR rows, all loads of a batch issued before any is used; rows past the end of the
+    // slice are read from the slice's last row and contribute zero
+    for (; k0 < k1; k0 += UNR) {
       float4 x[UNR];
 #pragma unroll
-      for (int u = 0; u < UNR; ++u) x[u] = ld4_stream<TX>(X + (int64_t)(k0 + u) * p.Q);
+      for (int u = 0; u < UNR; ++u) x[u] = ld4_stream<TX>(X + (int64_t)((k0 + u < k1) ? (k0 + u) : (k1 - 1)) * p.Q);
 #pragma unroll
       for (int u = 0; u < UNR; ++u) {
-        const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+        const bool on = k0 + u < k1;
+        const float xs[4] = {on ? x[u].x : 0.f, on ? x[u].y : 0.f, on ? x[u].z : 0.f, on ? x[u].w : 0.f};
+        const int kr = on ? (k0 + u) : (k1 - 1);
 #pragma unroll
         for (int j = 0; j < R; j += 4) {
-          const float4 b = *reinterpret_cast<const float4*>(Bsm + (k0 + u) * R + j);
+          const float4 b = *reinterpret_cast<const float4*>(Bsm + kr * R + j);
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             acc[c][j] = fmaf(xs[c], b.x, acc[c][j]);
@@ -335,16 +339,6 @@ __global__ void __launch_bounds__(256) k_rowstream(ModeProdArgs p) {
             acc[c][j + 3] = fmaf(xs[c], b.w, acc[c][j + 3]);
           }
         }
-      }
-    }
-    for (; k0 < k1; ++k0) {
-      const float4 xv = ld4_stream<TX>(X + (int64_t)k0 * p.Q);
-      const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-      for (int j = 0; j < R; ++j) {
-        const float b = Bsm[k0 * R + j];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[c][j] = fmaf(xs[c], b, acc[c][j]);
       }
     }
   }

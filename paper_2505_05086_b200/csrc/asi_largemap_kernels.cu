@@ -89,7 +89,7 @@ constexpr int kF2Threads = 256, kF2Groups = 16, kF2TQ = 64;   // 16 half-warps: 
 // further tiles in flight (16-byte cp.async), which is what keeps HBM busy: one 32 KB tile per SM in flight
 // is far below latency x bandwidth.
 // ---------------------------------------------------------------------------------------------
-template <int RW, typename TX>
+template <int RW, int NJ, typename TX>
 __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   constexpr int TQ = kF2TQ, NT = kF2Threads, NG = kF2Groups;
   constexpr int EPU = 16 / (int)sizeof(TX);          // elements per 16-byte unit
@@ -99,11 +99,11 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   const int a = p.a, r = p.r, nst = p.nstage;
   const size_t stage_bytes = (size_t)a * TQ * sizeof(TX);
   unsigned char* stages = f2_smem;
-  f2* Ud = reinterpret_cast<f2*>(f2_smem + (size_t)nst * stage_bytes);   // [NG RW][4]: (u, u)
-  float* Vp = reinterpret_cast<float*>(Ud + (size_t)NG * RW * 4);        // [NG / 2][4][TQ]
-  float* Vt = Vp + (NG / 2) * 4 * TQ;                                    // [4][TQ]
-  for (int idx = tid; idx < NG * RW * 4; idx += NT) {
-    const int k = idx >> 2, j = idx & 3;
+  f2* Ud = reinterpret_cast<f2*>(f2_smem + (size_t)nst * stage_bytes);   // [NG RW][NJ]: (u, u)
+  float* Vp = reinterpret_cast<float*>(Ud + (size_t)NG * RW * NJ);       // [NG / 2][NJ][TQ]
+  float* Vt = Vp + (NG / 2) * NJ * TQ;                                   // [NJ][TQ]
+  for (int idx = tid; idx < NG * RW * NJ; idx += NT) {
+    const int k = idx / NJ, j = idx % NJ;
     const float u = (k < a && j < r) ? p.U[k * p.ldu + j] : 0.f;
     Ud[idx] = pack2(u, u);
   }
@@ -122,11 +122,11 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
     }
   };
 
-  f2 accP[RW][4];
+  f2 accP[RW][NJ];
 #pragma unroll
   for (int i = 0; i < RW; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) accP[i][j] = 0ull;
+    for (int j = 0; j < NJ; ++j) accP[i][j] = 0ull;
 
   // prologue: nst - 1 tiles in flight
   int64_t t_issue = blockIdx.x;
@@ -153,40 +153,43 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
     }
     const TX* Xs = reinterpret_cast<const TX*>(stages + (size_t)st * stage_bytes);
     // ---- projection: partial V over this half-warp's rows
-    f2 accV[4][2];
+    f2 accV[NJ][2];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) accV[j][0] = accV[j][1] = 0ull;
+    for (int j = 0; j < NJ; ++j) accV[j][0] = accV[j][1] = 0ull;
 #pragma unroll
     for (int i = 0; i < RW; ++i) {
       const int k = grp * RW + i;
       if (k < a) {
         f2 x01, x23;
         ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
-        const ulonglong2 ua = *reinterpret_cast<const ulonglong2*>(Ud + k * 4);
-        const ulonglong2 ub = *reinterpret_cast<const ulonglong2*>(Ud + k * 4 + 2);
-        ffma2(accV[0][0], x01, ua.x); ffma2(accV[0][1], x23, ua.x);
-        ffma2(accV[1][0], x01, ua.y); ffma2(accV[1][1], x23, ua.y);
-        ffma2(accV[2][0], x01, ub.x); ffma2(accV[2][1], x23, ub.x);
-        ffma2(accV[3][0], x01, ub.y); ffma2(accV[3][1], x23, ub.y);
+#pragma unroll
+        for (int j = 0; j < NJ; j += 2) {
+          const ulonglong2 u = *reinterpret_cast<const ulonglong2*>(Ud + k * NJ + j);
+          ffma2(accV[j][0], x01, u.x); ffma2(accV[j][1], x23, u.x);
+          ffma2(accV[j + 1][0], x01, u.y); ffma2(accV[j + 1][1], x23, u.y);
+        }
       }
     }
     // the two half-warps of a warp (same columns, neighbouring row groups) meet by one shuffle
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+    for (int j = 0; j < NJ; ++j)
 #pragma unroll
       for (int h = 0; h < 2; ++h) accV[j][h] = fadd2(accV[j][h], __shfl_xor_sync(0xffffffffu, accV[j][h], 16));
     if ((tid & 16) == 0) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-        *reinterpret_cast<ulonglong2*>(Vp + ((grp >> 1) * 4 + j) * TQ + 4 * lane) = make_ulonglong2(accV[j][0], accV[j][1]);
+      for (int j = 0; j < NJ; ++j)
+        *reinterpret_cast<ulonglong2*>(Vp + ((grp >> 1) * NJ + j) * TQ + 4 * lane) = make_ulonglong2(accV[j][0], accV[j][1]);
     }
     __syncthreads();
     {
       // the eight partials meet in warp order: Vt[j][q]
-      float s = 0.f;
 #pragma unroll
-      for (int w = 0; w < NG / 2; ++w) s += Vp[w * 4 * TQ + tid];
-      Vt[tid] = s;
+      for (int e = tid; e < NJ * TQ; e += NT) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < NG / 2; ++w) s += Vp[w * NJ * TQ + e];
+        Vt[e] = s;
+      }
     }
     __syncthreads();
     if (p.project_only) {
@@ -201,9 +204,9 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
       }
     } else {
       // ---- expansion: P[k][:] += sum over this lane's columns
-      f2 vt[4][2];
+      f2 vt[NJ][2];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < NJ; ++j) {
         const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(Vt + j * TQ + 4 * lane);
         vt[j][0] = v.x;
         vt[j][1] = v.y;
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
           f2 x01, x23;
           ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
+          for (int j = 0; j < NJ; ++j) {
             ffma2(accP[i][j], x01, vt[j][0]);
             ffma2(accP[i][j], x23, vt[j][1]);
           }
@@ -231,7 +234,7 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   for (int i = 0; i < RW; ++i) {
     const int k = grp * RW + i;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NJ; ++j) {
       float v = fold2(accP[i][j]);
 #pragma unroll
       for (int off = 8; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
@@ -240,9 +243,9 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   }
 }
 
-size_t fiber2_smem(int a, int rw, int nstage, bool bf16) {
-  return (size_t)nstage * a * kF2TQ * (bf16 ? 2 : 4) + (size_t)kF2Groups * rw * 4 * 8 +
-         (size_t)(kF2Groups / 2 + 1) * 4 * kF2TQ * 4;
+size_t fiber2_smem(int a, int rw, int nj, int nstage, bool bf16) {
+  return (size_t)nstage * a * kF2TQ * (bf16 ? 2 : 4) + (size_t)kF2Groups * rw * nj * 8 +
+         (size_t)(kF2Groups / 2 + 1) * nj * kF2TQ * 4;
 }
 
 int fiber2_rows_per_group(int a) {
@@ -251,42 +254,50 @@ int fiber2_rows_per_group(int a) {
 }
 
 // as many stages (2..4) as leave room for two CTAs per SM
-int fiber2_stages(int a, bool bf16) {
+int fiber2_stages(int a, int nj, bool bf16) {
   const int rw = fiber2_rows_per_group(a);
   int n = 4;
-  while (n > 2 && fiber2_smem(a, rw, n, bf16) > 112 * 1024) --n;
+  while (n > 2 && fiber2_smem(a, rw, nj, n, bf16) > 112 * 1024) --n;
   return n;
 }
 
+// ranks up to 4 for a <= 128, up to 8 for a <= 64 (the register budget of the row accumulators)
 bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
   (void)O;
-  return r <= 4 && a >= 2 && a <= 128 && I >= kF2TQ && I % (bf16 ? 8 : 4) == 0;
+  return r <= 8 && a >= 2 && a <= (r <= 4 ? 128 : 64) && I >= kF2TQ && I % (bf16 ? 8 : 4) == 0;
 }
 
 int64_t fiber2_tiles(int64_t O, int64_t I) { return O * ((I + kF2TQ - 1) / kF2TQ); }
 
-template <int RW, typename TX>
+template <int RW, int NJ, typename TX>
 static cudaError_t launch_fiber2_t(const Fiber2Args& p, int grid, size_t smem, cudaStream_t st) {
-  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_fiber2<RW, TX>), smem);
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_fiber2<RW, NJ, TX>), smem);
   if (e != cudaSuccess) return e;
-  k_fiber2<RW, TX><<<grid, kF2Threads, smem, st>>>(p);
+  k_fiber2<RW, NJ, TX><<<grid, kF2Threads, smem, st>>>(p);
   return cudaGetLastError();
 }
 
 cudaError_t launch_fiber2(const Fiber2Args& p0, int grid, bool bf16, cudaStream_t st) {
   Fiber2Args p = p0;
-  const int rw = fiber2_rows_per_group(p.a);
-  p.nstage = fiber2_stages(p.a, bf16);
-  const size_t smem = fiber2_smem(p.a, rw, p.nstage, bf16);
+  const int rw = fiber2_rows_per_group(p.a), nj = p.r <= 4 ? 4 : 8;
+  p.nstage = fiber2_stages(p.a, nj, bf16);
+  const size_t smem = fiber2_smem(p.a, rw, nj, p.nstage, bf16);
   const double xbytes = (double)p.O * p.a * p.I * (bf16 ? 2 : 4);
   ProfScope prof(p.project_only ? ASI_K_MODEPROD : ASI_K_EXPAND, st, xbytes);
-#define ASI_F2(RW_)                                                                        \
-  return bf16 ? launch_fiber2_t<RW_, __nv_bfloat16>(p, grid, smem, st) : launch_fiber2_t<RW_, float>(p, grid, smem, st)
+#define ASI_F2(RW_, NJ_)                                                                        \
+  return bf16 ? launch_fiber2_t<RW_, NJ_, __nv_bfloat16>(p, grid, smem, st) : launch_fiber2_t<RW_, NJ_, float>(p, grid, smem, st)
+  if (nj == 4) {
+    switch (rw) {
+      case 1: ASI_F2(1, 4);
+      case 2: ASI_F2(2, 4);
+      case 4: ASI_F2(4, 4);
+      default: ASI_F2(8, 4);
+    }
+  }
   switch (rw) {
-    case 1: ASI_F2(1);
-    case 2: ASI_F2(2);
-    case 4: ASI_F2(4);
-    default: ASI_F2(8);
+    case 1: ASI_F2(1, 8);
+    case 2: ASI_F2(2, 8);
+    default: ASI_F2(4, 8);
   }
 #undef ASI_F2
 }
