@@ -1013,7 +1013,8 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
     a.a = cd[m]; a.Q = a.O * a.I;
     a.n_out = pl->r[m]; a.ldb_k = pl->r[m]; a.ldb_j = 1;
     a.so = (int64_t)pl->r[m] * a.I; a.sj = a.I; a.si = 1;
-    ASI_CUDA(launch_modeprod(a, src_bf16, st));
+    a.status = reinterpret_cast<int*>(w);
+    ASI_CUDA(stream_modeprod(pl, a, src_bf16, st));
     cd[m] = pl->r[m];
     lead_r *= pl->r[m];
     src = a.Y;

@@ -97,28 +97,52 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   extern __shared__ __align__(128) unsigned char f2_smem[];
   const int tid = threadIdx.x, grp = tid >> 4, lane = tid & 15;
   const int a = p.a, r = p.r, nst = p.nstage;
-  const size_t stage_bytes = (size_t)a * TQ * sizeof(TX);
+  constexpr int AR = NG * RW;                        // staged rows: rows a..AR-1 stay zero, so no loop tests k < a
+  constexpr size_t stage_bytes = (size_t)AR * TQ * sizeof(TX);
   unsigned char* stages = f2_smem;
-  f2* Ud = reinterpret_cast<f2*>(f2_smem + (size_t)nst * stage_bytes);   // [NG RW][NJ]: (u, u)
-  float* Vp = reinterpret_cast<float*>(Ud + (size_t)NG * RW * NJ);       // [NG / 2][NJ][TQ]
+  f2* Ud = reinterpret_cast<f2*>(f2_smem + (size_t)nst * stage_bytes);   // [AR][NJ]: (u, u)
+  float* Vp = reinterpret_cast<float*>(Ud + (size_t)AR * NJ);            // [NG / 2][NJ][TQ]
   float* Vt = Vp + (NG / 2) * NJ * TQ;                                   // [NJ][TQ]
-  for (int idx = tid; idx < NG * RW * NJ; idx += NT) {
+  for (int idx = tid; idx < AR * NJ; idx += NT) {
     const int k = idx / NJ, j = idx % NJ;
     const float u = (k < a && j < r) ? p.U[k * p.ldu + j] : 0.f;
     Ud[idx] = pack2(u, u);
   }
+  if (a < AR) {
+    for (int s = 0; s < nst; ++s) {
+      uint32_t* z = reinterpret_cast<uint32_t*>(stages + (size_t)s * stage_bytes + (size_t)a * TQ * sizeof(TX));
+      for (int idx = tid; idx < (int)((AR - a) * TQ * sizeof(TX) / 4); idx += NT) z[idx] = 0u;
+    }
+  }
+  __syncthreads();
   const TX* __restrict__ X = reinterpret_cast<const TX*>(p.X);
-  const int64_t tpo = (p.I + TQ - 1) / TQ;
+  const int tpo = (int)((p.I + TQ - 1) / TQ);        // tiles per outer index (< 2^31: checked on the host)
+  const int nt = (int)p.n_tiles, gs = (int)gridDim.x;
 
-  auto issue = [&](int64_t t, int st) {
-    const int64_t o = t / tpo, i0 = (t - o * tpo) * TQ;
-    const TX* src = X + (o * a) * p.I + i0;
-    TX* dst = reinterpret_cast<TX*>(stages + (size_t)st * stage_bytes);
+  // A thread copies the same 16-byte unit of every KSTEP-th row: unit u of rows k0, k0 + KSTEP, ...
+  constexpr int KSTEP = NT / UPR;
+  const int cu = tid % UPR, ck0 = tid / UPR;
+  const int64_t src_row_step = (int64_t)KSTEP * p.I;
+  auto issue = [&](int o, int ic, int st) {
+    const int64_t i0 = (int64_t)ic * TQ;
     const int ncol = (int)((p.I - i0 < TQ) ? (p.I - i0) : TQ);
-    for (int idx = tid; idx < a * UPR; idx += NT) {
-      const int k = idx / UPR, u = idx - k * UPR;
-      const bool on = u * EPU < ncol;
-      cp_async16(dst + k * TQ + u * EPU, on ? (src + (int64_t)k * p.I + u * EPU) : src, on);
+    const bool on = cu * EPU < ncol;
+    const TX* src = X + ((int64_t)o * a + ck0) * p.I + i0 + (on ? cu * EPU : 0);
+    TX* dst = reinterpret_cast<TX*>(stages + (size_t)st * stage_bytes) + ck0 * TQ + cu * EPU;
+    for (int k = ck0; k < a; k += KSTEP) {
+      cp_async16(dst, src, on);
+      src += src_row_step;
+      dst += KSTEP * TQ;
+    }
+  };
+  // (o, ic) of a tile index advance by gs tiles at a time without divisions
+  const int step_o = gs / tpo, step_i = gs - step_o * tpo;
+  auto advance = [&](int& o, int& ic) {
+    o += step_o;
+    ic += step_i;
+    if (ic >= tpo) {
+      ic -= tpo;
+      ++o;
     }
   };
 
@@ -129,14 +153,17 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
     for (int j = 0; j < NJ; ++j) accP[i][j] = 0ull;
 
   // prologue: nst - 1 tiles in flight
-  int64_t t_issue = blockIdx.x;
+  int t_issue = blockIdx.x;
+  int io = (int)blockIdx.x / tpo, ii = (int)blockIdx.x - io * tpo;   // tile being issued
+  int co = io, ci = ii;                                              // tile being computed
   for (int s = 0; s < nst - 1; ++s) {
-    if (t_issue < p.n_tiles) issue(t_issue, s);
+    if (t_issue < nt) issue(io, ii, s);
     cp_commit();
-    t_issue += gridDim.x;
+    t_issue += gs;
+    advance(io, ii);
   }
   int st = 0;
-  for (int64_t t = blockIdx.x; t < p.n_tiles; t += gridDim.x) {
+  for (int t = blockIdx.x; t < nt; t += gs) {
     // one group is committed per iteration, so all but the newest nst - 2 groups are complete
     // exactly when the tile about to be used has landed
     if (nst == 2) cp_wait<0>();
@@ -147,9 +174,10 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
       // refill the stage freed by the previous iteration; its group is waited for nst - 1 iterations later
       int sf = st + nst - 1;
       if (sf >= nst) sf -= nst;
-      if (t_issue < p.n_tiles) issue(t_issue, sf);
+      if (t_issue < nt) issue(io, ii, sf);
       cp_commit();
-      t_issue += gridDim.x;
+      t_issue += gs;
+      advance(io, ii);
     }
     const TX* Xs = reinterpret_cast<const TX*>(stages + (size_t)st * stage_bytes);
     // ---- projection: partial V over this half-warp's rows
@@ -159,15 +187,13 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
 #pragma unroll
     for (int i = 0; i < RW; ++i) {
       const int k = grp * RW + i;
-      if (k < a) {
-        f2 x01, x23;
-        ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
+      f2 x01, x23;
+      ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
 #pragma unroll
-        for (int j = 0; j < NJ; j += 2) {
-          const ulonglong2 u = *reinterpret_cast<const ulonglong2*>(Ud + k * NJ + j);
-          ffma2(accV[j][0], x01, u.x); ffma2(accV[j][1], x23, u.x);
-          ffma2(accV[j + 1][0], x01, u.y); ffma2(accV[j + 1][1], x23, u.y);
-        }
+      for (int j = 0; j < NJ; j += 2) {
+        const ulonglong2 u = *reinterpret_cast<const ulonglong2*>(Ud + k * NJ + j);
+        ffma2(accV[j][0], x01, u.x); ffma2(accV[j][1], x23, u.x);
+        ffma2(accV[j + 1][0], x01, u.y); ffma2(accV[j + 1][1], x23, u.y);
       }
     }
     // the two half-warps of a warp (same columns, neighbouring row groups) meet by one shuffle
@@ -194,7 +220,7 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
     __syncthreads();
     if (p.project_only) {
       // Y[j][o, i0 + q] = V[q][j]
-      const int64_t o = t / tpo, i0 = (t - o * tpo) * TQ;
+      const int64_t o = co, i0 = (int64_t)ci * TQ;
       const int ncol = (int)((p.I - i0 < TQ) ? (p.I - i0) : TQ);
       for (int idx = tid; idx < r * (TQ / 4); idx += NT) {
         const int j = idx / (TQ / 4), v = idx - j * (TQ / 4);
@@ -214,18 +240,17 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
 #pragma unroll
       for (int i = 0; i < RW; ++i) {
         const int k = grp * RW + i;
-        if (k < a) {
-          f2 x01, x23;
-          ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
+        f2 x01, x23;
+        ld_quad<TX>(Xs + k * TQ + 4 * lane, x01, x23);
 #pragma unroll
-          for (int j = 0; j < NJ; ++j) {
-            ffma2(accP[i][j], x01, vt[j][0]);
-            ffma2(accP[i][j], x23, vt[j][1]);
-          }
+        for (int j = 0; j < NJ; ++j) {
+          ffma2(accP[i][j], x01, vt[j][0]);
+          ffma2(accP[i][j], x23, vt[j][1]);
         }
       }
     }
     st = (st + 1 == nst) ? 0 : st + 1;
+    advance(co, ci);
   }
   cp_wait<0>();
   if (p.project_only) return;
@@ -244,7 +269,8 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
 }
 
 size_t fiber2_smem(int a, int rw, int nj, int nstage, bool bf16) {
-  return (size_t)nstage * a * kF2TQ * (bf16 ? 2 : 4) + (size_t)kF2Groups * rw * nj * 8 +
+  (void)a;
+  return (size_t)nstage * kF2Groups * rw * kF2TQ * (bf16 ? 2 : 4) + (size_t)kF2Groups * rw * nj * 8 +
          (size_t)(kF2Groups / 2 + 1) * nj * kF2TQ * 4;
 }
 
@@ -264,7 +290,8 @@ int fiber2_stages(int a, int nj, bool bf16) {
 // ranks up to 4 for a <= 128, up to 8 for a <= 64 (the register budget of the row accumulators)
 bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
   (void)O;
-  return r <= 8 && a >= 2 && a <= (r <= 4 ? 128 : 64) && I >= kF2TQ && I % (bf16 ? 8 : 4) == 0;
+  return r <= 8 && a >= 2 && a <= (r <= 4 ? 128 : 64) && I >= kF2TQ && I % (bf16 ? 8 : 4) == 0 &&
+         O * ((I + kF2TQ - 1) / kF2TQ) < (1ll << 30);
 }
 
 int64_t fiber2_tiles(int64_t O, int64_t I) { return O * ((I + kF2TQ - 1) / kF2TQ); }
@@ -314,7 +341,7 @@ cudaError_t launch_fiber2(const Fiber2Args& p0, int grid, bool bf16, cudaStream_
 // through the bulk-copy engine (cp.async.bulk + mbarrier, bounded waits).
 // ---------------------------------------------------------------------------------------------
 namespace {
-constexpr int kP2Threads = 224, kP2Stages = 2;
+constexpr int kP2Threads = 224, kP2Stages = 3;
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -357,7 +384,7 @@ __device__ __forceinline__ bool mbar_wait_1s(uint64_t* bar, uint32_t parity) {
 }  // namespace
 
 template <int S, typename TX>
-__global__ void __launch_bounds__(kP2Threads, 3) k_plane2(PlaneArgs p) {
+__global__ void __launch_bounds__(kP2Threads, 2) k_plane2(PlaneArgs p) {
   constexpr int NT = kP2Threads, NST = kP2Stages;
   constexpr int QUADS = S / 4, HS = S / 7, WS = QUADS / 7, G = NT / (QUADS * HS);
   static_assert(S % 28 == 0 && QUADS * HS * G == NT && G * S * WS == NT, "S = 28 or 56");
@@ -425,16 +452,25 @@ __global__ void __launch_bounds__(kP2Threads, 3) k_plane2(PlaneArgs p) {
       t_issue += gridDim.x;
     }
     const TX* Xs = stages + (size_t)st * G * SS;
+    // the thread's values of the tile stay in registers for both passes: seven quads of its columns (rows
+    // 7 hs ..) and the seven quads of its row
+    f2 xc[7][2], xr[7][2];
+    {
+      const TX* xp = Xs + c_g * SS + (7 * c_hs) * S + 4 * c_quad;
+#pragma unroll
+      for (int i = 0; i < 7; ++i) ld_quad<TX>(xp + i * S, xc[i][0], xc[i][1]);
+      const TX* xq = Xs + r_row * S + 28 * r_ws;
+#pragma unroll
+      for (int q = 0; q < 7; ++q) ld_quad<TX>(xq + 4 * q, xr[q][0], xr[q][1]);
+    }
     // ---- pass A, column role: V3 partial over rows 7 hs ..
     {
       f2 acc[4][2];
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[j][0] = acc[j][1] = 0ull;
-      const TX* xp = Xs + c_g * SS + (7 * c_hs) * S + 4 * c_quad;
 #pragma unroll
       for (int i = 0; i < 7; ++i) {
-        f2 x01, x23;
-        ld_quad<TX>(xp + i * S, x01, x23);
+        const f2 x01 = xc[i][0], x23 = xc[i][1];
         const f2* ud = U3d + (7 * c_hs + i) * 4;
         const ulonglong2 ua = *reinterpret_cast<const ulonglong2*>(ud);
         const ulonglong2 ub = *reinterpret_cast<const ulonglong2*>(ud + 2);
@@ -453,11 +489,9 @@ __global__ void __launch_bounds__(kP2Threads, 3) k_plane2(PlaneArgs p) {
       f2 acc[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[j] = 0ull;
-      const TX* xp = Xs + r_row * S + 28 * r_ws;
 #pragma unroll
       for (int q = 0; q < 7; ++q) {
-        f2 x01, x23;
-        ld_quad<TX>(xp + 4 * q, x01, x23);
+        const f2 x01 = xr[q][0], x23 = xr[q][1];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const ulonglong2 u = *reinterpret_cast<const ulonglong2*>(U4t + j * S + 28 * r_ws + 4 * q);
@@ -487,12 +521,10 @@ __global__ void __launch_bounds__(kP2Threads, 3) k_plane2(PlaneArgs p) {
     __syncthreads();
     // ---- pass B, row role: P3[h] += sum_w X[h][w] V3[g][w]
     {
-      const TX* xp = Xs + r_row * S + 28 * r_ws;
       const float* vp = V3t + r_g * 4 * S + 28 * r_ws;
 #pragma unroll
       for (int q = 0; q < 7; ++q) {
-        f2 x01, x23;
-        ld_quad<TX>(xp + 4 * q, x01, x23);
+        const f2 x01 = xr[q][0], x23 = xr[q][1];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(vp + j * S + 4 * q);
@@ -503,11 +535,9 @@ __global__ void __launch_bounds__(kP2Threads, 3) k_plane2(PlaneArgs p) {
     }
     // ---- pass B, column role: P4[w] += sum_h X[h][w] V4[g,h]
     {
-      const TX* xp = Xs + c_g * SS + (7 * c_hs) * S + 4 * c_quad;
 #pragma unroll
       for (int i = 0; i < 7; ++i) {
-        f2 x01, x23;
-        ld_quad<TX>(xp + i * S, x01, x23);
+        const f2 x01 = xc[i][0], x23 = xc[i][1];
         const f2* vd = V4d + (c_g * S + 7 * c_hs + i) * 4;
         const ulonglong2 va = *reinterpret_cast<const ulonglong2*>(vd);
         const ulonglong2 vb = *reinterpret_cast<const ulonglong2*>(vd + 2);
