@@ -249,12 +249,29 @@ void layout_wgrad(asi_plan* pl) {
     for (int m = 1; m < nlead; ++m) rest *= pl->dims[m];
     z[0] = (int64_t)pl->r[0] * rest;                                   // dY x_1 U_1^T
     z[1] = (nlead > 1) ? (int64_t)pl->r[0] * pl->r[1] * pl->d.cout : 0;  // .. x_2 U_2^T
-    z[2] = (int64_t)pl->r[pl->nd - 1] * pl->d.cout;                    // Z4^T
-    pl->launches_wgrad = nlead + 2;
+    z[2] = (int64_t)pl->r[pl->nd - 1] * pl->d.cout;                    // Z4^T (generic kernels only)
+    pl->launches_wgrad = nlead + ((pl->d.flags & ASI_FLAG_GENERIC_ONLY) ? 2 : 1);
+    // bf16 token layers whose token-mode factor fits the tensor-core kernel: contract the token mode of dY
+    // first (dY is then read once, by tcgen05, and no [r1 x N x Dout] intermediate exists)
+    pl->lin_reorder = pl->nd == 3 && pl->bf16 && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) && pl->r[0] <= 8 &&
+                      pl->r[1] % 4 == 0 && pl->r[1] >= 16 && pl->r[1] <= 64 && pl->d.cout % 64 == 0 &&
+                      pl->dims[0] < 65536;
+    if (pl->lin_reorder) {
+      z[0] = pl->dims[0] * pl->d.cout * pl->r[1];                      // dY x_2 U_2^T  [B][Dout][r2]
+      z[1] = (int64_t)pl->r[0] * pl->d.cout * pl->r[1];                // .. x_1 U_1^T  [r1][Dout][r2]
+      z[2] = 0;
+      pl->launches_wgrad = 4;
+    }
   }
   for (int t = 0; t < 3; ++t) {
     pl->off_Z[t] = off;
     off = align_up(off + (size_t)z[t] * 4, 256);
+  }
+  pl->off_wtc = off;
+  pl->wtc_bytes = 0;
+  if (pl->d.kind == ASI_LINEAR && pl->lin_reorder) {
+    pl->wtc_bytes = tc_scratch_bytes(pl->dims[1], pl->r[1]);
+    off = align_up(off + pl->wtc_bytes, 256);
   }
   pl->conv_nsp = 1;
   pl->off_Z4p = off;
@@ -429,7 +446,13 @@ cudaError_t stream_modeprod(const asi_plan* pl, const ModeProdArgs& a, bool x_bf
                     a.so == (int64_t)a.n_out * a.I && a.Q * a.a >= (1 << 20) &&
                     fiber2_supported(a.O, a.a, a.I, a.n_out, x_bf16) &&
                     (reinterpret_cast<uintptr_t>(a.X) & 15u) == 0 && (reinterpret_cast<uintptr_t>(a.Y) & 15u) == 0;
-  if (!fits) return launch_modeprod(a, x_bf16, st);
+  if (!fits) {
+    int ichunk = 0;
+    size_t smem = 0;
+    if (!x_bf16 && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) && modeprod_stage_fits(a, &ichunk, &smem))
+      return launch_modeprod_stage(a, ichunk, smem, st);      // few columns, long mode
+    return launch_modeprod(a, x_bf16, st);
+  }
   Fiber2Args f;
   std::memset(&f, 0, sizeof(f));
   f.X = a.X;
@@ -996,6 +1019,34 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
   const int64_t Dout = pl->d.cout, Din = pl->dims[nd - 1];
   const int rl = pl->r[nd - 1];
 
+  ModeProdArgs a;
+  if (pl->lin_reorder) {
+    // dY x_2 U_2^T on the tensor cores -> [B][Dout][r2], then x_1 U_1^T -> [r1][Dout][r2]
+    const int64_t B = pl->dims[0], N = pl->dims[1];
+    const int r1 = pl->r[0], r2 = pl->r[1];
+    float* Y1 = reinterpret_cast<float*>(w + pl->off_Z[0]);
+    float* Y2 = reinterpret_cast<float*>(w + pl->off_Z[1]);
+    a.X = dY; a.B = U + pl->u_off[1]; a.Y = Y1;
+    a.O = B; a.a = N; a.I = Dout; a.Q = B * Dout;
+    a.n_out = r2; a.ldb_k = r2; a.ldb_j = 1;
+    a.so = Dout * r2; a.sj = 1; a.si = r2;
+    a.tc_scratch = w + pl->off_wtc; a.tc_scratch_bytes = pl->wtc_bytes;
+    a.status = reinterpret_cast<int*>(w);
+    ASI_CUDA(launch_modeprod(a, true, st));
+    ModeProdArgs b;
+    b.X = Y1; b.B = U + pl->u_off[0]; b.Y = Y2;
+    b.O = 1; b.a = B; b.I = Dout * r2; b.Q = b.I;
+    b.n_out = r1; b.ldb_k = r1; b.ldb_j = 1;
+    b.so = (int64_t)r1 * b.I; b.sj = b.I; b.si = 1;
+    b.status = reinterpret_cast<int*>(w);
+    ASI_CUDA(stream_modeprod(pl, b, false, st));
+    LinTailArgs t;
+    t.Z = Y2; t.core = core; t.U = U + pl->u_off[2]; t.dW = dW;
+    t.s1 = Dout * r2; t.s2 = 1; t.so = r2;
+    t.L1 = r1; t.L2 = r2; t.Dout = (int)Dout; t.Din = (int)Din; t.r = rl; t.lead_fastest = 1;
+    ASI_CUDA(launch_lin_tail(t, st));
+    return ASI_OK;
+  }
   // Z = dY x_1 U_1^T (x_2 U_2^T): leading modes one by one
   int64_t cd[ASI_MAX_MODES];
   for (int m = 0; m < nlead; ++m) cd[m] = pl->dims[m];
@@ -1003,7 +1054,6 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
   const void* src = dY;
   bool src_bf16 = pl->bf16;
   int64_t lead_r = 1;
-  ModeProdArgs a;
   for (int m = 0; m < nlead; ++m) {
     a.X = src; a.B = U + pl->u_off[m];
     a.Y = reinterpret_cast<float*>(w + pl->off_Z[m]);
@@ -1019,6 +1069,16 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
     lead_r *= pl->r[m];
     src = a.Y;
     src_bf16 = false;
+  }
+  if (!(pl->d.flags & ASI_FLAG_GENERIC_ONLY)) {
+    // Z4 = Z . core over the leading ranks and dW = Z4 U_last^T in one launch; Z is [r1 (r2)][Dout]
+    LinTailArgs t;
+    t.Z = static_cast<const float*>(src); t.core = core; t.U = U + pl->u_off[nd - 1]; t.dW = dW;
+    t.L1 = pl->r[0]; t.L2 = (nlead > 1) ? pl->r[1] : 1;
+    t.s1 = (int64_t)t.L2 * Dout; t.s2 = Dout; t.so = 1;
+    t.Dout = (int)Dout; t.Din = (int)Din; t.r = rl; t.lead_fastest = 0;
+    ASI_CUDA(launch_lin_tail(t, st));
+    return ASI_OK;
   }
   // Z4^T[k, o] = sum_{lead} Z[lead, o] core[lead, k]
   float* Z4t = reinterpret_cast<float*>(w + pl->off_Z[2]);

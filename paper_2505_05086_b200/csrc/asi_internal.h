@@ -248,6 +248,20 @@ size_t core_tail_part_elems(int r1, int r2, int r3, int r4, int C, int H, int W)
 cudaError_t launch_core_tail(const CoreTailArgs& p, cudaStream_t st);
 cudaError_t launch_z3(const float* core, const float* U3, const float* U4, float* Z3, int r12, int r3, int r4,
                       int H, int W, cudaStream_t st);
+// token path (asi_token_kernels.cu)
+struct LinTailArgs {
+  const float* Z;      // Z(l1, l2, o) = Z[l1 * s1 + l2 * s2 + o * so]
+  const float* core;   // [L1 L2][r]
+  const float* U;      // [Din][r]
+  float* dW;           // [Dout][Din]
+  int64_t s1, s2, so;
+  int L1, L2, Dout, Din, r;
+  int lead_fastest;    // 1: the lead index is the contiguous one in memory (s2 == 1), else o is
+};
+bool lin_tail_supported(int r);
+cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st);
+bool modeprod_stage_fits(const ModeProdArgs& p, int* ichunk, size_t* smem);
+cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem, cudaStream_t st);
 bool plane2_supported(int S, int64_t n_planes, int r3, int r4);
 int plane2_grid(int S, int64_t n_planes, int max_ctas);
 cudaError_t launch_plane2(const PlaneArgs& p, int grid, bool bf16, cudaStream_t st);
@@ -294,6 +308,8 @@ struct asi_plan {
   size_t off_Z[3], off_Z4p;
   int conv_nsp;                    // > 1: terms 4-5 in two launches with conv_nsp partial Z4 per channel
   bool conv_z3;                    // terms 2-3 in one launch (k_z3)
+  bool lin_reorder;                // linear backward of a bf16 token layer: dY x_2 U_2^T first (tensor cores)
+  size_t off_wtc, wtc_bytes;       // bf16 operand scratch of that product
   bool core_tail;                  // the core products after the first in one launch
   size_t off_ctp;                  // partial cores of that launch
   size_t wgrad_ws;
