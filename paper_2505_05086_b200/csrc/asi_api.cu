@@ -118,7 +118,7 @@ void layout_compress(asi_plan* pl) {
   for (int m = 0; m < pl->nd; ++m)
     if (pl->fiber[m] && fiber2_supported(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16)) {
       pl->fiber2[m] = true;
-      pl->fiber_grid[m] = (int)std::min<int64_t>(fiber2_tiles(pl->mv[m].O, pl->mv[m].I), 296);
+      pl->fiber_grid[m] = fiber2_grid(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I);
     }
   int64_t vmax = 0;
   if (!pl->fast_compress)
@@ -249,8 +249,9 @@ void layout_wgrad(asi_plan* pl) {
     for (int m = 1; m < nlead; ++m) rest *= pl->dims[m];
     z[0] = (int64_t)pl->r[0] * rest;                                   // dY x_1 U_1^T
     z[1] = (nlead > 1) ? (int64_t)pl->r[0] * pl->r[1] * pl->d.cout : 0;  // .. x_2 U_2^T
-    z[2] = (int64_t)pl->r[pl->nd - 1] * pl->d.cout;                    // Z4^T (generic kernels only)
-    pl->launches_wgrad = nlead + ((pl->d.flags & ASI_FLAG_GENERIC_ONLY) ? 2 : 1);
+    pl->lin_nsplit = lin_tail_nsplit(pl->r[0] * (nlead > 1 ? pl->r[1] : 1), pl->d.cout);
+    z[2] = (int64_t)pl->lin_nsplit * pl->r[pl->nd - 1] * pl->d.cout;   // Z4 (its shares)
+    pl->launches_wgrad = nlead + 2;
     // bf16 token layers whose token-mode factor fits the tensor-core kernel: contract the token mode of dY
     // first (dY is then read once, by tcgen05, and no [r1 x N x Dout] intermediate exists)
     pl->lin_reorder = pl->nd == 3 && pl->bf16 && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY) && pl->r[0] <= 8 &&
@@ -259,8 +260,7 @@ void layout_wgrad(asi_plan* pl) {
     if (pl->lin_reorder) {
       z[0] = pl->dims[0] * pl->d.cout * pl->r[1];                      // dY x_2 U_2^T  [B][Dout][r2]
       z[1] = (int64_t)pl->r[0] * pl->d.cout * pl->r[1];                // .. x_1 U_1^T  [r1][Dout][r2]
-      z[2] = 0;
-      pl->launches_wgrad = 4;
+      pl->launches_wgrad = 5;
     }
   }
   for (int t = 0; t < 3; ++t) {
@@ -464,7 +464,7 @@ cudaError_t stream_modeprod(const asi_plan* pl, const ModeProdArgs& a, bool x_bf
   f.O = a.O; f.I = a.I; f.a = (int)a.a; f.r = a.n_out;
   f.n_tiles = fiber2_tiles(a.O, a.I);
   f.project_only = 1;
-  return launch_fiber2(f, (int)std::min<int64_t>(f.n_tiles, 296), x_bf16, st);
+  return launch_fiber2(f, fiber2_grid(a.O, a.a, a.I), x_bf16, st);
 }
 
 // Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).
@@ -1044,6 +1044,7 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
     t.Z = Y2; t.core = core; t.U = U + pl->u_off[2]; t.dW = dW;
     t.s1 = Dout * r2; t.s2 = 1; t.so = r2;
     t.L1 = r1; t.L2 = r2; t.Dout = (int)Dout; t.Din = (int)Din; t.r = rl; t.lead_fastest = 1;
+    t.Z4p = reinterpret_cast<float*>(w + pl->off_Z[2]); t.nsplit = pl->lin_nsplit;
     ASI_CUDA(launch_lin_tail(t, st));
     return ASI_OK;
   }
@@ -1077,6 +1078,7 @@ asi_status_t asi_linear_wgrad(const asi_plan_t* pl, const float* core, const flo
     t.L1 = pl->r[0]; t.L2 = (nlead > 1) ? pl->r[1] : 1;
     t.s1 = (int64_t)t.L2 * Dout; t.s2 = Dout; t.so = 1;
     t.Dout = (int)Dout; t.Din = (int)Din; t.r = rl; t.lead_fastest = 0;
+    t.Z4p = reinterpret_cast<float*>(w + pl->off_Z[2]); t.nsplit = pl->lin_nsplit;
     ASI_CUDA(launch_lin_tail(t, st));
     return ASI_OK;
   }

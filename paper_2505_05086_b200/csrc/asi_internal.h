@@ -233,6 +233,10 @@ cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t
 size_t plane_smem(int S);
 bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16);
 int64_t fiber2_tiles(int64_t O, int64_t I);
+int fiber2_grid(int64_t O, int64_t a, int64_t I);
+bool fiber_reg_supported(int64_t O, int64_t a, int64_t I, int r);
+int fiber_reg_grid(int64_t O, int64_t a, int64_t I);
+cudaError_t launch_fiber_reg(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st);
 cudaError_t launch_fiber2(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st);
 // core = T x_2 U_2^T x_3 U_3^T x_4 U_4^T for T [r1][C][H][W] in one launch (k_core_tail)
 struct CoreTailArgs {
@@ -254,11 +258,14 @@ struct LinTailArgs {
   const float* core;   // [L1 L2][r]
   const float* U;      // [Din][r]
   float* dW;           // [Dout][Din]
+  float* Z4p;          // [nsplit][Dout][r] shares of Z4 (scratch)
+  int nsplit;
   int64_t s1, s2, so;
   int L1, L2, Dout, Din, r;
   int lead_fastest;    // 1: the lead index is the contiguous one in memory (s2 == 1), else o is
 };
 bool lin_tail_supported(int r);
+int lin_tail_nsplit(int nlead, int64_t Dout);
 cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st);
 bool modeprod_stage_fits(const ModeProdArgs& p, int* ichunk, size_t* smem);
 cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem, cudaStream_t st);
@@ -308,6 +315,7 @@ struct asi_plan {
   size_t off_Z[3], off_Z4p;
   int conv_nsp;                    // > 1: terms 4-5 in two launches with conv_nsp partial Z4 per channel
   bool conv_z3;                    // terms 2-3 in one launch (k_z3)
+  int lin_nsplit;                  // shares of the leading indices in the Z4 kernel of the linear backward
   bool lin_reorder;                // linear backward of a bf16 token layer: dY x_2 U_2^T first (tensor cores)
   size_t off_wtc, wtc_bytes;       // bf16 operand scratch of that product
   bool core_tail;                  // the core products after the first in one launch

@@ -5,19 +5,26 @@
 //                      (Algorithm 1, core update).  One thread per column leaves such a product on a handful
 //                      of CTAs walking the mode serially; here a CTA stages X(o, :, i-chunk) and B in shared
 //                      memory and its threads share the outputs (j, i).
-//   k_lin_tail       : the end of the linear backward (Sec. 3.1 footnote, derived steps L2-L3) in one launch:
+//   k_fiber_reg      : the two products of a mode with a short fiber (a <= 32), through registers only.
+//   k_lin_z4, k_lin_tail : the end of the linear backward (Sec. 3.1 footnote, derived steps L2-L3):
 //                        Z4[o][k] = sum_{l1,l2} Z(l1, l2, o) core[l1][l2][k],   dW[o][d] = sum_k Z4[o][k] U[d][k].
-//                      A CTA owns 64 output rows x 128 columns of dW: it forms its 64 rows of Z4 in shared
-//                      memory (recomputed per column tile: the contraction is small next to the 4-byte
-//                      write of every dW entry), then expands them in 8 x 4 register tiles with coalesced
-//                      stores.  dW is written exactly once.
+//                      k_lin_z4 forms Z4 once (16 output rows per CTA, the leading indices shared between up to
+//                      eight CTAs that each write their own share -- no atomics, the sum order is fixed);
+//                      k_lin_tail adds the shares and expands 64 x 128 tiles of dW in 8 x 4 register tiles with
+//                      coalesced stores.  dW is written exactly once.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
 #include "asi_internal.h"
 
 namespace asi {
 
 namespace {
 constexpr int kStageThreads = 256;
-constexpr int kLtO = 64, kLtD = 128, kLtLead = 32;
+constexpr int kFrThreads = 256;
+constexpr int kLtO = 64, kLtD = 128;
+constexpr int kLzO = 16, kLzLead = 64;
 }  // namespace
 
 __global__ void __launch_bounds__(kStageThreads) k_modeprod_stage(ModeProdArgs p, int ichunk) {
@@ -95,84 +102,299 @@ cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem
 }
 
 // ---------------------------------------------------------------------------------------------
-// k_lin_tail
+// k_fiber_reg: both products of a mode with a SHORT fiber (a <= 32: the batch mode of a token tensor), or
+// with project_only the mode product alone, streamed through registers.  A lane owns four neighbouring
+// columns of the unfolding and eight rows; KS lanes (a <= 8 KS) share a column quad and add their partial
+// V with shuffles, so no tile is staged and nothing meets in shared memory until the CTA's final sum of P.
 // ---------------------------------------------------------------------------------------------
-template <int NQ>      // a thread of phase 1 keeps NQ sums: ranks up to 4 NQ
+template <typename TX> struct RawQuad;
+template <> struct RawQuad<float> {
+  float4 v;
+  __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
+  __device__ __forceinline__ void get(float (&x)[4], bool on) const {
+    x[0] = on ? v.x : 0.f; x[1] = on ? v.y : 0.f; x[2] = on ? v.z : 0.f; x[3] = on ? v.w : 0.f;
+  }
+};
+template <> struct RawQuad<__nv_bfloat16> {
+  uint2 v;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint2*>(p)); }
+  __device__ __forceinline__ void get(float (&x)[4], bool on) const {
+    const uint32_t a = on ? v.x : 0u, b = on ? v.y : 0u;
+    x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xffff0000u);
+    x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xffff0000u);
+  }
+};
+
+template <int NJ, int KS, typename TX>
+__global__ void __launch_bounds__(kFrThreads, 1) k_fiber_reg(Fiber2Args p) {
+  constexpr int QW = 32 / KS;                        // column quads per warp
+  constexpr int NW = kFrThreads / 32;
+  __shared__ __align__(16) float Us[8 * KS * NJ];    // rows >= a and columns >= r are zero
+  __shared__ float red[NW][8 * KS * NJ];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ks = lane / QW, cq = lane - ks * QW;
+  const int a = p.a, r = p.r, r0 = 8 * ks;
+  for (int e = tid; e < 8 * KS * NJ; e += kFrThreads) {
+    const int k = e / NJ, j = e - k * NJ;
+    Us[e] = (k < a && j < r) ? p.U[(int64_t)k * p.ldu + j] : 0.f;
+  }
+  __syncthreads();
+  const int Iq = (int)(p.I >> 2);
+  const int total = (int)p.O * Iq;                   // column quads of the unfolding (< 2^31, checked by the host)
+  const int stride = gridDim.x * NW * QW;
+  const TX* X = static_cast<const TX*>(p.X);
+  int64_t roff[8];                                   // rows past the end re-read row a - 1 (their factor row is 0)
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) roff[kk] = (int64_t)((r0 + kk < a) ? r0 + kk : a - 1) * p.I;
+  float accP[8][NJ];
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) accP[kk][j] = 0.f;
+
+  int gbase = (blockIdx.x * NW + warp) * QW;         // warp-uniform: the loop test is the same in every lane
+  RawQuad<TX> cur[8], nxt[8];
+  int o_c = 0, iq_c = 0;
+  bool on_c = false;
+  if (gbase < total) {
+    const int g = gbase + cq;
+    on_c = g < total;
+    const int gl = on_c ? g : total - 1;
+    o_c = gl / Iq; iq_c = gl - o_c * Iq;
+    const TX* src = X + (int64_t)o_c * a * p.I + 4 * (int64_t)iq_c;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) cur[kk].load(src + roff[kk]);
+  }
+  while (gbase < total) {
+    // the next quad's rows are requested before this one's arithmetic (always from a valid address)
+    const int gnb = gbase + stride;
+    const int gn = gnb + cq;
+    const bool on_n = gnb < total && gn < total;
+    const int gl = on_n ? gn : total - 1;
+    const int o_n = gl / Iq, iq_n = gl - o_n * Iq;
+    {
+      const TX* src = X + (int64_t)o_n * a * p.I + 4 * (int64_t)iq_n;
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) nxt[kk].load(src + roff[kk]);
+    }
+    float V[4][NJ];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) V[c][j] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      float x[4];
+      cur[kk].get(x, on_c);
+#pragma unroll
+      for (int j4 = 0; j4 < NJ; j4 += 4) {
+        const float4 u = *reinterpret_cast<const float4*>(&Us[(r0 + kk) * NJ + j4]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          V[c][j4 + 0] = fmaf(x[c], u.x, V[c][j4 + 0]);
+          V[c][j4 + 1] = fmaf(x[c], u.y, V[c][j4 + 1]);
+          V[c][j4 + 2] = fmaf(x[c], u.z, V[c][j4 + 2]);
+          V[c][j4 + 3] = fmaf(x[c], u.w, V[c][j4 + 3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int s = QW; s < 32; s *= 2)                 // the KS row groups of a column quad
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) V[c][j] += __shfl_xor_sync(0xffffffffu, V[c][j], s);
+    if (p.project_only) {
+      if (on_c) {
+        float* dst = p.Y + (int64_t)o_c * p.y_so + 4 * (int64_t)iq_c;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j)
+          if (j < r && (j % KS) == ks)
+            *reinterpret_cast<float4*>(dst + (int64_t)j * p.y_sj) = make_float4(V[0][j], V[1][j], V[2][j], V[3][j]);
+      }
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        float x[4];
+        cur[kk].get(x, on_c);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int j = 0; j < NJ; ++j) accP[kk][j] = fmaf(x[c], V[c][j], accP[kk][j]);
+      }
+    }
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) cur[kk] = nxt[kk];
+    o_c = o_n; iq_c = iq_n; on_c = on_n;
+    gbase = gnb;
+  }
+  if (p.project_only) return;
+  // P of this CTA: over the lanes of a row group, then over the warps
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk)
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      float v = accP[kk][j];
+#pragma unroll
+      for (int s = 1; s < QW; s *= 2) v += __shfl_xor_sync(0xffffffffu, v, s);
+      if (cq == 0) red[warp][(r0 + kk) * NJ + j] = v;
+    }
+  __syncthreads();
+  for (int e = tid; e < 8 * KS * NJ; e += kFrThreads) {
+    const int k = e / NJ, j = e - k * NJ;
+    if (k >= a || j >= r) continue;
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) v += red[w][e];
+    p.Pp[((int64_t)blockIdx.x * a + k) * r + j] = v;
+  }
+}
+
+bool fiber_reg_supported(int64_t O, int64_t a, int64_t I, int r) {
+  return r >= 1 && r <= 8 && a >= 1 && a <= 32 && I % 4 == 0 && O * (I / 4) < (1ll << 30);
+}
+
+static int fiber_reg_ks(int a) { return a <= 8 ? 1 : a <= 16 ? 2 : 4; }
+
+int fiber_reg_grid(int64_t O, int64_t a, int64_t I) {
+  const int qw = 32 / fiber_reg_ks((int)a);
+  const int64_t per_cta = (int64_t)(kFrThreads / 32) * qw;
+  return (int)std::min<int64_t>(148, (O * (I / 4) + per_cta - 1) / per_cta);
+}
+
+template <int NJ, int KS>
+static cudaError_t launch_fiber_reg_t(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st) {
+  if (bf16) k_fiber_reg<NJ, KS, __nv_bfloat16><<<grid, kFrThreads, 0, st>>>(p);
+  else k_fiber_reg<NJ, KS, float><<<grid, kFrThreads, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fiber_reg(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st) {
+  const double xbytes = (double)p.O * p.a * p.I * (bf16 ? 2 : 4);
+  ProfScope prof(p.project_only ? ASI_K_MODEPROD : ASI_K_EXPAND, st, xbytes);
+  const int ks = fiber_reg_ks(p.a);
+  if (p.r <= 4) {
+    if (ks == 1) return launch_fiber_reg_t<4, 1>(p, grid, bf16, st);
+    if (ks == 2) return launch_fiber_reg_t<4, 2>(p, grid, bf16, st);
+    return launch_fiber_reg_t<4, 4>(p, grid, bf16, st);
+  }
+  if (ks == 1) return launch_fiber_reg_t<8, 1>(p, grid, bf16, st);
+  if (ks == 2) return launch_fiber_reg_t<8, 2>(p, grid, bf16, st);
+  return launch_fiber_reg_t<8, 4>(p, grid, bf16, st);
+}
+
+// ---------------------------------------------------------------------------------------------
+// k_lin_z4 and k_lin_tail
+// ---------------------------------------------------------------------------------------------
+// Z4p[split][o][k] = sum over the split's leading indices of Z(lead, o) core[lead][k].  A CTA owns 16 output
+// rows and one share of the leading indices; thread (o, kg) keeps the sums k = kg, kg + 16, ..
+template <int NQ>
+__global__ void __launch_bounds__(256) k_lin_z4(LinTailArgs p) {
+  extern __shared__ __align__(16) float lt_smem[];
+  const int r = p.r;
+  float* Zc = lt_smem;                               // [kLzLead][16 + 1]
+  float* Sc = Zc + kLzLead * (kLzO + 1);             // [kLzLead][r]
+  const int tid = threadIdx.x;
+  const int o0 = blockIdx.x * kLzO;
+  const int nlead = p.L1 * p.L2;
+  const int per = ((nlead + p.nsplit - 1) / p.nsplit + kLzLead - 1) / kLzLead * kLzLead;
+  const int lbeg = blockIdx.y * per, lend = (lbeg + per < nlead) ? lbeg + per : nlead;
+  const int po = tid & (kLzO - 1), kg = tid >> 4;
+  float acc[NQ];
+#pragma unroll
+  for (int q = 0; q < NQ; ++q) acc[q] = 0.f;
+  for (int l0 = lbeg; l0 < lend; l0 += kLzLead) {
+    const int nl = (lend - l0 < kLzLead) ? lend - l0 : kLzLead;
+    float v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {                    // 64 x 16 values, four per thread, loads first
+      const int e = tid + u * 256;
+      int l, o;
+      if (p.lead_fastest) { o = e / kLzLead; l = e - o * kLzLead; } else { l = e >> 4; o = e & (kLzO - 1); }
+      const int lead = l0 + l, l1 = lead / p.L2, l2 = lead - l1 * p.L2;
+      const bool on = l < nl && o0 + o < p.Dout;
+      v[u] = p.Z[on ? (int64_t)l1 * p.s1 + (int64_t)l2 * p.s2 + (int64_t)(o0 + o) * p.so : 0];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = tid + u * 256;
+      int l, o;
+      if (p.lead_fastest) { o = e / kLzLead; l = e - o * kLzLead; } else { l = e >> 4; o = e & (kLzO - 1); }
+      Zc[l * (kLzO + 1) + o] = (l < nl && o0 + o < p.Dout) ? v[u] : 0.f;
+    }
+    for (int e = tid; e < kLzLead * r; e += 256)
+      Sc[e] = (e < nl * r) ? p.core[(int64_t)l0 * r + e] : 0.f;
+    __syncthreads();
+#pragma unroll 4
+    for (int l = 0; l < kLzLead; ++l) {
+      const float z = Zc[l * (kLzO + 1) + po];
+#pragma unroll
+      for (int q = 0; q < NQ; ++q)
+        if (kg + 16 * q < r) acc[q] = fmaf(z, Sc[l * r + kg + 16 * q], acc[q]);
+    }
+    __syncthreads();
+  }
+  if (o0 + po < p.Dout) {
+    float* dst = p.Z4p + ((int64_t)blockIdx.y * p.Dout + o0 + po) * r;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q)
+      if (kg + 16 * q < r) dst[kg + 16 * q] = acc[q];
+  }
+}
+
+// dW[o][d] = sum_k Z4[o][k] U[d][k], Z4 = the sum of the nsplit shares: 64 x 128 tile per CTA, 8 x 4 per thread
 __global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p) {
   extern __shared__ __align__(16) float lt_smem[];
   const int r = p.r, PR = r | 1;                     // odd pitch: conflict-free reads down a column of rows
   float* Z4s = lt_smem;                              // [64][PR]
   float* Us = Z4s + kLtO * PR;                       // [128][PR]
-  float* Zc = Us + kLtD * PR;                        // [kLtLead][64 + 1]
-  float* Sc = Zc + kLtLead * (kLtO + 1);             // [kLtLead][r]
   const int tid = threadIdx.x, lane = tid & 31;
   const int o0 = blockIdx.x * kLtO, d0 = blockIdx.y * kLtD;
-  const int nlead = p.L1 * p.L2;
-  // ---- phase 1: Z4s[o][k] = sum_lead Z(lead, o0 + o) core[lead][k]; thread (o, kg) keeps k = kg, kg + 4, ..
-  const int po = tid & 63, kg = tid >> 6;
-  float acc[NQ];
+  const int no = (p.Dout - o0 < kLtO) ? p.Dout - o0 : kLtO;
+  const int nd = (p.Din - d0 < kLtD) ? p.Din - d0 : kLtD;
+  const float* zsrc = p.Z4p + (int64_t)o0 * r;
+  const int64_t zstep = (int64_t)p.Dout * r;
+  for (int e0 = 0; e0 < kLtO * r; e0 += 4 * 256) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int s = 0; s < p.nsplit; ++s) {
+      float t[4];
 #pragma unroll
-  for (int q = 0; q < NQ; ++q) acc[q] = 0.f;
-  for (int l0 = 0; l0 < nlead; l0 += kLtLead) {
-    const int nl = (nlead - l0 < kLtLead) ? nlead - l0 : kLtLead;
-    {
-      float v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {                  // 32 x 64 values, eight per thread, loads first
-        const int e = tid + u * 256;
-        int l, o;
-        if (p.lead_fastest) { o = e / kLtLead; l = e - o * kLtLead; } else { l = e >> 6; o = e & 63; }
-        const int lead = l0 + l, l1 = lead / p.L2, l2 = lead - l1 * p.L2;
-        const bool on = l < nl && o0 + o < p.Dout;
-        v[u] = p.Z[on ? (int64_t)l1 * p.s1 + (int64_t)l2 * p.s2 + (int64_t)(o0 + o) * p.so : 0];
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + tid + u * 256;
+        t[u] = zsrc[s * zstep + (e < no * r ? e : 0)];
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int e = tid + u * 256;
-        int l, o;
-        if (p.lead_fastest) { o = e / kLtLead; l = e - o * kLtLead; } else { l = e >> 6; o = e & 63; }
-        Zc[l * (kLtO + 1) + o] = (l < nl && o0 + o < p.Dout) ? v[u] : 0.f;
-      }
-      for (int e = tid; e < kLtLead * r; e += 256) {
-        const int l = e / r, k = e - l * r;
-        Sc[e] = (l < nl) ? p.core[(int64_t)(l0 + l) * r + k] : 0.f;
-      }
+      for (int u = 0; u < 4; ++u) v[u] += t[u];
     }
-    __syncthreads();
-#pragma unroll 4
-    for (int l = 0; l < kLtLead; ++l) {
-      const float z = Zc[l * (kLtO + 1) + po];
 #pragma unroll
-      for (int q = 0; q < NQ; ++q)
-        if (kg + 4 * q < r) acc[q] = fmaf(z, Sc[l * r + kg + 4 * q], acc[q]);
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + tid + u * 256, o = e / r;
+      if (e < kLtO * r) Z4s[o * PR + (e - o * r)] = (e < no * r) ? v[u] : 0.f;
     }
-    __syncthreads();
   }
-#pragma unroll
-  for (int q = 0; q < NQ; ++q)
-    if (kg + 4 * q < r) Z4s[po * PR + kg + 4 * q] = acc[q];
-  // the factor rows of this column tile
+  const float* usrc = p.U + (int64_t)d0 * r;
   for (int e0 = 0; e0 < kLtD * r; e0 += 8 * 256) {
     float v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int e = e0 + tid + u * 256, d = e / r;
-      v[u] = p.U[(e < kLtD * r && d0 + d < p.Din) ? (int64_t)(d0 + d) * r + (e - d * r) : 0];
+      const int e = e0 + tid + u * 256;
+      v[u] = usrc[e < nd * r ? e : 0];
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + tid + u * 256, d = e / r;
-      if (e < kLtD * r) Us[d * PR + (e - d * r)] = (d0 + d < p.Din) ? v[u] : 0.f;
+      if (e < kLtD * r) Us[d * PR + (e - d * r)] = (e < nd * r) ? v[u] : 0.f;
     }
   }
   __syncthreads();
-  // ---- phase 2: dW[o0 + o][d0 + d] for o = 8 to .. 8 to + 7, d = lane + 32 i
+  // dW[o0 + o][d0 + d] for o = 8 to .. 8 to + 7, d = lane + 32 i
   const int to = tid >> 5;
   float out[8][4];
 #pragma unroll
   for (int x = 0; x < 8; ++x)
 #pragma unroll
     for (int y = 0; y < 4; ++y) out[x][y] = 0.f;
+#pragma unroll 2
   for (int k = 0; k < r; ++k) {
     float zz[8], uu[4];
 #pragma unroll
@@ -198,25 +420,43 @@ __global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p) {
 
 bool lin_tail_supported(int r) { return r >= 1 && r <= 128; }
 
+int lin_tail_nsplit(int nlead, int64_t Dout) {
+  const int64_t tiles = (Dout + kLzO - 1) / kLzO;
+  int64_t ns = 296 / (tiles > 0 ? tiles : 1);
+  const int64_t cap = (nlead + kLzLead - 1) / kLzLead;      // at least one chunk of leads per share
+  if (ns > cap) ns = cap;
+  if (ns > 8) ns = 8;
+  return (int)(ns < 1 ? 1 : ns);
+}
+
 cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st) {
   const int PR = p.r | 1;
-  const size_t smem = 4 * ((size_t)(kLtO + kLtD) * PR + (size_t)kLtLead * (kLtO + 1) + (size_t)kLtLead * p.r);
   ProfScope prof(ASI_K_MODEPROD, st, 4.0 * ((double)p.Dout * p.Din + (double)p.L1 * p.L2 * p.Dout));
-  dim3 grid((unsigned)((p.Dout + kLtO - 1) / kLtO), (unsigned)((p.Din + kLtD - 1) / kLtD));
-  cudaError_t e;
-  if (p.r <= 32) {
-    e = opt_in_smem(reinterpret_cast<const void*>(k_lin_tail<8>), smem);
+  {
+    const size_t smem = 4 * ((size_t)kLzLead * (kLzO + 1) + (size_t)kLzLead * p.r);
+    dim3 grid((unsigned)((p.Dout + kLzO - 1) / kLzO), (unsigned)p.nsplit);
+    cudaError_t e;
+    if (p.r <= 32) {
+      e = opt_in_smem(reinterpret_cast<const void*>(k_lin_z4<2>), smem);
+      if (e != cudaSuccess) return e;
+      k_lin_z4<2><<<grid, 256, smem, st>>>(p);
+    } else if (p.r <= 64) {
+      e = opt_in_smem(reinterpret_cast<const void*>(k_lin_z4<4>), smem);
+      if (e != cudaSuccess) return e;
+      k_lin_z4<4><<<grid, 256, smem, st>>>(p);
+    } else {
+      e = opt_in_smem(reinterpret_cast<const void*>(k_lin_z4<8>), smem);
+      if (e != cudaSuccess) return e;
+      k_lin_z4<8><<<grid, 256, smem, st>>>(p);
+    }
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    k_lin_tail<8><<<grid, 256, smem, st>>>(p);
-  } else if (p.r <= 64) {
-    e = opt_in_smem(reinterpret_cast<const void*>(k_lin_tail<16>), smem);
-    if (e != cudaSuccess) return e;
-    k_lin_tail<16><<<grid, 256, smem, st>>>(p);
-  } else {
-    e = opt_in_smem(reinterpret_cast<const void*>(k_lin_tail<32>), smem);
-    if (e != cudaSuccess) return e;
-    k_lin_tail<32><<<grid, 256, smem, st>>>(p);
   }
+  const size_t smem = 4 * (size_t)(kLtO + kLtD) * PR;
+  dim3 grid((unsigned)((p.Dout + kLtO - 1) / kLtO), (unsigned)((p.Din + kLtD - 1) / kLtD));
+  cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_lin_tail), smem);
+  if (e != cudaSuccess) return e;
+  k_lin_tail<<<grid, 256, smem, st>>>(p);
   return cudaGetLastError();
 }
 
