@@ -118,7 +118,7 @@ void layout_compress(asi_plan* pl) {
   for (int m = 0; m < pl->nd; ++m)
     if (pl->fiber[m] && fiber2_supported(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16)) {
       pl->fiber2[m] = true;
-      pl->fiber_grid[m] = fiber2_grid(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I);
+      pl->fiber_grid[m] = fiber2_grid(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16);
     }
   int64_t vmax = 0;
   if (!pl->fast_compress)
@@ -464,7 +464,7 @@ cudaError_t stream_modeprod(const asi_plan* pl, const ModeProdArgs& a, bool x_bf
   f.O = a.O; f.I = a.I; f.a = (int)a.a; f.r = a.n_out;
   f.n_tiles = fiber2_tiles(a.O, a.I);
   f.project_only = 1;
-  return launch_fiber2(f, fiber2_grid(a.O, a.a, a.I), x_bf16, st);
+  return launch_fiber2(f, fiber2_grid(a.O, a.a, a.I, a.n_out, x_bf16), x_bf16, st);
 }
 
 // Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).

@@ -298,8 +298,8 @@ bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
 int64_t fiber2_tiles(int64_t O, int64_t I) { return O * ((I + kF2TQ - 1) / kF2TQ); }
 
 // CTAs (= partials of P) of the kernel launch_fiber2 picks: the register kernel for short fibers
-int fiber2_grid(int64_t O, int64_t a, int64_t I) {
-  if (fiber_reg_supported(O, a, I, 8)) return fiber_reg_grid(O, a, I);
+int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
+  if (fiber_reg_supported(O, a, I, r, bf16)) return fiber_reg_grid(O, a, I, r, bf16);
   return (int)std::min<int64_t>(fiber2_tiles(O, I), 296);
 }
 
@@ -313,7 +313,7 @@ static cudaError_t launch_fiber2_t(const Fiber2Args& p, int grid, size_t smem, c
 
 cudaError_t launch_fiber2(const Fiber2Args& p0, int grid, bool bf16, cudaStream_t st) {
   Fiber2Args p = p0;
-  if (fiber_reg_supported(p.O, p.a, p.I, p.r)) return launch_fiber_reg(p, grid, bf16, st);
+  if (fiber_reg_supported(p.O, p.a, p.I, p.r, bf16)) return launch_fiber_reg(p, grid, bf16, st);
   const int rw = fiber2_rows_per_group(p.a), nj = p.r <= 4 ? 4 : 8;
   p.nstage = fiber2_stages(p.a, nj, bf16);
   const size_t smem = fiber2_smem(p.a, rw, nj, p.nstage, bf16);

@@ -5,7 +5,6 @@
 //                      (Algorithm 1, core update).  One thread per column leaves such a product on a handful
 //                      of CTAs walking the mode serially; here a CTA stages X(o, :, i-chunk) and B in shared
 //                      memory and its threads share the outputs (j, i).
-//   k_fiber_reg      : the two products of a mode with a short fiber (a <= 32), through registers only.
 //   k_lin_z4, k_lin_tail : the end of the linear backward (Sec. 3.1 footnote, derived steps L2-L3):
 //                        Z4[o][k] = sum_{l1,l2} Z(l1, l2, o) core[l1][l2][k],   dW[o][d] = sum_k Z4[o][k] U[d][k].
 //                      k_lin_z4 forms Z4 once (16 output rows per CTA, the leading indices shared between up to
@@ -22,7 +21,6 @@ namespace asi {
 
 namespace {
 constexpr int kStageThreads = 256;
-constexpr int kFrThreads = 256;
 constexpr int kLtO = 64, kLtD = 128;
 constexpr int kLzO = 16, kLzLead = 64;
 }  // namespace
@@ -99,188 +97,6 @@ cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem
   const int64_t nic = (p.I + ichunk - 1) / ichunk;
   k_modeprod_stage<<<(unsigned)(p.O * nic), kStageThreads, smem, st>>>(p, ichunk);
   return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------------------------
-// k_fiber_reg: both products of a mode with a SHORT fiber (a <= 32: the batch mode of a token tensor), or
-// with project_only the mode product alone, streamed through registers.  A lane owns four neighbouring
-// columns of the unfolding and eight rows; KS lanes (a <= 8 KS) share a column quad and add their partial
-// V with shuffles, so no tile is staged and nothing meets in shared memory until the CTA's final sum of P.
-// ---------------------------------------------------------------------------------------------
-template <typename TX> struct RawQuad;
-template <> struct RawQuad<float> {
-  float4 v;
-  __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
-  __device__ __forceinline__ void get(float (&x)[4], bool on) const {
-    x[0] = on ? v.x : 0.f; x[1] = on ? v.y : 0.f; x[2] = on ? v.z : 0.f; x[3] = on ? v.w : 0.f;
-  }
-};
-template <> struct RawQuad<__nv_bfloat16> {
-  uint2 v;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint2*>(p)); }
-  __device__ __forceinline__ void get(float (&x)[4], bool on) const {
-    const uint32_t a = on ? v.x : 0u, b = on ? v.y : 0u;
-    x[0] = __uint_as_float(a << 16); x[1] = __uint_as_float(a & 0xffff0000u);
-    x[2] = __uint_as_float(b << 16); x[3] = __uint_as_float(b & 0xffff0000u);
-  }
-};
-
-template <int NJ, int KS, typename TX>
-__global__ void __launch_bounds__(kFrThreads, 1) k_fiber_reg(Fiber2Args p) {
-  constexpr int QW = 32 / KS;                        // column quads per warp
-  constexpr int NW = kFrThreads / 32;
-  __shared__ __align__(16) float Us[8 * KS * NJ];    // rows >= a and columns >= r are zero
-  __shared__ float red[NW][8 * KS * NJ];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int ks = lane / QW, cq = lane - ks * QW;
-  const int a = p.a, r = p.r, r0 = 8 * ks;
-  for (int e = tid; e < 8 * KS * NJ; e += kFrThreads) {
-    const int k = e / NJ, j = e - k * NJ;
-    Us[e] = (k < a && j < r) ? p.U[(int64_t)k * p.ldu + j] : 0.f;
-  }
-  __syncthreads();
-  const int Iq = (int)(p.I >> 2);
-  const int total = (int)p.O * Iq;                   // column quads of the unfolding (< 2^31, checked by the host)
-  const int stride = gridDim.x * NW * QW;
-  const TX* X = static_cast<const TX*>(p.X);
-  int64_t roff[8];                                   // rows past the end re-read row a - 1 (their factor row is 0)
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk) roff[kk] = (int64_t)((r0 + kk < a) ? r0 + kk : a - 1) * p.I;
-  float accP[8][NJ];
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk)
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) accP[kk][j] = 0.f;
-
-  int gbase = (blockIdx.x * NW + warp) * QW;         // warp-uniform: the loop test is the same in every lane
-  RawQuad<TX> cur[8], nxt[8];
-  int o_c = 0, iq_c = 0;
-  bool on_c = false;
-  if (gbase < total) {
-    const int g = gbase + cq;
-    on_c = g < total;
-    const int gl = on_c ? g : total - 1;
-    o_c = gl / Iq; iq_c = gl - o_c * Iq;
-    const TX* src = X + (int64_t)o_c * a * p.I + 4 * (int64_t)iq_c;
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) cur[kk].load(src + roff[kk]);
-  }
-  while (gbase < total) {
-    // the next quad's rows are requested before this one's arithmetic (always from a valid address)
-    const int gnb = gbase + stride;
-    const int gn = gnb + cq;
-    const bool on_n = gnb < total && gn < total;
-    const int gl = on_n ? gn : total - 1;
-    const int o_n = gl / Iq, iq_n = gl - o_n * Iq;
-    {
-      const TX* src = X + (int64_t)o_n * a * p.I + 4 * (int64_t)iq_n;
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) nxt[kk].load(src + roff[kk]);
-    }
-    float V[4][NJ];
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-#pragma unroll
-      for (int j = 0; j < NJ; ++j) V[c][j] = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      float x[4];
-      cur[kk].get(x, on_c);
-#pragma unroll
-      for (int j4 = 0; j4 < NJ; j4 += 4) {
-        const float4 u = *reinterpret_cast<const float4*>(&Us[(r0 + kk) * NJ + j4]);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          V[c][j4 + 0] = fmaf(x[c], u.x, V[c][j4 + 0]);
-          V[c][j4 + 1] = fmaf(x[c], u.y, V[c][j4 + 1]);
-          V[c][j4 + 2] = fmaf(x[c], u.z, V[c][j4 + 2]);
-          V[c][j4 + 3] = fmaf(x[c], u.w, V[c][j4 + 3]);
-        }
-      }
-    }
-#pragma unroll
-    for (int s = QW; s < 32; s *= 2)                 // the KS row groups of a column quad
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int j = 0; j < NJ; ++j) V[c][j] += __shfl_xor_sync(0xffffffffu, V[c][j], s);
-    if (p.project_only) {
-      if (on_c) {
-        float* dst = p.Y + (int64_t)o_c * p.y_so + 4 * (int64_t)iq_c;
-#pragma unroll
-        for (int j = 0; j < NJ; ++j)
-          if (j < r && (j % KS) == ks)
-            *reinterpret_cast<float4*>(dst + (int64_t)j * p.y_sj) = make_float4(V[0][j], V[1][j], V[2][j], V[3][j]);
-      }
-    } else {
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        float x[4];
-        cur[kk].get(x, on_c);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int j = 0; j < NJ; ++j) accP[kk][j] = fmaf(x[c], V[c][j], accP[kk][j]);
-      }
-    }
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) cur[kk] = nxt[kk];
-    o_c = o_n; iq_c = iq_n; on_c = on_n;
-    gbase = gnb;
-  }
-  if (p.project_only) return;
-  // P of this CTA: over the lanes of a row group, then over the warps
-#pragma unroll
-  for (int kk = 0; kk < 8; ++kk)
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) {
-      float v = accP[kk][j];
-#pragma unroll
-      for (int s = 1; s < QW; s *= 2) v += __shfl_xor_sync(0xffffffffu, v, s);
-      if (cq == 0) red[warp][(r0 + kk) * NJ + j] = v;
-    }
-  __syncthreads();
-  for (int e = tid; e < 8 * KS * NJ; e += kFrThreads) {
-    const int k = e / NJ, j = e - k * NJ;
-    if (k >= a || j >= r) continue;
-    float v = 0.f;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) v += red[w][e];
-    p.Pp[((int64_t)blockIdx.x * a + k) * r + j] = v;
-  }
-}
-
-bool fiber_reg_supported(int64_t O, int64_t a, int64_t I, int r) {
-  return r >= 1 && r <= 8 && a >= 1 && a <= 32 && I % 4 == 0 && O * (I / 4) < (1ll << 30);
-}
-
-static int fiber_reg_ks(int a) { return a <= 8 ? 1 : a <= 16 ? 2 : 4; }
-
-int fiber_reg_grid(int64_t O, int64_t a, int64_t I) {
-  const int qw = 32 / fiber_reg_ks((int)a);
-  const int64_t per_cta = (int64_t)(kFrThreads / 32) * qw;
-  return (int)std::min<int64_t>(148, (O * (I / 4) + per_cta - 1) / per_cta);
-}
-
-template <int NJ, int KS>
-static cudaError_t launch_fiber_reg_t(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st) {
-  if (bf16) k_fiber_reg<NJ, KS, __nv_bfloat16><<<grid, kFrThreads, 0, st>>>(p);
-  else k_fiber_reg<NJ, KS, float><<<grid, kFrThreads, 0, st>>>(p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_fiber_reg(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st) {
-  const double xbytes = (double)p.O * p.a * p.I * (bf16 ? 2 : 4);
-  ProfScope prof(p.project_only ? ASI_K_MODEPROD : ASI_K_EXPAND, st, xbytes);
-  const int ks = fiber_reg_ks(p.a);
-  if (p.r <= 4) {
-    if (ks == 1) return launch_fiber_reg_t<4, 1>(p, grid, bf16, st);
-    if (ks == 2) return launch_fiber_reg_t<4, 2>(p, grid, bf16, st);
-    return launch_fiber_reg_t<4, 4>(p, grid, bf16, st);
-  }
-  if (ks == 1) return launch_fiber_reg_t<8, 1>(p, grid, bf16, st);
-  if (ks == 2) return launch_fiber_reg_t<8, 2>(p, grid, bf16, st);
-  return launch_fiber_reg_t<8, 4>(p, grid, bf16, st);
 }
 
 // ---------------------------------------------------------------------------------------------
