@@ -268,6 +268,7 @@ bool lin_tail_supported(int r);
 int lin_tail_nsplit(int nlead, int64_t Dout);
 cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st);
 bool modeprod_stage_fits(const ModeProdArgs& p, int* ichunk, size_t* smem);
+int modeprod_stage_ksp(int64_t a);
 cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem, cudaStream_t st);
 bool plane2_supported(int S, int64_t n_planes, int r3, int r4);
 int plane2_grid(int S, int64_t n_planes, int max_ctas);

@@ -3,14 +3,16 @@
 //   k_modeprod_stage : a mode product Y(o, j, i) = sum_k X(o, k, i) B(k, j) whose tensor has FEW columns
 //                      (O * I small) but a long contracted mode -- the later core products of a token layer
 //                      (Algorithm 1, core update).  One thread per column leaves such a product on a handful
-//                      of CTAs walking the mode serially; here a CTA stages X(o, :, i-chunk) and B in shared
-//                      memory and its threads share the outputs (j, i).
+//                      of CTAs walking the mode serially; here a cluster of up to eight CTAs owns X(o, :, i-chunk):
+//                      each stages a slab of the mode's rows and of B in shared memory, its threads share the
+//                      outputs (j, i), and the slabs' partial outputs meet in distributed shared memory.
 //   k_lin_z4, k_lin_tail : the end of the linear backward (Sec. 3.1 footnote, derived steps L2-L3):
 //                        Z4[o][k] = sum_{l1,l2} Z(l1, l2, o) core[l1][l2][k],   dW[o][d] = sum_k Z4[o][k] U[d][k].
 //                      k_lin_z4 forms Z4 once (16 output rows per CTA, the leading indices shared between up to
 //                      eight CTAs that each write their own share -- no atomics, the sum order is fixed);
 //                      k_lin_tail adds the shares and expands 64 x 128 tiles of dW in 8 x 4 register tiles with
 //                      coalesced stores.  dW is written exactly once.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -25,16 +27,26 @@ constexpr int kLtO = 64, kLtD = 128;
 constexpr int kLzO = 16, kLzLead = 64;
 }  // namespace
 
-__global__ void __launch_bounds__(kStageThreads) k_modeprod_stage(ModeProdArgs p, int ichunk) {
+// The CTAs of a cluster share one (o, i-chunk): CTA `rank` contracts the rows [rank * aslab, ..) of the mode and
+// leaves its partial outputs in its own shared memory; rank 0 adds them in rank order through distributed shared
+// memory and writes Y.  Both cluster barriers are reached by every thread of every CTA.
+__global__ void __launch_bounds__(kStageThreads) k_modeprod_stage(ModeProdArgs p, int ichunk, int ksp, int aslab) {
   extern __shared__ __align__(16) float ms_smem[];
-  const int a = (int)p.a, n = p.n_out;
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int n = p.n_out;
   const int nic = (int)((p.I + ichunk - 1) / ichunk);
-  const int64_t o = blockIdx.x / nic;
-  const int i0 = (int)(blockIdx.x % nic) * ichunk;
+  const int rank = (int)(blockIdx.x % ksp);
+  const int64_t tile = blockIdx.x / ksp;
+  const int64_t o = tile / nic;
+  const int i0 = (int)(tile % nic) * ichunk;
   const int ni = (int)((p.I - i0 < ichunk) ? (p.I - i0) : ichunk);
-  float* Xs = ms_smem;                       // [a][ichunk]
-  float* Bs = Xs + (size_t)a * ichunk;       // [a][n]
-  const float* X = reinterpret_cast<const float*>(p.X) + o * p.a * p.I + i0;
+  const int k0 = rank * aslab;
+  const int a = (int)((p.a - k0 < aslab) ? ((p.a > k0) ? p.a - k0 : 0) : aslab);   // rows of this CTA
+  float* Xs = ms_smem;                            // [aslab][ichunk]
+  float* Bs = Xs + (size_t)aslab * ichunk;        // [aslab][n]
+  float* part = Bs + (size_t)aslab * n;           // [n][ichunk]
+  const float* X = reinterpret_cast<const float*>(p.X) + (o * p.a + k0) * p.I + i0;
   const int tid = threadIdx.x;
   // all loads of a batch first, then the stores (a load next to the store of its value waits for it)
   for (int e0 = 0; e0 < a * ichunk; e0 += 8 * kStageThreads) {
@@ -57,7 +69,7 @@ __global__ void __launch_bounds__(kStageThreads) k_modeprod_stage(ModeProdArgs p
     for (int u = 0; u < 8; ++u) {
       const int e = e0 + tid + u * kStageThreads;
       const int k = e / n, j = e - k * n;
-      v[u] = p.B[(e < a * n) ? (int64_t)k * p.ldb_k + (int64_t)j * p.ldb_j : 0];
+      v[u] = p.B[(e < a * n) ? (int64_t)(k0 + k) * p.ldb_k + (int64_t)j * p.ldb_j : 0];
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
@@ -75,19 +87,37 @@ __global__ void __launch_bounds__(kStageThreads) k_modeprod_stage(ModeProdArgs p
       s1 = fmaf(Xs[(k + 1) * ichunk + i], Bs[(k + 1) * n + j], s1);
     }
     if (k < a) s0 = fmaf(Xs[k * ichunk + i], Bs[k * n + j], s0);
-    p.Y[o * p.so + (int64_t)j * p.sj + (int64_t)(i0 + i) * p.si] = s0 + s1;
+    part[j * ichunk + i] = s0 + s1;
   }
+  cluster.sync();
+  if (rank == 0) {
+    for (int e = tid; e < n * ni; e += kStageThreads) {
+      const int j = e / ni, i = e - j * ni;
+      float s = part[j * ichunk + i];
+      for (int q = 1; q < ksp; ++q) s += cluster.map_shared_rank(part, q)[j * ichunk + i];
+      p.Y[o * p.so + (int64_t)j * p.sj + (int64_t)(i0 + i) * p.si] = s;
+    }
+  }
+  cluster.sync();                                 // the partials stay alive until rank 0 has read them
 }
 
 bool modeprod_stage_fits(const ModeProdArgs& p, int* ichunk, size_t* smem) {
   if (p.a < 64 || p.a > 8192 || p.O * p.I > 8192 || p.n_out > 128) return false;
+  const int ksp = modeprod_stage_ksp(p.a);
+  const int64_t aslab = (p.a + ksp - 1) / ksp;
   int ic = (int)(p.I < 64 ? p.I : 64);
-  while (ic > 1 && (size_t)p.a * (ic + p.n_out) * 4 > 160 * 1024) ic = (ic + 1) / 2;
-  const size_t need = (size_t)p.a * (ic + p.n_out) * 4;
-  if (need > 160 * 1024) return false;
+  auto need_of = [&](int c) { return ((size_t)aslab * (c + p.n_out) + (size_t)p.n_out * c) * 4; };
+  while (ic > 1 && need_of(ic) > 160 * 1024) ic = (ic + 1) / 2;
+  if (need_of(ic) > 160 * 1024) return false;
   *ichunk = ic;
-  *smem = need;
+  *smem = need_of(ic);
   return true;
+}
+
+int modeprod_stage_ksp(int64_t a) {
+  int k = 1;
+  while (k < 8 && a / (2 * k) >= 32) k *= 2;      // at least 32 rows per CTA, at most the portable cluster size
+  return k;
 }
 
 cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem, cudaStream_t st) {
@@ -95,8 +125,21 @@ cudaError_t launch_modeprod_stage(const ModeProdArgs& p, int ichunk, size_t smem
   cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_modeprod_stage), smem);
   if (e != cudaSuccess) return e;
   const int64_t nic = (p.I + ichunk - 1) / ichunk;
-  k_modeprod_stage<<<(unsigned)(p.O * nic), kStageThreads, smem, st>>>(p, ichunk);
-  return cudaGetLastError();
+  const int ksp = modeprod_stage_ksp(p.a);
+  const int aslab = (int)((p.a + ksp - 1) / ksp);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(p.O * nic * ksp));
+  cfg.blockDim = dim3(kStageThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)ksp;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_modeprod_stage, p, ichunk, ksp, aslab);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -116,31 +159,46 @@ __global__ void __launch_bounds__(256) k_lin_z4(LinTailArgs p) {
   const int per = ((nlead + p.nsplit - 1) / p.nsplit + kLzLead - 1) / kLzLead * kLzLead;
   const int lbeg = blockIdx.y * per, lend = (lbeg + per < nlead) ? lbeg + per : nlead;
   const int po = tid & (kLzO - 1), kg = tid >> 4;
+  constexpr int NS = 4 * NQ;                         // core values of a chunk per thread: 64 r / 256 <= 4 NQ
   float acc[NQ];
 #pragma unroll
   for (int q = 0; q < NQ; ++q) acc[q] = 0.f;
-  for (int l0 = lbeg; l0 < lend; l0 += kLzLead) {
+  float vz[4], vs[NS];
+  // the values of the chunk that starts at l0, into registers (loads only: nothing here uses them)
+  auto fetch = [&](int l0) {
     const int nl = (lend - l0 < kLzLead) ? lend - l0 : kLzLead;
-    float v[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {                    // 64 x 16 values, four per thread, loads first
+    for (int u = 0; u < 4; ++u) {                    // 64 x 16 values, four per thread
       const int e = tid + u * 256;
       int l, o;
       if (p.lead_fastest) { o = e / kLzLead; l = e - o * kLzLead; } else { l = e >> 4; o = e & (kLzO - 1); }
       const int lead = l0 + l, l1 = lead / p.L2, l2 = lead - l1 * p.L2;
       const bool on = l < nl && o0 + o < p.Dout;
-      v[u] = p.Z[on ? (int64_t)l1 * p.s1 + (int64_t)l2 * p.s2 + (int64_t)(o0 + o) * p.so : 0];
+      vz[u] = p.Z[on ? (int64_t)l1 * p.s1 + (int64_t)l2 * p.s2 + (int64_t)(o0 + o) * p.so : 0];
     }
+#pragma unroll
+    for (int u = 0; u < NS; ++u) {
+      const int e = tid + u * 256;
+      vs[u] = p.core[(e < nl * r) ? (int64_t)l0 * r + e : 0];
+    }
+  };
+  if (lbeg < lend) fetch(lbeg);
+  for (int l0 = lbeg; l0 < lend; l0 += kLzLead) {
+    const int nl = (lend - l0 < kLzLead) ? lend - l0 : kLzLead;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int e = tid + u * 256;
       int l, o;
       if (p.lead_fastest) { o = e / kLzLead; l = e - o * kLzLead; } else { l = e >> 4; o = e & (kLzO - 1); }
-      Zc[l * (kLzO + 1) + o] = (l < nl && o0 + o < p.Dout) ? v[u] : 0.f;
+      Zc[l * (kLzO + 1) + o] = (l < nl && o0 + o < p.Dout) ? vz[u] : 0.f;
     }
-    for (int e = tid; e < kLzLead * r; e += 256)
-      Sc[e] = (e < nl * r) ? p.core[(int64_t)l0 * r + e] : 0.f;
+#pragma unroll
+    for (int u = 0; u < NS; ++u) {
+      const int e = tid + u * 256;
+      if (e < kLzLead * r) Sc[e] = (e < nl * r) ? vs[u] : 0.f;
+    }
     __syncthreads();
+    if (l0 + kLzLead < lend) fetch(l0 + kLzLead);    // the next chunk travels while this one is used
 #pragma unroll 4
     for (int l = 0; l < kLzLead; ++l) {
       const float z = Zc[l * (kLzO + 1) + po];
@@ -238,7 +296,7 @@ bool lin_tail_supported(int r) { return r >= 1 && r <= 128; }
 
 int lin_tail_nsplit(int nlead, int64_t Dout) {
   const int64_t tiles = (Dout + kLzO - 1) / kLzO;
-  int64_t ns = 296 / (tiles > 0 ? tiles : 1);
+  int64_t ns = 592 / (tiles > 0 ? tiles : 1);       // about four CTAs per SM
   const int64_t cap = (nlead + kLzLead - 1) / kLzLead;      // at least one chunk of leads per share
   if (ns > cap) ns = cap;
   if (ns > 8) ns = 8;
