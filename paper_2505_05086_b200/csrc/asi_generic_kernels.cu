@@ -878,22 +878,29 @@ __global__ void __launch_bounds__(256) k_qr_gram(QRArgs args) {
   double acc[kPer];
 #pragma unroll
   for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
-  for (int s0 = 0; s0 < M.nsplit; s0 += ssub) {
-    float t[kPer];
+  // four batches of 16 loads are issued before the first is used: with many splits and a full chunk (one
+  // split per batch) the loop is otherwise one memory round trip per split
+  constexpr int kBatch = 4;
+  for (int s0 = 0; s0 < M.nsplit; s0 += kBatch * ssub) {
+    float t[kBatch][kPer];
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-      const int idx = tid + (q & (ethr - 1)) * 256;
-      const int s = s0 + (q >> lg);
-      const bool on = idx < nval && s < M.nsplit;
-      // Every load is issued, from a clamped address when off, and nothing here touches its
-      // result: a use or a condition next to a load makes the following loads wait for it.
-      t[q] = __ldcg(M.Pp + (on ? s * sstride + base + idx : 0));
-    }
+    for (int b = 0; b < kBatch; ++b)
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-      const bool on = tid + (q & (ethr - 1)) * 256 < nval && s0 + (q >> lg) < M.nsplit;
-      acc[q] += on ? (double)t[q] : 0.0;
-    }
+      for (int q = 0; q < kPer; ++q) {
+        const int idx = tid + (q & (ethr - 1)) * 256;
+        const int s = s0 + b * ssub + (q >> lg);
+        const bool on = idx < nval && s < M.nsplit;
+        // Every load is issued, from a clamped address when off, and nothing here touches its
+        // result: a use or a condition next to a load makes the following loads wait for it.
+        t[b][q] = __ldcg(M.Pp + (on ? s * sstride + base + idx : 0));
+      }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+      for (int q = 0; q < kPer; ++q) {
+        const bool on = tid + (q & (ethr - 1)) * 256 < nval && s0 + b * ssub + (q >> lg) < M.nsplit;
+        acc[q] += on ? (double)t[b][q] : 0.0;
+      }
   }
 #pragma unroll
   for (int h = kPer / 2; h >= 1; h >>= 1)
@@ -949,7 +956,7 @@ __global__ void __launch_bounds__(256) k_qr_gsum(QRArgs args) {
   if (M.r > kQRMaxRank || e >= rr || (e % M.r) < (e / M.r)) return;
   const double* G = M.Gp + e;
   double acc = 0.0;
-#pragma unroll 8
+#pragma unroll 16
   for (int cc = 0; cc < M.nchunk; ++cc) acc += __ldcg(G + (int64_t)cc * rr);
   M.Gp[e] = acc;
 }
