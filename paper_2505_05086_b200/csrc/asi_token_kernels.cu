@@ -216,10 +216,13 @@ __global__ void __launch_bounds__(256) k_lin_z4(LinTailArgs p) {
   }
 }
 
-// dW[o][d] = sum_k Z4[o][k] U[d][k], Z4 = the sum of the nsplit shares: 64 x 128 tile per CTA, 8 x 4 per thread
-__global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p) {
+// dW[o][d] = sum_k Z4[o][k] U[d][k], Z4 = the sum of the nsplit shares: 64 x 128 tile per CTA, 8 x 4 per thread.
+// Rows of Z4 and of U sit in shared memory with a pitch of 4 * (odd number) floats and zeros up to it, so the
+// k loop reads four k at a time with 16-byte loads (the 8 Z4 rows of a warp are broadcasts; the 32 lanes' U
+// rows fall in distinct banks): 12 loads per 128 multiply-adds.
+__global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p, int PR) {
   extern __shared__ __align__(16) float lt_smem[];
-  const int r = p.r, PR = r | 1;                     // odd pitch: conflict-free reads down a column of rows
+  const int r = p.r;
   float* Z4s = lt_smem;                              // [64][PR]
   float* Us = Z4s + kLtO * PR;                       // [128][PR]
   const int tid = threadIdx.x, lane = tid & 31;
@@ -228,36 +231,41 @@ __global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p) {
   const int nd = (p.Din - d0 < kLtD) ? p.Din - d0 : kLtD;
   const float* zsrc = p.Z4p + (int64_t)o0 * r;
   const int64_t zstep = (int64_t)p.Dout * r;
-  for (int e0 = 0; e0 < kLtO * r; e0 += 4 * 256) {
+  for (int e0 = 0; e0 < kLtO * PR; e0 += 4 * 256) {  // e = (o, k) over the padded pitch
     float v[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int s = 0; s < p.nsplit; ++s) {
+    int src[4];
+    bool on[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + tid + u * 256, o = e / PR, k = e - o * PR;
+      on[u] = e < kLtO * PR && o < no && k < r;
+      src[u] = on[u] ? o * r + k : 0;
+    }
+    for (int sp = 0; sp < p.nsplit; ++sp) {
       float t[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int e = e0 + tid + u * 256;
-        t[u] = zsrc[s * zstep + (e < no * r ? e : 0)];
-      }
+      for (int u = 0; u < 4; ++u) t[u] = zsrc[sp * zstep + src[u]];
 #pragma unroll
       for (int u = 0; u < 4; ++u) v[u] += t[u];
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int e = e0 + tid + u * 256, o = e / r;
-      if (e < kLtO * r) Z4s[o * PR + (e - o * r)] = (e < no * r) ? v[u] : 0.f;
+      const int e = e0 + tid + u * 256;
+      if (e < kLtO * PR) Z4s[e] = on[u] ? v[u] : 0.f;
     }
   }
   const float* usrc = p.U + (int64_t)d0 * r;
-  for (int e0 = 0; e0 < kLtD * r; e0 += 8 * 256) {
+  for (int e0 = 0; e0 < kLtD * PR; e0 += 8 * 256) {
     float v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int e = e0 + tid + u * 256;
-      v[u] = usrc[e < nd * r ? e : 0];
+      const int e = e0 + tid + u * 256, d = e / PR, k = e - d * PR;
+      v[u] = usrc[(e < kLtD * PR && d < nd && k < r) ? d * r + k : 0];
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int e = e0 + tid + u * 256, d = e / r;
-      if (e < kLtD * r) Us[d * PR + (e - d * r)] = (e < nd * r) ? v[u] : 0.f;
+      const int e = e0 + tid + u * 256, d = e / PR, k = e - d * PR;
+      if (e < kLtD * PR) Us[e] = (d < nd && k < r) ? v[u] : 0.f;
     }
   }
   __syncthreads();
@@ -268,17 +276,23 @@ __global__ void __launch_bounds__(256) k_lin_tail(LinTailArgs p) {
   for (int x = 0; x < 8; ++x)
 #pragma unroll
     for (int y = 0; y < 4; ++y) out[x][y] = 0.f;
-#pragma unroll 2
-  for (int k = 0; k < r; ++k) {
-    float zz[8], uu[4];
+  const float* zrow = Z4s + 8 * to * PR;
+  const float* urow = Us + lane * PR;
+  for (int k = 0; k < PR; k += 4) {
+    float4 zz[8], uu[4];
 #pragma unroll
-    for (int x = 0; x < 8; ++x) zz[x] = Z4s[(8 * to + x) * PR + k];
+    for (int x = 0; x < 8; ++x) zz[x] = *reinterpret_cast<const float4*>(zrow + x * PR + k);
 #pragma unroll
-    for (int y = 0; y < 4; ++y) uu[y] = Us[(lane + 32 * y) * PR + k];
+    for (int y = 0; y < 4; ++y) uu[y] = *reinterpret_cast<const float4*>(urow + 32 * y * PR + k);
 #pragma unroll
     for (int x = 0; x < 8; ++x)
 #pragma unroll
-      for (int y = 0; y < 4; ++y) out[x][y] = fmaf(zz[x], uu[y], out[x][y]);
+      for (int y = 0; y < 4; ++y) {
+        out[x][y] = fmaf(zz[x].x, uu[y].x, out[x][y]);
+        out[x][y] = fmaf(zz[x].y, uu[y].y, out[x][y]);
+        out[x][y] = fmaf(zz[x].z, uu[y].z, out[x][y]);
+        out[x][y] = fmaf(zz[x].w, uu[y].w, out[x][y]);
+      }
   }
 #pragma unroll
   for (int x = 0; x < 8; ++x) {
@@ -304,7 +318,8 @@ int lin_tail_nsplit(int nlead, int64_t Dout) {
 }
 
 cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st) {
-  const int PR = p.r | 1;
+  int PR = (p.r + 3) / 4 * 4;                     // pitch: 4 * (odd number) floats
+  if ((PR / 4) % 2 == 0) PR += 4;
   ProfScope prof(ASI_K_MODEPROD, st, 4.0 * ((double)p.Dout * p.Din + (double)p.L1 * p.L2 * p.Dout));
   {
     const size_t smem = 4 * ((size_t)kLzLead * (kLzO + 1) + (size_t)kLzLead * p.r);
@@ -330,7 +345,7 @@ cudaError_t launch_lin_tail(const LinTailArgs& p, cudaStream_t st) {
   dim3 grid((unsigned)((p.Dout + kLtO - 1) / kLtO), (unsigned)((p.Din + kLtD - 1) / kLtD));
   cudaError_t e = opt_in_smem(reinterpret_cast<const void*>(k_lin_tail), smem);
   if (e != cudaSuccess) return e;
-  k_lin_tail<<<grid, 256, smem, st>>>(p);
+  k_lin_tail<<<grid, 256, smem, st>>>(p, PR);
   return cudaGetLastError();
 }
 
