@@ -126,6 +126,21 @@ asi_status_t asi_compress(const asi_plan_t* plan, const void* act, const float* 
 asi_status_t asi_init_factors(const asi_plan_t* plan, const void* act, const float* omega,
                               float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
 
+/* The same cold start with the Gaussian test matrices drawn by the library (Algorithm 1, t = 0: "V ~ N(0, 1)";
+ * the paper names no generator).  Omega_m is the first b_m r_m values of the counter-based stream
+ * (seed, stream = m): Philox4x32-10 with key = seed and counter = (group index, stream, 0), a word x mapped to
+ * u = ((x >> 9) + 0.5) 2^-23, pairs of words through Box-Muller in fp32; element e of a stream is value e mod 4
+ * of group e div 4.  The matrices are drawn mode by mode into the workspace, so the caller holds no Omega and
+ * the scratch grows by the largest b_m r_m floats only.  Same seed, same plan: same factors.
+ *   ws  device scratch of at least asi_init_seeded_ws_bytes(plan). */
+size_t asi_init_seeded_ws_bytes(const asi_plan_t* plan);
+asi_status_t asi_init_factors_seeded(const asi_plan_t* plan, const void* act, uint64_t seed, float* U_new,
+                                     float* core, void* ws, size_t ws_bytes, void* stream);
+/* The generator by itself: out[0..n) = the first n values of the N(0, 1) stream (seed, stream_id) (device fp32),
+ * and the raw words of its first n_groups groups (device uint32, 4 per group, 16-byte aligned). */
+asi_status_t asi_gaussian_stream(uint64_t seed, uint32_t stream_id, int64_t n, float* out, void* stream);
+asi_status_t asi_philox_words(uint64_t seed, uint32_t stream_id, int64_t n_groups, uint32_t* out, void* stream);
+
 /* The layers one training step handles together, in one call each way: Algorithm 1 is run for every
  * fine-tuned layer at every step (Sec. 4 fine-tunes the last two to four layers), and the backward pass
  * needs every layer's weight gradient.  Arrays of n entries, entry i as in asi_compress / asi_*_wgrad;

@@ -30,7 +30,8 @@ ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT = 1, 2
 
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
-    "asi_init_factors", "asi_compress_batched", "asi_wgrad_batched",
+    "asi_init_factors", "asi_init_seeded_ws_bytes", "asi_init_factors_seeded", "asi_gaussian_stream",
+    "asi_philox_words", "asi_compress_batched", "asi_wgrad_batched",
     "asi_spectrum_ws_bytes", "asi_mode_spectrum", "asi_pick_ranks", "asi_perplexity_ws_bytes", "asi_perplexity",
     "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host_arena_bytes", "asi_step_host", "asi_step_host_status",
     "asi_poll_status", "asi_launch_count", "asi_status_string", "asi_profile_begin",
@@ -81,6 +82,11 @@ def lib():
     L.asi_compress.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     L.asi_compress_static_ws.argtypes = [vp, vp, vp, vp, vp, vp]
     L.asi_init_factors.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    L.asi_init_seeded_ws_bytes.argtypes = [vp]
+    L.asi_init_seeded_ws_bytes.restype = sz
+    L.asi_init_factors_seeded.argtypes = [vp, vp, C.c_uint64, vp, vp, vp, sz, vp]
+    L.asi_gaussian_stream.argtypes = [C.c_uint64, C.c_uint32, C.c_int64, vp, vp]
+    L.asi_philox_words.argtypes = [C.c_uint64, C.c_uint32, C.c_int64, vp, vp]
     pvp, psz = C.POINTER(vp), C.POINTER(sz)
     L.asi_compress_batched.argtypes = [pvp, pvp, pvp, pvp, pvp, pvp, psz, i32, vp]
     L.asi_wgrad_batched.argtypes = [pvp, pvp, pvp, pvp, pvp, pvp, psz, i32, vp]
@@ -109,7 +115,8 @@ def lib():
     L.asi_status_string.argtypes = [i32]
     L.asi_status_string.restype = C.c_char_p
     for name in ("asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",
-                 "asi_init_factors", "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
+                 "asi_init_factors", "asi_init_factors_seeded", "asi_gaussian_stream", "asi_philox_words",
+                 "asi_conv_wgrad", "asi_linear_wgrad", "asi_step_host",
                  "asi_poll_status", "asi_step_host_status", "asi_compress_batched", "asi_wgrad_batched",
                  "asi_mode_spectrum", "asi_pick_ranks", "asi_perplexity"):
         getattr(L, name).restype = i32
@@ -192,6 +199,13 @@ class Plan:
         _check(lib().asi_init_factors(self._h, act, omega, U_new, core, ws, ws_bytes, stream),
                "asi_init_factors")
 
+    def init_seeded_ws_bytes(self):
+        return lib().asi_init_seeded_ws_bytes(self._h)
+
+    def init_factors_seeded(self, act, seed, U_new, core, ws, ws_bytes, stream=0):
+        _check(lib().asi_init_factors_seeded(self._h, act, int(seed), U_new, core, ws, ws_bytes, stream),
+               "asi_init_factors_seeded")
+
     def conv_wgrad(self, core, U, dY, dW, ws, ws_bytes, stream=0):
         _check(lib().asi_conv_wgrad(self._h, core, U, dY, dW, ws, ws_bytes, stream), "asi_conv_wgrad")
 
@@ -259,6 +273,16 @@ class Batch:
 def perplexity(dW, dW_approx, n, out, ws, ws_bytes, stream=0):
     """asi_perplexity: ||dW - dW_approx||_F into the device double `out`."""
     _check(lib().asi_perplexity(dW, dW_approx, int(n), out, ws, ws_bytes, stream), "asi_perplexity")
+
+
+def gaussian_stream(seed, stream_id, n, out, stream=0):
+    """asi_gaussian_stream: the first n values of the N(0, 1) stream (seed, stream_id) into device fp32 `out`."""
+    _check(lib().asi_gaussian_stream(int(seed), int(stream_id), int(n), out, stream), "asi_gaussian_stream")
+
+
+def philox_words(seed, stream_id, n_groups, out, stream=0):
+    """asi_philox_words: the raw words of the first n_groups groups into device uint32 `out` (4 per group)."""
+    _check(lib().asi_philox_words(int(seed), int(stream_id), int(n_groups), out, stream), "asi_philox_words")
 
 
 def perplexity_ws_bytes():

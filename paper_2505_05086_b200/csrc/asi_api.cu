@@ -946,6 +946,47 @@ asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float
   return finish_compress(pl, act, U_new, core, w, nullptr, st);
 }
 
+static size_t omega_scratch_bytes(const asi_plan* pl) {
+  int64_t mx = 0;
+  for (int m = 0; m < pl->nd; ++m) mx = std::max<int64_t>(mx, pl->mv[m].Q * pl->r[m]);
+  return align_up((size_t)mx * 4, 256);
+}
+
+size_t asi_init_seeded_ws_bytes(const asi_plan_t* pl) {
+  return pl ? align_up(pl->compress_ws, 256) + omega_scratch_bytes(pl) : 0;
+}
+
+asi_status_t asi_init_factors_seeded(const asi_plan_t* pl, const void* act, uint64_t seed, float* U_new,
+                                     float* core, void* ws, size_t ws_bytes, void* stream) {
+  if (!pl || !valid_ptr(act) || !valid_ptr(U_new) || !valid_ptr(core)) return ASI_ERR_INVALID_ARG;
+  asi_status_t s = check_ws(ws, ws_bytes, asi_init_seeded_ws_bytes(pl));
+  if (s != ASI_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  float* omega = reinterpret_cast<float*>(w + align_up(pl->compress_ws, 256));
+  if (pl->fast_compress && !pl->bf16 && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
+  ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
+  for (int m = 0; m < pl->nd; ++m) {               // one mode's Omega at a time, in the same scratch
+    ASI_CUDA(launch_fill_gaussian(seed, (uint32_t)m, pl->mv[m].Q * pl->r[m], omega, st));
+    s = expand_mode(pl, m, act, omega, w, st);
+    if (s != ASI_OK) return s;
+  }
+  return finish_compress(pl, act, U_new, core, w, nullptr, st);
+}
+
+asi_status_t asi_gaussian_stream(uint64_t seed, uint32_t stream_id, int64_t n, float* out, void* stream) {
+  if (n < 0 || (n > 0 && !valid_ptr(out))) return ASI_ERR_INVALID_ARG;
+  ASI_CUDA(launch_fill_gaussian(seed, stream_id, n, out, static_cast<cudaStream_t>(stream)));
+  return ASI_OK;
+}
+
+asi_status_t asi_philox_words(uint64_t seed, uint32_t stream_id, int64_t n_groups, uint32_t* out, void* stream) {
+  if (n_groups < 0 || (n_groups > 0 && (!valid_ptr(out) || (reinterpret_cast<uintptr_t>(out) & 15u))))
+    return ASI_ERR_INVALID_ARG;
+  ASI_CUDA(launch_philox_words(seed, stream_id, n_groups, out, static_cast<cudaStream_t>(stream)));
+  return ASI_OK;
+}
+
 asi_status_t asi_conv_wgrad(const asi_plan_t* pl, const float* core, const float* U, const void* dY,
                             float* dW, void* ws, size_t ws_bytes, void* stream) {
   if (!pl || !valid_ptr(core) || !valid_ptr(U) || !valid_ptr(dY) || !valid_ptr(dW))

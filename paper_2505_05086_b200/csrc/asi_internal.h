@@ -283,6 +283,8 @@ cudaError_t launch_conv_tail_split(const ConvTailArgs& p, float* Z4p, int nsp, c
 namespace asi {
 // rank selection aids (asi_spectrum_kernels.cu)
 size_t spectrum_ws_bytes(const struct ::asi_plan* pl);
+cudaError_t launch_philox_words(uint64_t seed, uint32_t stream, int64_t n_groups, uint32_t* out, cudaStream_t st);
+cudaError_t launch_fill_gaussian(uint64_t seed, uint32_t stream, int64_t n, float* out, cudaStream_t st);
 cudaError_t launch_mode_spectrum(const struct ::asi_plan* pl, const void* act, double* eig, double* energy, char* w,
                                  cudaStream_t st);
 cudaError_t launch_pick_ranks(const struct ::asi_plan* pl, const double* eig, const double* energy, double eps,

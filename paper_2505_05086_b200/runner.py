@@ -71,6 +71,16 @@ class LayerRunner:
                                self.ws_c.data_ptr(), self.ws_c.numel(), _stream_handle(stream))
         self.cur = 1 - self.cur
 
+    def init_factors_seeded(self, act: torch.Tensor, seed: int, stream=None):
+        """Cold start with the library's counter-based Gaussian test matrices (allocates its scratch once)."""
+        need = self.plan.init_seeded_ws_bytes()
+        if getattr(self, "ws_seed", None) is None or self.ws_seed.numel() < need:
+            self.ws_seed = torch.empty(need, dtype=torch.uint8, device=self.core.device)
+        new = self.U[1 - self.cur]
+        self.plan.init_factors_seeded(act.data_ptr(), seed, new.data_ptr(), self.core.data_ptr(),
+                                      self.ws_seed.data_ptr(), self.ws_seed.numel(), _stream_handle(stream))
+        self.cur = 1 - self.cur
+
     def wgrad(self, dY: torch.Tensor, stream=None):
         self.plan.wgrad(self.core.data_ptr(), self.U[self.cur].data_ptr(), dY.data_ptr(),
                         self.dW.data_ptr(), self.ws_w.data_ptr(), self.ws_w.numel(),
