@@ -121,6 +121,12 @@ LINEAR = [  # (dims, ranks, cout, rho, generating ranks)
     ((6, 37, 50), (3, 5, 7), 21, (0.5, 0.67, 0.7), (6, 10, 14)),
     ((45, 33), (6, 9), 17, (0.9, 0.9), (12, 12)),
     ((8, 40, 130), (4, 16, 64), 40, (0.8, 0.95, 0.985), (8, 32, 128)),
+    # batch modes of 12 / 20 / 3 rows on the register-streaming kernel (two, four and one lane per column quad;
+    # the last row group of the 20-row case is idle, the 3-row case re-reads its last row; 450 quads leave a
+    # ragged warp), a 100-long token mode on the cluster mode product, 128 leading indices split in two shares
+    ((12, 100, 64), (5, 12, 8), 24, (0.75, 0.9, 0.85), (10, 24, 16)),
+    ((20, 24, 36), (8, 16, 8), 40, (0.85, 0.93, 0.85), (16, 24, 16)),
+    ((3, 50, 36), (2, 6, 6), 19, (0.5, 0.8, 0.8), (3, 12, 12)),
 ]
 
 
@@ -151,6 +157,8 @@ LINEAR_TC = [  # (dims, ranks, cout, rho, generating ranks)
     ((2, 197, 192), (2, 32, 32), 40, (0.5, 0.96, 0.96), (2, 64, 64)),   # 197 tokens: ragged K chunks and row tiles
     ((4, 72, 128), (3, 20, 24), 24, (0.6, 0.94, 0.95), (4, 40, 48)),    # ranks 20 / 24: factors zero-padded to 32 columns
     ((3, 128, 256), (3, 20, 36), 32, (0.6, 0.94, 0.965), (3, 40, 72)),  # rank 36 padded to 48
+    ((12, 64, 128), (5, 8, 16), 24, (0.75, 0.85, 0.93), (10, 16, 32)),    # bf16 batch mode of 12 rows: two lanes per quad
+    ((24, 40, 64), (8, 8, 16), 32, (0.85, 0.85, 0.93), (16, 16, 32)),    # 24 rows: four lanes per quad, one group idle
 ]
 
 
