@@ -113,7 +113,12 @@ asi_status_t asi_plan_query(const asi_plan_t* plan, asi_plan_info_t* info);
  *   U_new   [out] device fp32, u_elems; must not alias U_prev
  *   core    [out] device fp32, core_elems
  *   ws      device scratch of at least compress_ws_bytes; contents undefined
- *           afterwards except the status word. */
+ *           afterwards except the status word.
+ * All work is ordered after what `stream` held before the call and before what is enqueued on it
+ * afterwards.  For 3-mode linear layers the passes of the modes run side by side on two streams owned
+ * by the plan (created at the plan's first call on the current device; the plan keeps using that
+ * device's streams), forked from and joined to `stream` by events, so the call may be captured into a
+ * CUDA graph like any other. */
 asi_status_t asi_compress(const asi_plan_t* plan, const void* act, const float* U_prev,
                           float* U_new, float* core, void* ws, size_t ws_bytes, void* stream);
 

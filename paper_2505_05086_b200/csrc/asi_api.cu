@@ -123,8 +123,10 @@ void layout_compress(asi_plan* pl) {
   int64_t vmax = 0;
   if (!pl->fast_compress)
     for (int m = 0; m < pl->nd; ++m) vmax = std::max<int64_t>(vmax, pl->mv[m].Q * pl->r[m]);
+  pl->fork = pl->d.kind == ASI_LINEAR && pl->nd == 3 && !pl->fast_compress && !(pl->d.flags & ASI_FLAG_GENERIC_ONLY);
   pl->off_V = off;
-  off = align_up(off + (size_t)vmax * 4, 256);
+  pl->v_stride = pl->fork ? align_up((size_t)vmax * 4, 256) : 0;
+  off = align_up(off + (size_t)vmax * 4, 256) + (pl->fork ? (size_t)(pl->nd - 1) * pl->v_stride : 0);
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
     const int64_t kchunks = (v.a + kExpandKC - 1) / kExpandKC;
@@ -171,7 +173,8 @@ void layout_compress(asi_plan* pl) {
       pl->tc_mode[m] = last ? 1 : 2;
       pl->tc_bytes = std::max(pl->tc_bytes, tc_scratch_bytes(std::max(v.a, v.Q), pl->r[m]));
     }
-  off = align_up(off + pl->tc_bytes, 256);
+  pl->tc_stride = pl->fork ? align_up(pl->tc_bytes, 256) : 0;
+  off = align_up(off + pl->tc_bytes, 256) + (pl->fork ? (size_t)(pl->nd - 1) * pl->tc_stride : 0);
   pl->off_Rf = off;                                   // Cholesky factors of the fused path
   off = align_up(off + (size_t)ASI_MAX_MODES * kRfStride * 8, 256);
   for (int m = 0; m < ASI_MAX_MODES; ++m) pl->off_Pg[m] = 0;
@@ -525,8 +528,34 @@ asi_status_t finish_compress(const asi_plan* pl, const void* act, float* U_new, 
   return ASI_OK;
 }
 
+std::mutex g_fork_mu;
+
+// The plan's side streams and events, created on first use for the current device.  false: run the modes one
+// after another on the caller's stream (creation failed once, or the plan was first used on another device).
+bool fork_ready(const asi_plan* pl) {
+  if (!pl->fork) return false;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(g_fork_mu);
+  asi_plan::ForkRes& f = pl->fr;
+  if (f.failed) return false;
+  if (f.ready) return f.device == dev;
+  bool ok = cudaEventCreateWithFlags(&f.fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < pl->nd - 1; ++i)
+    ok = cudaStreamCreateWithFlags(&f.side[i], cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&f.join[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    (void)cudaGetLastError();
+    f.failed = true;
+    return false;
+  }
+  f.device = dev;
+  f.ready = true;
+  return true;
+}
+
 asi_status_t expand_mode(const asi_plan* pl, int m, const void* act, const float* V, char* w,
-                         cudaStream_t st) {
+                         cudaStream_t st, int slot = 0) {
   const ModeView& v = pl->mv[m];
   ExpandArgs e;
   e.X = act;
@@ -539,7 +568,7 @@ asi_status_t expand_mode(const asi_plan* pl, int m, const void* act, const float
   e.r = v.r;
   e.nsplit = pl->nsplit[m];
   e.q_per_split = pl->q_per_split[m];
-  e.tc_scratch = w + pl->off_tc;
+  e.tc_scratch = w + pl->off_tc + (size_t)slot * pl->tc_stride;
   e.tc_scratch_bytes = pl->tc_bytes;
   e.status = reinterpret_cast<int*>(w);
   ASI_CUDA(launch_expand(e, pl->bf16, st));
@@ -634,6 +663,13 @@ asi_status_t asi_plan_create(const asi_layer_desc_t* desc, asi_plan_t** out) {
 
 asi_status_t asi_plan_destroy(asi_plan_t* plan) {
   if (!plan) return ASI_ERR_INVALID_ARG;
+  if (plan->fr.ready) {
+    for (int i = 0; i < plan->nd - 1; ++i) {
+      cudaStreamDestroy(plan->fr.side[i]);
+      cudaEventDestroy(plan->fr.join[i]);
+    }
+    cudaEventDestroy(plan->fr.fork);
+  }
   delete plan;
   return ASI_OK;
 }
@@ -690,8 +726,9 @@ int32_t asi_launch_count(const asi_plan_t* pl, int32_t which) {
   return which == 0 ? pl->launches_compress : pl->launches_wgrad;
 }
 
-asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_prev, float* U_new,
-                          float* core, void* ws, size_t ws_bytes, void* stream) {
+// allow_fork: the passes of a token layer's modes may run side by side on the plan's own streams
+static asi_status_t compress_impl(const asi_plan_t* pl, const void* act, const float* U_prev, float* U_new,
+                                  float* core, void* ws, size_t ws_bytes, void* stream, bool allow_fork) {
   if (!pl || !valid_ptr(act) || !valid_ptr(U_prev) || !valid_ptr(U_new) || !valid_ptr(core))
     return ASI_ERR_INVALID_ARG;
   if (U_prev == U_new) return ASI_ERR_INVALID_ARG;
@@ -709,6 +746,12 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
   }
   ASI_CUDA(cudaMemsetAsync(w, 0, kStatusBytes, st));
   float* V = reinterpret_cast<float*>(w + pl->off_V);
+  const bool forked = allow_fork && fork_ready(pl);
+  if (forked) {
+    ASI_CUDA(cudaEventRecord(pl->fr.fork, st));
+    for (int i = 0; i < pl->nd - 1; ++i) ASI_CUDA(cudaStreamWaitEvent(pl->fr.side[i], pl->fr.fork, 0));
+  }
+  const cudaStream_t st0 = st;
   if (pl->plane) {
     PlaneArgs g;
     g.X = act;
@@ -729,9 +772,14 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
       ASI_CUDA(launch_plane(g, pl->plane_grid, pl->bf16, st));
     }
   }
+  for (int m = 0; m < pl->nd; ++m)                   // argument errors before anything is forked
+    if (pl->fiber2[m] && !(pl->plane && m >= 2) && (reinterpret_cast<uintptr_t>(act) & 15u)) return ASI_ERR_INVALID_ARG;
   for (int m = 0; m < pl->nd; ++m) {
     const ModeView& v = pl->mv[m];
     if (pl->plane && m >= 2) continue;
+    const int slot = forked ? m : 0;                 // scratch and stream of this mode's pass
+    st = (forked && m > 0) ? pl->fr.side[m - 1] : st0;
+    V = reinterpret_cast<float*>(w + pl->off_V + (size_t)slot * pl->v_stride);
     if (pl->fiber2[m]) {
       if (reinterpret_cast<uintptr_t>(act) & 15u) return ASI_ERR_INVALID_ARG;
       Fiber2Args f;
@@ -773,15 +821,26 @@ asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_
     a.so = v.I * v.r;
     a.sj = 1;
     a.si = v.r;
-    a.tc_scratch = w + pl->off_tc;
+    a.tc_scratch = w + pl->off_tc + (size_t)slot * pl->tc_stride;
     a.tc_scratch_bytes = pl->tc_bytes;
     a.status = reinterpret_cast<int*>(w);
     ASI_CUDA(launch_modeprod(a, pl->bf16, st));
     // P = A_m V
-    s = expand_mode(pl, m, act, V, w, st);
+    s = expand_mode(pl, m, act, V, w, st, slot);
     if (s != ASI_OK) return s;
   }
+  st = st0;
+  if (forked)
+    for (int i = 0; i < pl->nd - 1; ++i) {
+      ASI_CUDA(cudaEventRecord(pl->fr.join[i], pl->fr.side[i]));
+      ASI_CUDA(cudaStreamWaitEvent(st, pl->fr.join[i], 0));
+    }
   return finish_compress(pl, act, U_new, core, w, nullptr, st);
+}
+
+asi_status_t asi_compress(const asi_plan_t* pl, const void* act, const float* U_prev, float* U_new,
+                          float* core, void* ws, size_t ws_bytes, void* stream) {
+  return compress_impl(pl, act, U_prev, U_new, core, ws, ws_bytes, stream, true);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -924,7 +983,7 @@ asi_status_t asi_compress_static_ws(const asi_plan_t* pl, const void* act, const
   }
   // asi_compress clears the status word and the completion counters itself; everything else in the
   // array is written before it is read.
-  return asi_compress(pl, act, U_prev, U_new, core, ws, (size_t)ASI_STATIC_WS_MAX_BYTES, stream);
+  return compress_impl(pl, act, U_prev, U_new, core, ws, (size_t)ASI_STATIC_WS_MAX_BYTES, stream, false);
 }
 
 asi_status_t asi_init_factors(const asi_plan_t* pl, const void* act, const float* omega, float* U_new,

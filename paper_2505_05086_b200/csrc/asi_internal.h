@@ -308,6 +308,18 @@ struct asi_plan {
   size_t off_V, off_Pp[ASI_MAX_MODES], off_Pred[ASI_MAX_MODES], off_Gp[ASI_MAX_MODES], off_T[2];
   size_t off_Rf, off_Pg[ASI_MAX_MODES];
   size_t off_tc, tc_bytes;         // bf16 operand of the tensor-core products (0 bytes: not used)
+  // Token layers run the passes of their modes side by side (they read the same activation and write disjoint
+  // scratch): mode m > 0 is enqueued on a stream of the plan's own that forks from and joins the caller's
+  // stream by events.  Each mode then has its own V and operand scratch (strides below; 0 when not forked).
+  bool fork;
+  size_t v_stride, tc_stride;
+  struct ForkRes {
+    cudaStream_t side[ASI_MAX_MODES - 1];
+    cudaEvent_t fork, join[ASI_MAX_MODES - 1];
+    int device;
+    bool ready, failed;
+  };
+  mutable ForkRes fr;              // created at the first forked call (under a library-wide lock)
   int tc_mode[ASI_MAX_MODES];      // 0: SIMT, 1: last-mode tensor-core kernels, 2: inner-extent (token) kernels
   int nsplit[ASI_MAX_MODES], nchunk[ASI_MAX_MODES];
   int64_t q_per_split[ASI_MAX_MODES];
