@@ -421,3 +421,46 @@ def test_cuda_graph_replay_matches_direct_launches():
         assert torch.equal(run.U[run.cur], ref[0])
         assert torch.equal(run.core, ref[1])
         assert torch.equal(run.dW, ref[2])
+
+
+def test_cuda_graph_replay_of_a_token_layer_matches_direct_launches():
+    """A 3-mode linear layer runs the passes of its modes on streams of the plan's own, forked from and joined
+    to the caller's stream: captured, these become parallel branches of the graph.  The replay (and a second
+    direct call) must give the bits of the first direct call."""
+    dims, ranks = (4, 72, 128), (3, 16, 16)
+    L = LayerSpec("t", "linear", dims, 24, ranks=ranks)
+    st = LayerStream(dims=dims, ranks=ranks, dy_shape=L.dy_shape, seed=151, rho=(0.6, 0.93, 0.93),
+                     gen_ranks=(4, 32, 32), bf16=True)
+    A, dY = st.next()
+    run = make_runner(L, bf16=True)
+    a, d = run.to_device(A), run.to_device(dY)
+    refs = []
+    for _ in range(2):
+        run.set_factors(st.u_prev0())
+        run.compress(a)
+        run.wgrad(d)
+        torch.cuda.synchronize()
+        assert run.ok()
+        refs.append((run.U[run.cur].clone(), run.core.clone(), run.dW.clone()))
+        run.cur = 1 - run.cur
+    for x, y in zip(*refs):
+        assert torch.equal(x, y)
+    run.set_factors(st.u_prev0())
+    s = torch.cuda.Stream()
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        cur = torch.cuda.current_stream()
+        side.wait_stream(cur)
+        run.compress(a, side)
+        run.wgrad(d, side)
+        cur.wait_stream(side)
+    for _ in range(2):
+        run.core.zero_()
+        run.dW.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert run.ok()
+        assert torch.equal(run.U[run.cur], refs[0][0])
+        assert torch.equal(run.core, refs[0][1])
+        assert torch.equal(run.dW, refs[0][2])
