@@ -120,27 +120,20 @@ __global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
   const int tpo = (int)((p.I + TQ - 1) / TQ);        // tiles per outer index (< 2^31: checked on the host)
   const int nt = (int)p.n_tiles, gs = (int)gridDim.x;
 
-  // A thread copies the same 16-byte unit of every KSTEP-th row: unit u of rows k0, k0 + KSTEP, ...  The
-  // shared-memory address is a 32-bit base plus compile-time offsets; rows past a_m get a zero-size copy (they
-  // hold zeros anyway), so the loop has a fixed trip count.
-  constexpr int KSTEP = NT / UPR, NK = AR / KSTEP;
-  static_assert(AR % KSTEP == 0, "whole steps");
+  // A thread copies the same 16-byte unit of every KSTEP-th row: unit u of rows k0, k0 + KSTEP, ...
+  constexpr int KSTEP = NT / UPR;
   const int cu = tid % UPR, ck0 = tid / UPR;
   const int64_t src_row_step = (int64_t)KSTEP * p.I;
-  const uint32_t dst0 = smem_u32(stages) + (uint32_t)((ck0 * TQ + cu * EPU) * sizeof(TX));
   auto issue = [&](int o, int ic, int st) {
     const int64_t i0 = (int64_t)ic * TQ;
     const int ncol = (int)((p.I - i0 < TQ) ? (p.I - i0) : TQ);
     const bool on = cu * EPU < ncol;
-    const TX* src = X + ((int64_t)o * a + (ck0 < a ? ck0 : a - 1)) * p.I + i0 + (on ? cu * EPU : 0);
-    const uint32_t dst = dst0 + (uint32_t)st * (uint32_t)stage_bytes;
-#pragma unroll
-    for (int i = 0; i < NK; ++i) {
-      const bool row = ck0 + i * KSTEP < a;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + (uint32_t)(i * KSTEP * TQ * sizeof(TX))),
-                   "l"(src), "r"((on && row) ? 16 : 0)
-                   : "memory");
-      if (ck0 + (i + 1) * KSTEP < a) src += src_row_step;     // stays on a valid row
+    const TX* src = X + ((int64_t)o * a + ck0) * p.I + i0 + (on ? cu * EPU : 0);
+    TX* dst = reinterpret_cast<TX*>(stages + (size_t)st * stage_bytes) + ck0 * TQ + cu * EPU;
+    for (int k = ck0; k < a; k += KSTEP) {
+      cp_async16(dst, src, on);
+      src += src_row_step;
+      dst += KSTEP * TQ;
     }
   };
   // (o, ic) of a tile index advance by gs tiles at a time without divisions
@@ -284,7 +277,7 @@ size_t fiber2_smem(int a, int rw, int nj, int nstage, bool bf16) {
 
 int fiber2_rows_per_group(int a) {
   const int rw = (a + kF2Groups - 1) / kF2Groups;
-  return rw <= 4 ? 4 : 8;
+  return rw <= 1 ? 1 : (rw <= 2 ? 2 : (rw <= 4 ? 4 : 8));
 }
 
 // as many stages (2..4) as leave room for two CTAs per SM
@@ -328,12 +321,19 @@ cudaError_t launch_fiber2(const Fiber2Args& p0, int grid, bool bf16, cudaStream_
   ProfScope prof(p.project_only ? ASI_K_MODEPROD : ASI_K_EXPAND, st, xbytes);
 #define ASI_F2(RW_, NJ_)                                                                        \
   return bf16 ? launch_fiber2_t<RW_, NJ_, __nv_bfloat16>(p, grid, smem, st) : launch_fiber2_t<RW_, NJ_, float>(p, grid, smem, st)
-  // modes of up to 32 rows went to the register kernel above: four or eight rows per group remain
   if (nj == 4) {
-    if (rw <= 4) ASI_F2(4, 4);
-    ASI_F2(8, 4);
+    switch (rw) {
+      case 1: ASI_F2(1, 4);
+      case 2: ASI_F2(2, 4);
+      case 4: ASI_F2(4, 4);
+      default: ASI_F2(8, 4);
+    }
   }
-  ASI_F2(4, 8);
+  switch (rw) {
+    case 1: ASI_F2(1, 8);
+    case 2: ASI_F2(2, 8);
+    default: ASI_F2(4, 8);
+  }
 #undef ASI_F2
 }
 
