@@ -91,7 +91,7 @@ constexpr int kF2Threads = 256, kF2Groups = 16, kF2TQ = 64;   // 16 half-warps: 
 // is far below latency x bandwidth.
 // ---------------------------------------------------------------------------------------------
 template <int RW, int NJ, typename TX>
-__global__ void __launch_bounds__(kF2Threads, 2) k_fiber2(Fiber2Args p) {
+__global__ void __launch_bounds__(kF2Threads, (RW * NJ <= 16) ? 3 : 2) k_fiber2(Fiber2Args p) {
   constexpr int TQ = kF2TQ, NT = kF2Threads, NG = kF2Groups;
   constexpr int EPU = 16 / (int)sizeof(TX);          // elements per 16-byte unit
   constexpr int UPR = TQ / EPU;                      // units per staged row
@@ -281,10 +281,14 @@ int fiber2_rows_per_group(int a) {
 }
 
 // as many stages (2..4) as leave room for two CTAs per SM
+// CTAs per SM the kernel is compiled for: three when the row accumulators are small (78 registers), else two
+int fiber2_ctas_per_sm(int rw, int nj) { return rw * nj <= 16 ? 3 : 2; }
+
 int fiber2_stages(int a, int nj, bool bf16) {
   const int rw = fiber2_rows_per_group(a);
+  const size_t cap = fiber2_ctas_per_sm(rw, nj) == 3 ? 74 * 1024 : 112 * 1024;
   int n = 4;
-  while (n > 2 && fiber2_smem(a, rw, nj, n, bf16) > 112 * 1024) --n;
+  while (n > 2 && fiber2_smem(a, rw, nj, n, bf16) > cap) --n;
   return n;
 }
 
@@ -300,7 +304,8 @@ int64_t fiber2_tiles(int64_t O, int64_t I) { return O * ((I + kF2TQ - 1) / kF2TQ
 // CTAs (= partials of P) of the kernel launch_fiber2 picks: the register kernel for short fibers
 int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
   if (fiber_reg_supported(O, a, I, r, bf16)) return fiber_reg_grid(O, a, I, r, bf16);
-  return (int)std::min<int64_t>(fiber2_tiles(O, I), 296);
+  const int per_sm = fiber2_ctas_per_sm(fiber2_rows_per_group((int)a), r <= 4 ? 4 : 8);
+  return (int)std::min<int64_t>(fiber2_tiles(O, I), 148 * per_sm);
 }
 
 template <int RW, int NJ, typename TX>
