@@ -86,9 +86,8 @@ constexpr int kF2Threads = 256, kF2Groups = 16, kF2TQ = 64;   // 16 half-warps: 
 
 // ---------------------------------------------------------------------------------------------
 // k_fiber2.  256 threads = 16 half-warps; half-warp g owns rows [g RW, g RW + RW) of the tile, its lane l the
-// four columns 4l..4l+3 (a tile is 64 columns wide).  Two CTAs share an SM and every CTA keeps up to three
-// further tiles in flight (16-byte cp.async), which is what keeps HBM busy: one 32 KB tile per SM in flight
-// is far below latency x bandwidth.
+// four columns 4l..4l+3 (a tile is 64 columns wide).  Two or three CTAs share an SM and every CTA keeps one
+// further tile in flight (16-byte cp.async).
 // ---------------------------------------------------------------------------------------------
 template <int RW, int NJ, typename TX>
 __global__ void __launch_bounds__(kF2Threads, (RW * NJ <= 16) ? 3 : 2) k_fiber2(Fiber2Args p) {
@@ -284,12 +283,12 @@ int fiber2_rows_per_group(int a) {
 // CTAs per SM the kernel is compiled for: three when the row accumulators are small (78 registers), else two
 int fiber2_ctas_per_sm(int rw, int nj) { return rw * nj <= 16 ? 3 : 2; }
 
+// Two stages: one tile in flight per CTA while the other is used.  Deeper pipelines (3-4 stages) ran the kernel
+// alone no faster, and their larger footprint kept other kernels of the same step off the SMs: the step of ten
+// layers replayed as a graph was 2 % slower with them.
 int fiber2_stages(int a, int nj, bool bf16) {
-  const int rw = fiber2_rows_per_group(a);
-  const size_t cap = fiber2_ctas_per_sm(rw, nj) == 3 ? 74 * 1024 : 112 * 1024;
-  int n = 4;
-  while (n > 2 && fiber2_smem(a, rw, nj, n, bf16) > cap) --n;
-  return n;
+  (void)a; (void)nj; (void)bf16;
+  return 2;
 }
 
 // ranks up to 4 for a <= 128, up to 8 for a <= 64 (the register budget of the row accumulators)
@@ -354,7 +353,7 @@ cudaError_t launch_fiber2(const Fiber2Args& p0, int grid, bool bf16, cudaStream_
 // through the bulk-copy engine (cp.async.bulk + mbarrier, bounded waits).
 // ---------------------------------------------------------------------------------------------
 namespace {
-constexpr int kP2Threads = 224, kP2Stages = 3;
+constexpr int kP2Threads = 224, kP2Stages = 2;   // a third stage bought nothing
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
