@@ -323,6 +323,7 @@ class Workload:
     """Device-resident inputs, runners and CUDA graphs of one configuration."""
 
     def __init__(self, ci, dev, use_graph, torch, n_host_sets=0):
+        from paper_2505_05086_b200.binding import ASI_FLAG_SHARE_SM
         from paper_2505_05086_b200.runner import LayerRunner, StepRunner
         self.ci, self.cfg, self.torch = ci, get_config(ci), torch
         cfg = self.cfg
@@ -332,11 +333,19 @@ class Workload:
         sets = int(np.ceil(3.0 * L2_BYTES / self.set_bytes))
         self.sets = max(2, min(8, sets + sets % 2))
         self.runners, self.acts, self.dys, self.host = [], [], [], []
+        self.graph_runners = []
         for li, L in enumerate(cfg.layers):
             st = make_stream(cfg, li)
             r = LayerRunner("linear" if L.kind == "linear" else "conv", L.dims, L.ranks, L.cout, k=L.k,
                             stride=L.stride, pad=L.pad, groups=L.groups, bf16=cfg.bf16, device=dev)
             r.set_factors(st.u_prev0())
+            if use_graph:
+                # the graph runs the layers side by side: its plans leave room on every SM for the neighbours
+                g = LayerRunner("linear" if L.kind == "linear" else "conv", L.dims, L.ranks, L.cout, k=L.k,
+                                stride=L.stride, pad=L.pad, groups=L.groups, bf16=cfg.bf16, device=dev,
+                                flags=ASI_FLAG_SHARE_SM)
+                g.set_factors(st.u_prev0())
+                self.graph_runners.append(g)
             a_l, d_l, h_l = [], [], []
             for s in range(self.sets):
                 A, dY = st.next()
@@ -355,7 +364,7 @@ class Workload:
         # measured faster than the batched launches on one branch, whose kernel stages run one after the other
         self.side = [torch.cuda.Stream(device=dev) for _ in range(self.nl)]
         self.launches_per_step = (self._count_launches() if not use_graph else
-                                  sum(r.plan.launch_count(0) + r.plan.launch_count(1) for r in self.runners))
+                                  sum(r.plan.launch_count(0) + r.plan.launch_count(1) for r in self.graph_runners))
         with torch.cuda.stream(self.stream):
             for i in range(2):
                 self.step_direct(i)
@@ -371,9 +380,9 @@ class Workload:
                     cur = torch.cuda.current_stream()
                     for li in range(self.nl):
                         self.side[li].wait_stream(cur)
-                        self.runners[li].compress(self.acts[li][s], self.side[li])
+                        self.graph_runners[li].compress(self.acts[li][s], self.side[li])
                     for li in reversed(range(self.nl)):
-                        self.runners[li].wgrad(self.dys[li][s], self.side[li])
+                        self.graph_runners[li].wgrad(self.dys[li][s], self.side[li])
                     for li in range(self.nl):
                         cur.wait_stream(self.side[li])
                 self.graphs.append(g)
@@ -411,11 +420,11 @@ class Workload:
             self.graphs[i % self.sets].replay()
 
     def ok(self):
-        return all(r.ok() for r in self.runners)
+        return all(r.ok() for r in self.runners) and all(r.ok() for r in self.graph_runners)
 
     def free(self):
         self.graphs = None
-        self.runners = self.acts = self.dys = self.host = None
+        self.runners = self.graph_runners = self.acts = self.dys = self.host = None
         self.torch.cuda.empty_cache()
 
 
@@ -641,7 +650,7 @@ def run_ours(args):
                    "l2_policy": f"inputs larger than L2: {head['input_sets']} rotating input sets, "
                                 f"{head['input_bytes_rotated'] / 1e6:.0f} MB of act+dY",
                    "launch": ("asi_compress_batched + asi_wgrad_batched on one stream" if args.no_graph else
-                              "CUDA-graph replay, one graph per input set, one branch per layer"),
+                              "CUDA-graph replay, one graph per input set, one branch per layer, plans with ASI_FLAG_SHARE_SM"),
                    "single_stream_launch": "asi_compress_batched + asi_wgrad_batched, one call each per step",
                    "timing": f"{head['timed_blocks']} blocks of {args.steps} steps, {head['timed_ms_total']:.0f} ms "
                              f"of device time; ms_per_step = median block / steps",

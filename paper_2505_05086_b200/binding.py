@@ -26,7 +26,7 @@ ASI_F32, ASI_BF16 = 0, 1
 ASI_CONV2D, ASI_LINEAR = 0, 1
 ASI_MAX_MODES = 4
 ASI_STATIC_WS_MAX_BYTES = 4 << 20
-ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT = 1, 2
+ASI_FLAG_GENERIC_ONLY, ASI_FLAG_TEST_EXPIRE_WAIT, ASI_FLAG_SHARE_SM = 1, 2, 4
 
 EXPORTS = (
     "asi_plan_create", "asi_plan_destroy", "asi_plan_query", "asi_compress", "asi_compress_static_ws",

@@ -113,12 +113,14 @@ void layout_compress(asi_plan* pl) {
   for (int m = 0; m < ASI_MAX_MODES; ++m) pl->fiber2[m] = false;
   if (pl->plane && plane2_supported((int)pl->dims[2], pl->dims[0] * pl->dims[1], pl->r[2], pl->r[3])) {
     pl->plane2 = true;
-    pl->plane_grid = plane2_grid((int)pl->dims[2], pl->dims[0] * pl->dims[1], 296);
+    pl->plane_grid = plane2_grid((int)pl->dims[2], pl->dims[0] * pl->dims[1],
+                                 (pl->d.flags & ASI_FLAG_SHARE_SM) ? 148 : 296);
   }
   for (int m = 0; m < pl->nd; ++m)
     if (pl->fiber[m] && fiber2_supported(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16)) {
       pl->fiber2[m] = true;
-      pl->fiber_grid[m] = fiber2_grid(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16);
+      pl->fiber_grid[m] = fiber2_grid(pl->mv[m].O, pl->mv[m].a, pl->mv[m].I, pl->r[m], pl->bf16,
+                                      (pl->d.flags & ASI_FLAG_SHARE_SM) != 0);
     }
   int64_t vmax = 0;
   if (!pl->fast_compress)
@@ -467,7 +469,8 @@ cudaError_t stream_modeprod(const asi_plan* pl, const ModeProdArgs& a, bool x_bf
   f.O = a.O; f.I = a.I; f.a = (int)a.a; f.r = a.n_out;
   f.n_tiles = fiber2_tiles(a.O, a.I);
   f.project_only = 1;
-  return launch_fiber2(f, fiber2_grid(a.O, a.a, a.I, a.n_out, x_bf16), x_bf16, st);
+  return launch_fiber2(f, fiber2_grid(a.O, a.a, a.I, a.n_out, x_bf16, (pl->d.flags & ASI_FLAG_SHARE_SM) != 0),
+                       x_bf16, st);
 }
 
 // Orthogonalize, then core = A x_1 U_1^T ... x_n U_n^T (Algorithm 1, core update with U^T).

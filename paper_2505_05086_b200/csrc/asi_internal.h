@@ -233,7 +233,7 @@ cudaError_t launch_plane(const PlaneArgs& p, int grid, bool x_bf16, cudaStream_t
 size_t plane_smem(int S);
 bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16);
 int64_t fiber2_tiles(int64_t O, int64_t I);
-int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16);
+int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16, bool share_sm);
 bool fiber_reg_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16);
 int fiber_reg_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16);
 cudaError_t launch_fiber_reg(const Fiber2Args& p, int grid, bool bf16, cudaStream_t st);

@@ -301,9 +301,12 @@ bool fiber2_supported(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
 int64_t fiber2_tiles(int64_t O, int64_t I) { return O * ((I + kF2TQ - 1) / kF2TQ); }
 
 // CTAs (= partials of P) of the kernel launch_fiber2 picks: the register kernel for short fibers
-int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16) {
+// share_sm: the variant that fills an SM's registers with two CTAs launches one per SM (other layers' kernels
+// are expected beside it)
+int fiber2_grid(int64_t O, int64_t a, int64_t I, int r, bool bf16, bool share_sm) {
   if (fiber_reg_supported(O, a, I, r, bf16)) return fiber_reg_grid(O, a, I, r, bf16);
-  const int per_sm = fiber2_ctas_per_sm(fiber2_rows_per_group((int)a), r <= 4 ? 4 : 8);
+  int per_sm = fiber2_ctas_per_sm(fiber2_rows_per_group((int)a), r <= 4 ? 4 : 8);
+  if (share_sm && per_sm == 2) per_sm = 1;
   return (int)std::min<int64_t>(fiber2_tiles(O, I), 148 * per_sm);
 }
 

@@ -18,11 +18,11 @@ class LayerRunner:
     workspaces) and the calls that fill them."""
 
     def __init__(self, kind, dims, ranks, cout, k=1, stride=1, pad=0, groups=1, bf16=False,
-                 device="cuda:0", generic_only=False):
+                 device="cuda:0", generic_only=False, flags=0):
         if not torch.cuda.is_available():
             raise RuntimeError("the ASI path needs a CUDA device; there is no CPU fallback")
         self.plan = Plan(kind, dims, ranks, cout, k, stride, pad, groups, bf16,
-                         generic_only=generic_only)
+                         generic_only=generic_only, flags=flags)
         self.dims, self.ranks, self.bf16 = tuple(dims), tuple(ranks), bf16
         self.device = torch.device(device)
         info = self.plan.info

@@ -89,3 +89,21 @@ def test_config5_vit_mlp_bf16(li):
 @pytest.mark.parametrize("li", [0, 1, 2])
 def test_config6_llm_tokens_bf16(li):
     _layer_steps(get_config(5), li, 2, TOL_BF16)
+
+
+def test_share_sm_plans_match_the_oracle_on_a_large_map():
+    """ASI_FLAG_SHARE_SM changes only the CTA counts of the streaming kernels (and with them the number of
+    partial sums): same tolerances on a 28 x 28 layer of the sweep, sampled at its first step."""
+    from paper_2505_05086_b200.binding import ASI_FLAG_SHARE_SM
+    from paper_2505_05086_b200.runner import LayerRunner
+    cfg = get_config(3)
+    li = next(i for i, L in enumerate(cfg.layers) if L.dims[2] == 28)
+    L = cfg.layers[li]
+    st = make_stream(cfg, li)
+    U_prev = st.u_prev0()
+    A, dY = st.next()
+    run = LayerRunner("conv", L.dims, L.ranks, L.cout, k=L.k, stride=L.stride, pad=L.pad, groups=L.groups,
+                      flags=ASI_FLAG_SHARE_SM)
+    err, _ = compare_step(run, L, A, dY, U_prev)
+    check(err, TOL_F32, f"share-sm {L.dims}")
+    assert run.ok()
