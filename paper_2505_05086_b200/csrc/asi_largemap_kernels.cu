@@ -90,7 +90,7 @@ constexpr int kF2Threads = 256, kF2Groups = 16, kF2TQ = 64;   // 16 half-warps: 
 // further tile in flight (16-byte cp.async).
 // ---------------------------------------------------------------------------------------------
 template <int RW, int NJ, typename TX>
-__global__ void __launch_bounds__(kF2Threads, (RW * NJ <= 16) ? 3 : 2) k_fiber2(Fiber2Args p) {
+__global__ void __launch_bounds__(kF2Threads, (RW <= 4 && NJ == 4) ? 3 : 2) k_fiber2(Fiber2Args p) {
   constexpr int TQ = kF2TQ, NT = kF2Threads, NG = kF2Groups;
   constexpr int EPU = 16 / (int)sizeof(TX);          // elements per 16-byte unit
   constexpr int UPR = TQ / EPU;                      // units per staged row
@@ -281,7 +281,7 @@ int fiber2_rows_per_group(int a) {
 
 // as many stages (2..4) as leave room for two CTAs per SM
 // CTAs per SM the kernel is compiled for: three when the row accumulators are small (78 registers), else two
-int fiber2_ctas_per_sm(int rw, int nj) { return rw * nj <= 16 ? 3 : 2; }
+int fiber2_ctas_per_sm(int rw, int nj) { return (rw <= 4 && nj == 4) ? 3 : 2; }
 
 // Two stages: one tile in flight per CTA while the other is used.  Deeper pipelines (3-4 stages) ran the kernel
 // alone no faster, and their larger footprint kept other kernels of the same step off the SMs: the step of ten
